@@ -1,0 +1,275 @@
+"""CPU oracle for LoRC latent-KV decode attention (arXiv 2410.03111).
+
+TEST INFRASTRUCTURE ONLY.  This is a plain, slow, fp64 numpy restatement of what
+the paper's method computes on the decode path.  It exists to judge the CUDA
+library and to be timed as a CPU baseline; the product never imports it, and it
+imports nothing from the product.  No blocking, fusion or re-association beyond
+what the paper states: keys and values are reconstructed explicitly from the
+cached latents, rotated, and fed to the textbook attention formula.
+
+Notation (row-vector convention, K = X W_k as in the Preliminary section):
+  D        model dimension            n = H_kv * d_h   width of the concatenated KV heads
+  W [D,n]  key or value weight        W ~= A B,  A = U_r Sigma_r [D,r],  B = V_r^T [r,n]
+  C = X A  the latent ("compressed") cache row, width r = d_c        (Sec. 3.1)
+
+Every function is pinned by tests/test_oracle_pins.py to something the paper or
+the mathematics fixes (full-rank identity, Eckart-Young, Theorem 1, RoPE closed
+forms, brute-force attention, a library attention routine).  The numeric
+tolerance used when comparing the GPU to this oracle is not from the paper
+(parity tolerance unpinned by the paper; fixed by the build's target).
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+ROPE_HALF_SPLIT = 0    # pairs (j, j + d_h/2)
+ROPE_INTERLEAVED = 1   # pairs (2j, 2j + 1)
+
+
+# --------------------------------------------------------------------------
+# rounding
+# --------------------------------------------------------------------------
+def bf16_round(x: np.ndarray) -> np.ndarray:
+    """Nearest bfloat16 value (round to nearest, ties to even) of fp64 x, as fp64.
+
+    bfloat16 keeps 8 significant bits over the float32 exponent range, so the
+    spacing at |x| in [2^e, 2^(e+1)) is 2^(e-7), with e floored at -126
+    (subnormals).  Rounding is done straight from fp64 (no float32 detour).
+    The paper is silent on the cache precision; bf16 is the build's reading.
+    """
+    x = np.asarray(x, dtype=np.float64)
+    _, ex = np.frexp(x)                      # x = m * 2^ex, 0.5 <= |m| < 1
+    e = np.maximum(ex - 1, -126)
+    quantum = np.ldexp(1.0, e - 7)
+    y = np.rint(x / quantum) * quantum       # np.rint rounds half to even
+    big = 3.3895313892515355e38              # largest finite bf16
+    y = np.where(np.abs(y) > big, np.copysign(np.inf, y), y)
+    return np.where(x == 0.0, x, y)
+
+
+# --------------------------------------------------------------------------
+# factorisation (offline step; Sec. 3.1, Algorithm 1 "Key/Value Matrix Compression")
+# --------------------------------------------------------------------------
+def truncated_svd_factors(W: np.ndarray, r: int):
+    """Rank-r factors of W [D,n]: A = U_r Sigma_r [D,r], B = V_r^T [r,n].
+
+    Sec. 3.1 (the SVD equations for W_k^H and W_v^H) splits W into an
+    orthonormal factor and a Sigma-carrying factor, and caches the product of X
+    with the Sigma-carrying one.  In the row-vector convention K = X W used
+    here, that cached quantity is X (U_r Sigma_r): Sigma stays on the cached
+    side, the orthonormal factor V_r^T is applied at attention time.
+    """
+    U, s, Vt = np.linalg.svd(np.asarray(W, dtype=np.float64), full_matrices=False)
+    return U[:, :r] * s[None, :r], Vt[:r, :].copy()
+
+
+def factors_from_generators(U: np.ndarray, sigma: np.ndarray, V: np.ndarray, r: int):
+    """Same factors when W = U diag(sigma) V^T is given by its SVD (sigma descending).
+
+    Avoids the sign/rotation freedom of a numerical SVD: A = U[:, :r] diag(sigma[:r]),
+    B = V[:, :r]^T.
+    """
+    return U[:, :r] * np.asarray(sigma, dtype=np.float64)[None, :r], V[:, :r].T.copy()
+
+
+def relative_frobenius_error(M: np.ndarray, M_hat: np.ndarray) -> float:
+    """epsilon = ||M - M_hat||_F / ||M||_F  (Appendix "Reconstruction Error of Matrix SVD")."""
+    M = np.asarray(M, dtype=np.float64)
+    d = M - np.asarray(M_hat, dtype=np.float64)
+    return math.sqrt(float(np.sum(d * d))) / math.sqrt(float(np.sum(M * M)))
+
+
+def kv_cache_elements(b: int, N: int, h: int, d: int) -> int:
+    """Per-layer cache size C_{k,v} = b * N * h * d (Preliminary section, cache-size equation)."""
+    return b * N * h * d
+
+
+def compression_ratio(d_c: int, h: int, d: int) -> float:
+    """rho = d_c / (h * d): the retained fraction of the cache width (Sec. 3.1, "Compression Ratio")."""
+    return d_c / float(h * d)
+
+
+# --------------------------------------------------------------------------
+# cache write (Sec. 3.1: the cache keeps X times the Sigma-carrying factor, for keys and for values)
+# --------------------------------------------------------------------------
+def append_latent(x: np.ndarray, A: np.ndarray) -> np.ndarray:
+    """Exact latent rows C = X A, fp64, [n_tok, r].  No rotation is applied (Appendix
+    "Adjusted Position Embedding": the cache holds un-rotated compressed keys)."""
+    return np.asarray(x, dtype=np.float64) @ np.asarray(A, dtype=np.float64)
+
+
+def append_latent_bf16(x: np.ndarray, A: np.ndarray) -> np.ndarray:
+    """The value a bf16 cache must hold: the exact latent rounded once to bf16."""
+    return bf16_round(append_latent(x, A))
+
+
+# --------------------------------------------------------------------------
+# rotary position embedding (Appendix "Adjusted Position Embedding", RoFormer's R_{Theta,p})
+# --------------------------------------------------------------------------
+def rope(v: np.ndarray, pos, theta: float, style: int = ROPE_HALF_SPLIT) -> np.ndarray:
+    """Apply R_{Theta,pos} to the last axis (length d_h) of v.
+
+    pos is a scalar or an array broadcastable to v.shape[:-1].  For j < d_h/2
+    the pair (a, b) = (v[j], v[j + d_h/2]) [half split] or (v[2j], v[2j+1])
+    [interleaved] is rotated by the angle pos * theta^(-2j/d_h):
+        a' = a cos - b sin,   b' = a sin + b cos.
+    Positions are 0-based.
+    """
+    v = np.asarray(v, dtype=np.float64)
+    d = v.shape[-1]
+    half = d // 2
+    j = np.arange(half, dtype=np.float64)
+    inv_freq = float(theta) ** (-2.0 * j / d)
+    ang = np.asarray(pos, dtype=np.float64)[..., None] * inv_freq
+    c, s = np.cos(ang), np.sin(ang)
+    out = np.empty_like(v)
+    if style == ROPE_HALF_SPLIT:
+        a, b = v[..., :half], v[..., half:]
+        out[..., :half] = a * c - b * s
+        out[..., half:] = a * s + b * c
+    elif style == ROPE_INTERLEAVED:
+        a, b = v[..., 0::2], v[..., 1::2]
+        out[..., 0::2] = a * c - b * s
+        out[..., 1::2] = a * s + b * c
+    else:
+        raise ValueError("unknown rope style")
+    return out
+
+
+# --------------------------------------------------------------------------
+# attention (Preliminary section, Attention(Q,K,V) = softmax(Q K^T / sqrt(d_k)) V; Sec. 3.3 GQA repeat)
+# --------------------------------------------------------------------------
+def attention_one_query(q_hat: np.ndarray, K_hat: np.ndarray, V: np.ndarray) -> np.ndarray:
+    """One decode query per head over N cached tokens.
+
+    q_hat [H_q, d_h] (already rotated), K_hat [N, H_kv, d_h] (already rotated),
+    V [N, H_kv, d_h].  Query head h uses KV head h // (H_q / H_kv): Sec. 3.3
+    replicates each fetched KV head across the query heads of its group.
+    Returns [H_q, d_h].
+    """
+    H_q, d = q_hat.shape
+    N, H_kv, _ = K_hat.shape
+    G = H_q // H_kv
+    out = np.empty((H_q, d), dtype=np.float64)
+    for h in range(H_q):
+        g = h // G
+        s = K_hat[:, g, :] @ q_hat[h] / math.sqrt(d)
+        s = s - np.max(s)
+        p = np.exp(s)
+        p = p / np.sum(p)
+        out[h] = p @ V[:, g, :]
+    return out
+
+
+def decode_attn_latent(c_k: np.ndarray, c_v: np.ndarray, B_k: np.ndarray, B_v: np.ndarray,
+                       q: np.ndarray, n_kv_heads: int, theta: float,
+                       style: int = ROPE_HALF_SPLIT, positions=None, q_position=None,
+                       use_rope: bool = True) -> np.ndarray:
+    """Decode attention of one sequence over its latent cache.
+
+    c_k [N, r_k], c_v [N, r_v]: cached latents (whatever precision the cache held,
+    passed as fp64).  B_k [r_k, n], B_v [r_v, n].  q [H_q, d_h] un-rotated.
+    Steps, in the paper's order: fetch the compressed rows; reconstruct keys and
+    values for all KV heads (K~ = C_K B_K, V~ = C_V B_V); rotate each key at its
+    own position and the query at its position (Appendix "Adjusted Position
+    Embedding"); attention with GQA repeat (Sec. 3.3).  By default the N cached
+    tokens sit at positions 0..N-1 and the query at N-1 (the token appended last).
+    """
+    c_k = np.asarray(c_k, dtype=np.float64)
+    c_v = np.asarray(c_v, dtype=np.float64)
+    q = np.asarray(q, dtype=np.float64)
+    N = c_k.shape[0]
+    H_q, d = q.shape
+    K = (c_k @ np.asarray(B_k, dtype=np.float64)).reshape(N, n_kv_heads, d)
+    V = (c_v @ np.asarray(B_v, dtype=np.float64)).reshape(N, n_kv_heads, d)
+    if positions is None:
+        positions = np.arange(N)
+    if q_position is None:
+        q_position = N - 1
+    if use_rope:
+        K = rope(K, np.asarray(positions)[:, None], theta, style)
+        q = rope(q, np.full((H_q,), q_position), theta, style)
+    return attention_one_query(q, K, V)
+
+
+def decode_attn_full(x: np.ndarray, W_k: np.ndarray, W_v: np.ndarray, q: np.ndarray,
+                     n_kv_heads: int, theta: float, style: int = ROPE_HALF_SPLIT,
+                     positions=None, q_position=None, use_rope: bool = True) -> np.ndarray:
+    """Uncompressed decode attention: K = X W_k, V = X W_v, rotate, attend.
+
+    x [N, D] are the hidden states of the N cached tokens.  This is the
+    definition the compressed path must reproduce exactly at full rank.
+    """
+    x = np.asarray(x, dtype=np.float64)
+    q = np.asarray(q, dtype=np.float64)
+    N = x.shape[0]
+    H_q, d = q.shape
+    K = (x @ np.asarray(W_k, dtype=np.float64)).reshape(N, n_kv_heads, d)
+    V = (x @ np.asarray(W_v, dtype=np.float64)).reshape(N, n_kv_heads, d)
+    if positions is None:
+        positions = np.arange(N)
+    if q_position is None:
+        q_position = N - 1
+    if use_rope:
+        K = rope(K, np.asarray(positions)[:, None], theta, style)
+        q = rope(q, np.full((H_q,), q_position), theta, style)
+    return attention_one_query(q, K, V)
+
+
+def decode_attn_cached_kv(k_rot: np.ndarray, v: np.ndarray, q: np.ndarray, theta: float,
+                          style: int = ROPE_HALF_SPLIT, q_position=None) -> np.ndarray:
+    """Attention over an uncompressed cache that already holds rotated keys.
+
+    k_rot, v [N, H_kv, d_h]; q [H_q, d_h] un-rotated, rotated here at q_position
+    (default N-1).  This is the conventional pipeline the appendix contrasts
+    with: an ordinary cache holds keys that were rotated before being stored.
+    """
+    k_rot = np.asarray(k_rot, dtype=np.float64)
+    q = np.asarray(q, dtype=np.float64)
+    N = k_rot.shape[0]
+    if q_position is None:
+        q_position = N - 1
+    qh = rope(q, np.full((q.shape[0],), q_position), theta, style)
+    return attention_one_query(qh, k_rot, np.asarray(v, dtype=np.float64))
+
+
+# --------------------------------------------------------------------------
+# batch / paged drivers (plain indexing around the functions above)
+# --------------------------------------------------------------------------
+def gather_rows(pool: np.ndarray, page_table_row: np.ndarray, length: int, page_size: int) -> np.ndarray:
+    """Rows 0..length-1 of one sequence from a paged pool [n_pages, page_size, r]."""
+    n_pg = (length + page_size - 1) // page_size
+    rows = pool[np.asarray(page_table_row[:n_pg], dtype=np.int64)].reshape(n_pg * page_size, -1)
+    return rows[:length]
+
+
+def decode_attn_latent_batch(cache_k, cache_v, seq_lens, B_k, B_v, q, n_kv_heads, theta,
+                             style=ROPE_HALF_SPLIT, page_table=None, page_size=64):
+    """Loop of decode_attn_latent over a ragged batch.
+
+    Contiguous: cache_* [b, N_max, r].  Paged: cache_* [n_pages, page_size, r] with
+    page_table [b, max_pages].  q [b, H_q, d_h].  Returns [b, H_q, d_h].
+    """
+    b = len(seq_lens)
+    out = np.empty(np.asarray(q).shape, dtype=np.float64)
+    for s in range(b):
+        L = int(seq_lens[s])
+        if page_table is None:
+            ck, cv = cache_k[s, :L], cache_v[s, :L]
+        else:
+            ck = gather_rows(cache_k, page_table[s], L, page_size)
+            cv = gather_rows(cache_v, page_table[s], L, page_size)
+        out[s] = decode_attn_latent(ck, cv, B_k, B_v, q[s], n_kv_heads, theta, style)
+    return out
+
+
+def rel_l2_rows(got: np.ndarray, want: np.ndarray) -> float:
+    """max over rows (last axis = row) of ||got - want||_2 / ||want||_2."""
+    got = np.asarray(got, dtype=np.float64)
+    want = np.asarray(want, dtype=np.float64)
+    num = np.sqrt(np.sum((got - want) ** 2, axis=-1))
+    den = np.sqrt(np.sum(want ** 2, axis=-1))
+    den = np.where(den == 0.0, 1.0, den)
+    return float(np.max(num / den))
