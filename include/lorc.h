@@ -1,0 +1,194 @@
+/*
+ * lorc.h - C ABI of the B200 (sm_100a) latent-KV decode-attention library.
+ *
+ * The library implements the run-time half of LoRC (arXiv 2410.03111): the KV
+ * cache of every layer holds rank-r latents C_K = X A_K, C_V = X A_V instead of
+ * keys and values, where W_k ~= A_K B_K and W_v ~= A_V B_V are truncated-SVD
+ * factorisations (A = U_r Sigma_r, B = V_r^T; Sec. 3.1, Algorithm 1), and decode
+ * attention runs directly on the latents.
+ *
+ * Conventions
+ *   - Row-vector convention K = X W (Preliminary section).  D = d_model,
+ *     n = n_kv_heads * d_head, query head h reads KV head h / (n_q_heads / n_kv_heads)
+ *     (Sec. 3.3).
+ *   - All tensors are dense, row-major, bfloat16 unless stated.  "device" pointers
+ *     are CUDA device memory owned by the caller; the library never frees or
+ *     reallocates caller memory.  "host" pointers are ordinary host memory.
+ *   - `stream` arguments are a cudaStream_t passed as void* (NULL = default stream).
+ *     Calls enqueue work on that stream and return without synchronising unless
+ *     stated.
+ *   - Every function returns LORC_OK (0) or a positive LORC_ERR_* code; nothing
+ *     throws, aborts or traps.  lorc_last_error() gives a text for the last failure
+ *     on that context.  Problems only a kernel can see (a page index outside the
+ *     pool, a position beyond the capacity, a bounded wait that ran out) set a
+ *     device status word that lorc_sync_status() returns.
+ *   - Positions are 0-based.  RoPE angle for pair j at position p is
+ *     p * rope_theta^(-2j/d_head).
+ */
+#ifndef LORC_H_
+#define LORC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* status codes */
+#define LORC_OK 0
+#define LORC_ERR_ARG 1          /* null pointer, bad size, bad alignment */
+#define LORC_ERR_LAYER 2        /* layer index out of range or factors not loaded */
+#define LORC_ERR_CAPACITY 3     /* position beyond cache capacity / page index outside the pool */
+#define LORC_ERR_EMPTY 4        /* a sequence with zero cached tokens was attended */
+#define LORC_ERR_TIMEOUT 5      /* a bounded device-side wait expired */
+#define LORC_ERR_CUDA 6         /* a CUDA runtime / driver call failed */
+#define LORC_ERR_UNSUPPORTED 7  /* shape outside what the kernels implement */
+#define LORC_ERR_WORKSPACE 8    /* workspace missing or too small */
+
+/* layer modes */
+#define LORC_MODE_LATENT 0      /* compressed layer: cache holds rank-r latents */
+#define LORC_MODE_FULL 1        /* layer skipped by the compression schedule: ordinary KV cache */
+
+/* RoPE pairing */
+#define LORC_ROPE_HALF_SPLIT 0  /* pair (j, j + d_head/2) */
+#define LORC_ROPE_INTERLEAVED 1 /* pair (2j, 2j + 1)      */
+
+/* context flags */
+#define LORC_FLAG_DEBUG_FP32 1  /* run the plain fp32 CUDA-core kernels everywhere (debug path) */
+
+typedef struct lorc_ctx lorc_ctx;
+
+/* Model geometry, fixed for the life of a context.  Shapes follow the paper's
+ * "Model Architectures" table (layers, heads, KV heads, head dimension, model
+ * dimension).  max_pos bounds every position used with this context (the
+ * library builds a cos/sin table of max_pos rows at creation). */
+typedef struct lorc_model_desc {
+    int32_t n_layers;
+    int32_t d_model;
+    int32_t n_q_heads;
+    int32_t n_kv_heads;
+    int32_t d_head;      /* 64 or 128 */
+    int32_t rope_style;  /* LORC_ROPE_* */
+    int32_t max_pos;     /* positions are in [0, max_pos) */
+    int32_t flags;       /* LORC_FLAG_* */
+    double rope_theta;
+} lorc_model_desc;
+
+/* One layer's cache for a batch of sequences.  The cache-size model of the
+ * Preliminary section (b x N x h x d per layer) becomes b x N x r here.
+ *
+ * Contiguous layout (page_table == NULL):
+ *     k = C_K[batch][seq_stride][r_k], v = C_V[batch][seq_stride][r_v]
+ * Paged layout (page_table != NULL):
+ *     k = pool_K[n_pages][page_size][r_k], v = pool_V[n_pages][page_size][r_v],
+ *     page_table[batch][max_pages_per_seq] (device int32) gives the physical page
+ *     of each logical page of each sequence.
+ * In LORC_MODE_FULL layers the row width is n = n_kv_heads*d_head for both, and
+ * k holds keys already rotated at their positions.
+ *
+ * seq_lens[batch] (device int32, caller-owned, never written by the library) is
+ * the number of cached tokens of each sequence.  max_seq_len is a host-side upper
+ * bound on seq_lens used to size launches; it must not exceed the capacity
+ * (seq_stride, or max_pages_per_seq*page_size).  Rows at positions >= seq_lens[s]
+ * may be read by tile loads; they must hold finite numbers (zero the cache once
+ * when allocating it). */
+typedef struct lorc_cache {
+    void* k;                      /* device */
+    void* v;                      /* device */
+    const int32_t* page_table;    /* device, or NULL for the contiguous layout */
+    const int32_t* seq_lens;      /* device */
+    int32_t batch;
+    int32_t max_seq_len;
+    int32_t page_size;            /* paged: tokens per page (multiple of 16) */
+    int32_t max_pages_per_seq;    /* paged */
+    int32_t n_pages;              /* paged: pages in the pool */
+    int32_t reserved;
+    int64_t seq_stride;           /* contiguous: rows between consecutive sequences */
+} lorc_cache;
+
+/* Create / destroy a context.  Creation allocates only library-owned tables
+ * (the cos/sin table of max_pos x d_head/2 pairs and a status word; per-layer
+ * factor copies come later, in lorc_load_factors).  Uses the current CUDA device.
+ * Errors: ARG (null, non-positive sizes, n_q_heads not a multiple of
+ * n_kv_heads), UNSUPPORTED (d_head not 64/128, more than 8 query heads per KV
+ * head), CUDA. */
+int lorc_create(const lorc_model_desc* desc, lorc_ctx** out);
+int lorc_destroy(lorc_ctx* ctx);
+
+/* Hand the factors of one layer to the library (Sec. 3.1; Algorithm 1, the two
+ * "Matrix Compression" blocks).  Setup call: it allocates library-owned device
+ * copies in the layouts the kernels want and synchronises `stream` before it
+ * returns, so the caller's buffers may be released afterwards.
+ *   mode LATENT: A_k [D, r_k], B_k [r_k, n], A_v [D, r_v], B_v [r_v, n], device bf16.
+ *                r_k, r_v in [8, n], multiples of 8.
+ *   mode FULL  : A_k = W_k [D, n], A_v = W_v [D, n]; B_k, B_v, r_k, r_v ignored
+ *                (a layer the schedule leaves uncompressed, Algorithm 1 "skip").
+ * Errors: ARG, LAYER, CUDA. */
+int lorc_load_factors(lorc_ctx* ctx, int layer, int mode, int r_k, int r_v,
+                      const void* A_k, const void* B_k, const void* A_v, const void* B_v,
+                      void* stream);
+
+/* Scratch memory for decode attention (split-context partial results) and for
+ * the host-buffer entry point (staging).  The caller allocates `bytes` of device
+ * memory (256-byte aligned) and lends it to the context until replaced or the
+ * context is destroyed.  lorc_workspace_bytes returns a size sufficient for any
+ * layer of this context with the given batch and max_seq_len. */
+size_t lorc_workspace_bytes(const lorc_ctx* ctx, int batch, int max_seq_len);
+int lorc_set_workspace(lorc_ctx* ctx, void* workspace, size_t bytes);
+
+/* Cache write (Sec. 3.1: the cache stores X times the Sigma-carrying factor;
+ * Appendix "Adjusted Position Embedding": compressed keys are stored un-rotated).
+ *   x [batch, T, D] device bf16: T new tokens for every sequence of the cache.
+ *   seq_lens must already count the new tokens: token i of sequence s is written
+ *   at position seq_lens[s] - T + i.
+ * LATENT layers write C_K = x A_K, C_V = x A_V (fp32 accumulation, one rounding
+ * to bf16).  FULL layers write RoPE(x W_k) and x W_v.
+ * Errors: ARG, LAYER, UNSUPPORTED; CAPACITY through the status word. */
+int lorc_append(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* x, int T,
+                void* stream);
+
+/* Decode attention for one layer (Preliminary section's Attention(Q,K,V) with the
+ * GQA repeat of Sec. 3.3 and the rotation placement of the appendix):
+ *   q   [batch, n_q_heads, d_head] device bf16, un-rotated, one query per sequence
+ *       at position seq_lens[s] - 1;
+ *   out [batch, n_q_heads, d_head] device bf16.
+ * For every sequence s and head h (g = KV head of h):
+ *   k_n = B_K[:, g]^T C_K[n], rotated at n;  q^ = RoPE(q, seq_lens[s]-1);
+ *   p = softmax_n(q^ . k_n / sqrt(d_head)),  out = (sum_n p_n C_V[n]) B_V[:, g]
+ * over n in [0, seq_lens[s]).  Keys and values are never written to memory.
+ * n_splits = 0 lets the library choose the split of the context; a positive value
+ * forces it (clamped to what the workspace holds).  Uses the workspace.
+ * A sequence with seq_lens[s] <= 0 gets a row of zeros and sets status EMPTY.
+ * Errors: ARG, LAYER, WORKSPACE, UNSUPPORTED. */
+int lorc_decode_attn(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* q, void* out,
+                     int n_splits, void* stream);
+
+/* One decode step of one layer from HOST buffers: copies x_host [batch, D] and
+ * q_host [batch, n_q_heads, d_head] to staging at the end of the workspace, runs
+ * lorc_append (T = 1) and lorc_decode_attn, and copies the result to out_host
+ * [batch, n_q_heads, d_head]; all on `stream`, asynchronously when the host
+ * buffers are pinned.  The caller synchronises the stream before reading
+ * out_host.  The cache stays on the device. */
+int lorc_decode_step_host(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* x_host,
+                          const void* q_host, void* out_host, int n_splits, void* stream);
+
+/* Synchronise `stream`, then read and clear the device status word.  Returns
+ * LORC_OK or the first error a kernel recorded since the last call. */
+int lorc_sync_status(lorc_ctx* ctx, void* stream);
+
+/* Text of the last error reported on this context (never NULL). */
+const char* lorc_last_error(const lorc_ctx* ctx);
+
+/* Which kernel family the last lorc_decode_attn / lorc_append call on this
+ * context used: 0 = none yet, 1 = plain fp32 CUDA-core kernels, 2 = tensor-core
+ * (tcgen05) kernels.  For tests and benchmarks. */
+int lorc_last_path(const lorc_ctx* ctx);
+
+/* Number of kernel launches the library has enqueued on this context so far. */
+int64_t lorc_launch_count(const lorc_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LORC_H_ */
