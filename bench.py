@@ -1,0 +1,409 @@
+#!/usr/bin/env python
+"""Benchmark of the latent-KV decode path (lorc_append + lorc_decode_attn per layer).
+
+A "step" is one decode step of the whole layer stack: for every layer, append
+the new token's latents for every sequence, then run decode attention over the
+latent cache.  Prints ONE JSON line (rank 0).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+With N > 1 (under torchrun) every rank runs its own replica of the workload on
+its own GPU (the path shards by sequence, without any exchange); the value is the
+number of tokens all ranks decoded divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "LoRC decode-attn tokens/s (latent KV, 8B shape); % of HBM/TC roofline"
+UNIT = "tokens/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="cfg2_8b_progressive")
+    ap.add_argument("--layers", type=int, default=0, help="debug: use only the first LAYERS layers")
+    ap.add_argument("--debug-fp32", action="store_true", help="time the plain fp32 kernels")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            f = [x.strip() for x in r.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx = float(f[1])
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        sm.sort()
+        med = sm[len(sm) // 2] if sm else None
+        return {"sm_mhz": med, "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------ workload set-up
+def algorithmic_counts(shape, ranks, batch, n_ctx):
+    """Per decode step over all layers: tensor-eligible FLOPs and latent+factor bytes of
+    lorc_decode_attn with every sequence holding n_ctx tokens."""
+    n, Hq, dh = shape.n, shape.n_q_heads, shape.d_head
+    flops = 0.0
+    byts = 0.0
+    for r in ranks:
+        per_tok = 2.0 * r * n + 2.0 * Hq * dh + 2.0 * Hq * r
+        flops += batch * n_ctx * per_tok + batch * 2.0 * Hq * r * dh
+        byts += batch * n_ctx * 2.0 * (r + r) + 2.0 * (r + r) * n + 4.0 * batch * Hq * dh
+    return flops, byts
+
+
+class Workload:
+    """Factors, prefilled latent caches and per-step inputs of one configuration on one GPU."""
+
+    def __init__(self, L, shape, n_layers, total_steps, device, flags):
+        import torch
+        from paper_2410_03111_b200 import host
+        from workloads import device as wdev
+        self.L, self.shape, self.torch = L, shape, torch
+        self.n_layers = n_layers
+        self.ranks = shape.ranks[:n_layers]
+        b, N = shape.batch, shape.context
+        self.batch = b
+        self.n_max = ((N + total_steps + 127) // 128) * 128
+        self.ctx = L.lorc_create(n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.d_head,
+                                 shape.rope_theta, max_pos=self.n_max, flags=flags)
+        self.caches, self.keep = [], []
+        self.seq_lens = torch.zeros(b, dtype=torch.int32, device=device)
+        chunk = 512
+        for l in range(n_layers):
+            r = self.ranks[l]
+            Uk, sk, Vk = wdev.weight_generators(shape.d_model, shape.n, shape.sigma_p, l, "k", device)
+            Uv, sv, Vv = wdev.weight_generators(shape.d_model, shape.n, shape.sigma_p, l, "v", device)
+            Ak, Bk = host.factors_from_svd(Uk, sk, Vk, r)
+            Av, Bv = host.factors_from_svd(Uv, sv, Vv, r)
+            L.lorc_load_factors(self.ctx, l, L.LORC_MODE_LATENT, r, r, Ak, Bk, Av, Bv)
+            k = torch.zeros(b, self.n_max, r, dtype=torch.bfloat16, device=device)
+            v = torch.zeros(b, self.n_max, r, dtype=torch.bfloat16, device=device)
+            self.keep.append((k, v))
+            self.caches.append(L.make_cache(k, v, self.seq_lens, b, self.n_max, seq_stride=self.n_max))
+            del Uk, Vk, Uv, Vv, Ak, Bk, Av, Bv
+        # prefill through the library's own cache write, in chunks
+        done = 0
+        while done < N:
+            T = min(chunk, N - done)
+            self.seq_lens.fill_(done + T)
+            for l in range(n_layers):
+                x = wdev.hidden_states((b, T, shape.d_model), l, done // chunk, device)
+                L.lorc_append(self.ctx, l, self.caches[l], x, T=T)
+            done += T
+        torch.cuda.synchronize()
+        rc = L.lorc_sync_status(self.ctx)
+        if rc:
+            raise RuntimeError(f"prefill failed: {L.lorc_last_error(self.ctx)}")
+        # per-step inputs: a fresh token and a fresh query per layer and step
+        self.x = [wdev.hidden_states((total_steps, b, shape.d_model), l, 10 ** 6, device) for l in range(n_layers)]
+        self.q = [wdev.queries((total_steps, b, shape.n_q_heads, shape.d_head), l, 0, device, 8.0)
+                  for l in range(n_layers)]
+        self.out = torch.zeros(n_layers, b, shape.n_q_heads, shape.d_head, dtype=torch.bfloat16, device=device)
+        ws_bytes = L.lorc_workspace_bytes(self.ctx, b, self.n_max)
+        self.ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=device)
+        L.lorc_set_workspace(self.ctx, self.ws)
+        self.step_index = 0
+
+    def step(self, attn_events=None):
+        """One decode step on the device: all layers, inputs already in HBM."""
+        L, i = self.L, self.step_index
+        self.seq_lens += 1
+        for l in range(self.n_layers):
+            L.lorc_append(self.ctx, l, self.caches[l], self.x[l][i], T=1)
+            if attn_events is not None:
+                e0 = self.torch.cuda.Event(enable_timing=True)
+                e1 = self.torch.cuda.Event(enable_timing=True)
+                e0.record()
+            L.lorc_decode_attn(self.ctx, l, self.caches[l], self.q[l][i], self.out[l])
+            if attn_events is not None:
+                e1.record()
+                attn_events.append((l, e0, e1))
+        self.step_index += 1
+
+    def step_host(self, xh, qh, oh):
+        """One decode step through the host-buffer entry point (H2D and D2H inside)."""
+        L = self.L
+        self.seq_lens += 1
+        for l in range(self.n_layers):
+            L.lorc_decode_step_host(self.ctx, l, self.caches[l], xh[l], qh[l], oh[l])
+        self.torch.cuda.current_stream().synchronize()
+        self.step_index += 1
+
+
+# ------------------------------------------------------------------- CPU baseline
+def oracle_sample(shape, n_layers, budget_s=15.0, layers=None, n_ctx=None):
+    """Time the fp64 oracle on a bounded sample of the workload: whole (layer, sequence)
+    units (one new token appended, then decode attention over the full context).
+    Returns (seconds per unit-rank, description, threads used, units timed)."""
+    import numpy as np
+    from oracle import lorc_oracle as O
+    from workloads import synth
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    N = n_ctx or shape.context
+    if layers is None:
+        layers = sorted(set([0, n_layers // 2, n_layers - 1]))
+    rng = np.random.default_rng(7)
+    t_total, r_total, units = 0.0, 0, 0
+    used = []
+    t_start = time.time()
+    seq = 0
+    while time.time() - t_start < budget_s:
+        for l in layers:
+            r = shape.ranks[l]
+            # synthetic factors and latents with the workload's shapes (values do not affect the timing)
+            Ak = synth.to_bf16_exact(rng.standard_normal((shape.d_model, r)) / 64).astype(np.float64)
+            Av = synth.to_bf16_exact(rng.standard_normal((shape.d_model, r)) / 64).astype(np.float64)
+            Bk = synth.to_bf16_exact(rng.standard_normal((r, shape.n)) / 32).astype(np.float64)
+            Bv = synth.to_bf16_exact(rng.standard_normal((r, shape.n)) / 32).astype(np.float64)
+            ck = synth.to_bf16_exact(rng.standard_normal((N + 1, r))).astype(np.float64)
+            cv = synth.to_bf16_exact(rng.standard_normal((N + 1, r))).astype(np.float64)
+            x = synth.hidden_states(1, shape.d_model, l, 5 + seq).astype(np.float64)
+            q = synth.queries(1, shape.n_q_heads, shape.d_head, l, seq, 8.0)[0].astype(np.float64)
+            t0 = time.perf_counter()
+            ck[N] = O.append_latent_bf16(x, Ak)[0]
+            cv[N] = O.append_latent_bf16(x, Av)[0]
+            O.decode_attn_latent(ck, cv, Bk, Bv, q, shape.n_kv_heads, shape.rope_theta)
+            t_total += time.perf_counter() - t0
+            r_total += r
+            units += 1
+            used.append(l)
+            if time.time() - t_start > budget_s:
+                break
+        seq += 1
+    layers = sorted(set(used))
+    desc = (f"{units} (layer, sequence) units of {shape.name} ({t_total:.1f} s of oracle time): layers {layers}, "
+            f"context {N}+1, append of 1 token + decode attention; scaled to the step by rank "
+            f"(time per unit proportional to r_l) and by the batch")
+    return t_total / r_total, desc, threads, units
+
+
+def run_reference(args, shape, n_layers):
+    """The oracle as the reference arm: each step times a bounded sample and scales it."""
+    vals = []
+    per_rank, desc, threads = None, "", 1
+    for i in range(args.warmup + args.steps):
+        per_rank, desc, threads, units = oracle_sample(shape, n_layers, budget_s=6.0,
+                                                       layers=[0, n_layers - 1] if n_layers > 1 else [0])
+        step_s = per_rank * sum(shape.ranks[:n_layers]) * shape.batch
+        if i >= args.warmup:
+            vals.append(step_s)
+    step_s = sum(vals) / len(vals)
+    value = shape.batch / step_s
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": shape.name, "layers": n_layers, "batch": shape.batch, "context": shape.context},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- main
+def main():
+    args = parse_args()
+    from workloads import synth
+    shape = synth.CONFIGS[args.config]
+    n_layers = args.layers if args.layers > 0 else shape.n_layers
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args, shape, n_layers)
+        return 0
+
+    import torch
+    import paper_2410_03111_b200 as pkg
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    pkg._build.build()
+    L = pkg.load()
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    peaks = load_peaks()
+    flags = L.LORC_FLAG_DEBUG_FP32 if args.debug_fp32 else 0
+    e2e_steps = 0 if args.no_e2e else max(2, min(args.steps, 8))
+    total_steps = args.warmup + args.steps + e2e_steps + 2
+    wl = Workload(L, shape, n_layers, total_steps, device, flags)
+    b = shape.batch
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        wl.step()
+    barrier()
+    launches0 = L.lorc_launch_count(wl.ctx)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    attn_events = []
+    n_ctx_start = shape.context + args.warmup
+    ev0.record()
+    for _ in range(args.steps):
+        wl.step(attn_events)
+    ev1.record()
+    barrier()
+    clocks = sampler.stop()
+    launches = L.lorc_launch_count(wl.ctx) - launches0
+    path = L.lorc_last_path(wl.ctx)
+    rc = L.lorc_sync_status(wl.ctx)
+    if rc:
+        raise RuntimeError(f"device status {rc}: {L.lorc_last_error(wl.ctx)}")
+    ms = ev0.elapsed_time(ev1)
+    attn_ms = sum(e0.elapsed_time(e1) for _, e0, e1 in attn_events)
+
+    # end-to-end: host buffers in, host buffers out, every step
+    e2e = None
+    if e2e_steps:
+        xh = [torch.empty(b, shape.d_model, dtype=torch.bfloat16).pin_memory() for _ in range(n_layers)]
+        qh = [torch.empty(b, shape.n_q_heads, shape.d_head, dtype=torch.bfloat16).pin_memory() for _ in range(n_layers)]
+        oh = [torch.empty(b, shape.n_q_heads, shape.d_head, dtype=torch.bfloat16).pin_memory() for _ in range(n_layers)]
+        for l in range(n_layers):
+            xh[l].copy_(wl.x[l][0])
+            qh[l].copy_(wl.q[l][0])
+        wl.step_host(xh, qh, oh)            # warm
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            wl.step_host(xh, qh, oh)
+        torch.cuda.synchronize()
+        e2e_s = time.perf_counter() - t0
+        h2d = n_layers * (xh[0].numel() + qh[0].numel()) * 2
+        d2h = n_layers * oh[0].numel() * 2
+        e2e = (e2e_s, h2d, d2h)
+
+    # max over ranks
+    t = torch.tensor([ms, attn_ms, e2e[0] if e2e else 0.0], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms, attn_ms, e2e_s = (float(v) for v in t.tolist())
+
+    if rank == 0:
+        tokens = b * args.steps * world
+        value = tokens / (ms * 1e-3)
+        n_ctx_mid = n_ctx_start + (args.steps + 1) / 2.0
+        flops, byts = algorithmic_counts(shape, wl.ranks, b, n_ctx_mid)
+        attn_ms_step = attn_ms / args.steps
+        t_tc = flops / (peaks["bf16_tflops_sustained"] * 1e12)
+        t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
+        achieved = flops / (attn_ms_step * 1e-3) / 1e12
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": shape.name, "layers": n_layers, "batch": b, "context": shape.context,
+                       "ranks_mean": sum(wl.ranks) / len(wl.ranks), "l2": "inputs larger than L2 (latent cache %.1f GB)" %
+                       (sum(2 * 2 * r for r in wl.ranks) * b * n_ctx_mid / 1e9),
+                       "kernel_path": {1: "plain fp32 CUDA-core", 2: "tcgen05"}.get(path, str(path)),
+                       "replicas": world},
+            "decode_attn": {"ms_per_step": attn_ms_step, "tokens_per_s": b * world / (attn_ms_step * 1e-3),
+                            "roofline_ms": max(t_tc, t_hbm) * 1e3, "frac_of_roofline": max(t_tc, t_hbm) * 1e3 / attn_ms_step,
+                            "hbm_gbs": byts / (attn_ms_step * 1e-3) / 1e9},
+            "roofline": {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"],
+                         "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"],
+                         "traffic": None, "peak_source": peaks["source"] + " (sustained bf16)",
+                         "kernel": "lorc_decode_attn launch train (reconstruction + attention + combine)",
+                         "flops_per_step": flops, "bytes_per_step": byts},
+            "clocks": clocks, "gpu_launches": launches,
+        }
+        if e2e:
+            line["e2e"] = {"value": b * e2e_steps * world / e2e_s, "unit": UNIT, "h2d_bytes_per_step": e2e[1],
+                           "d2h_bytes_per_step": e2e[2], "steps": e2e_steps}
+        if not args.no_cpu_baseline and world >= 1:
+            per_rank, desc, threads, units = oracle_sample(shape, n_layers)
+            step_s = per_rank * sum(wl.ranks) * b
+            line["cpu_baseline"] = {"value": b / step_s, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                    "sample": desc}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
