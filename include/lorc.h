@@ -164,6 +164,31 @@ int lorc_append(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* x
 int lorc_decode_attn(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* q, void* out,
                      int n_splits, void* stream);
 
+/* Decode attention without any caller-provided or freshly allocated scratch.
+ * (The paper has no counterpart to this call; it exists for deployment reasons.)
+ * Meant for hosts that cannot allocate device memory when they call in: a server
+ * that gave the whole GPU to its own memory pool at start-up, or a plug-in that
+ * receives tensors but no allocator.  Same arguments, meaning and result as
+ * lorc_decode_attn, computed by the plain CUDA-core kernels, but the per-split
+ * partial results live in a fixed array of LORC_STATIC_SCRATCH_BYTES inside the
+ * library (each GPU that loads the library holds that much until the process
+ * ends).  The call performs no cudaMalloc/cudaFree and ignores the workspace.
+ *   - Limit: batch * n_q_heads * n_splits * (2 + w) * 4 bytes must fit, w = r_v
+ *     of the layer (d_head for FULL layers).  The split count is lowered
+ *     automatically to fit; if one split still does not fit the call returns
+ *     LORC_ERR_WORKSPACE and runs nothing.
+ *   - The first call on each device looks up the array's device address
+ *     (a short host-side set-up step); make that first call outside any stream
+ *     capture.  The context's device must be current.
+ *   - All calls, on every context and stream, share the one array per GPU.  It
+ *     keeps whatever the previous call left; this call overwrites every slot it
+ *     later reads, so no clearing is needed.  Two calls whose kernels may overlap
+ *     on the GPU (different streams without ordering) race on the array: order
+ *     them. */
+#define LORC_STATIC_SCRATCH_BYTES (8u << 20)
+int lorc_decode_attn_static(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* q, void* out,
+                            int n_splits, void* stream);
+
 /* One decode step of one layer from HOST buffers: copies x_host [batch, D] and
  * q_host [batch, n_q_heads, d_head] to staging at the end of the workspace, runs
  * lorc_append (T = 1) and lorc_decode_attn, and copies the result to out_host

@@ -27,6 +27,7 @@ LORC_MODE_FULL = 1
 LORC_ROPE_HALF_SPLIT = 0
 LORC_ROPE_INTERLEAVED = 1
 LORC_FLAG_DEBUG_FP32 = 1
+LORC_STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class lorc_model_desc(C.Structure):
@@ -63,6 +64,7 @@ def _signatures():
         "lorc_set_workspace": ([vp, vp, C.c_size_t], i32),
         "lorc_append": ([vp, i32, cp, vp, i32, vp], i32),
         "lorc_decode_attn": ([vp, i32, cp, vp, vp, i32, vp], i32),
+        "lorc_decode_attn_static": ([vp, i32, cp, vp, vp, i32, vp], i32),
         "lorc_decode_step_host": ([vp, i32, cp, vp, vp, vp, i32, vp], i32),
         "lorc_sync_status": ([vp, vp], i32),
         "lorc_last_error": ([vp], C.c_char_p),
@@ -161,6 +163,12 @@ def lorc_append(ctx, layer, cache, x, T=1, stream=None):
 def lorc_decode_attn(ctx, layer, cache, q, out, n_splits=0, stream=None):
     _check(ctx, _lib.lorc_decode_attn(ctx, layer, C.byref(cache), _ptr(q), _ptr(out), n_splits,
                                        _stream(stream)))
+
+
+def lorc_decode_attn_static(ctx, layer, cache, q, out, n_splits=0, stream=None):
+    """lorc_decode_attn for callers that cannot allocate: scratch is a fixed array in the library."""
+    _check(ctx, _lib.lorc_decode_attn_static(ctx, layer, C.byref(cache), _ptr(q), _ptr(out), n_splits,
+                                              _stream(stream)))
 
 
 def lorc_decode_step_host(ctx, layer, cache, x_host, q_host, out_host, n_splits=0, stream=None):
