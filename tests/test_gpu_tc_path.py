@@ -1,0 +1,161 @@
+"""GPU parity of the tensor-core (tcgen05) decode path against the fp64 oracle, through the C ABI.
+
+Shapes here have the 8B head geometry (32 query heads, 8 KV heads of 128) so that the library picks
+its tensor-core kernels; each test asserts that it did.  Tolerance: max relative L2 error per
+(sequence, head) row <= 1e-2 (bf16 operands, fp32 accumulation).
+"""
+import numpy as np
+import pytest
+
+from oracle import lorc_oracle as O
+from workloads import synth
+
+import helpers as H
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-2
+GEOM = dict(D=1024, H_q=32, H_kv=8, d_h=128)
+_PROBS = {}
+
+
+def _prob(r_k, r_v, layer=20, theta=500000.0):
+    key = (r_k, r_v, layer, theta)
+    if key not in _PROBS:
+        _PROBS[key] = H.Problem(GEOM["D"], GEOM["H_q"], GEOM["H_kv"], GEOM["d_h"], r_k, r_v, theta=theta,
+                                layer=layer)
+    return _PROBS[key]
+
+
+def _latents(prob, lens, layer):
+    xs = [synth.hidden_states(int(L), prob.D, layer, chunk=200 + s).astype(np.float64) for s, L in enumerate(lens)]
+    return H.oracle_latents(prob, xs)
+
+
+def _run(sess, cache, q, n_splits=0):
+    import torch
+    b = q.shape[0]
+    out = torch.zeros(b, GEOM["H_q"], GEOM["d_h"], dtype=torch.bfloat16, device="cuda")
+    sess.L.lorc_decode_attn(sess.ctx, 0, cache, H.dev_bf16(q), out, n_splits=n_splits)
+    assert sess.L.lorc_sync_status(sess.ctx) == 0, sess.L.lorc_last_error(sess.ctx)
+    assert sess.L.lorc_last_path(sess.ctx) == 2, "the tensor-core path was not taken"
+    return out
+
+
+@pytest.mark.parametrize("r_k,r_v,lens", [
+    (96, 72, [1, 37, 300, 700]),          # rank tails below one 64-wide slice / one 128-row block
+    (256, 256, [129, 128, 1000]),
+    (928, 928, [513, 77]),                # largest rank of the 8B schedule: 14.5 slices, 7.25 blocks
+    (1024, 1024, [260]),                  # full rank in latent form
+])
+def test_tc_decode_contiguous(r_k, r_v, lens):
+    prob = _prob(r_k, r_v)
+    b, n_max = len(lens), max(lens) + 3
+    sess = H.Session(prob, max_pos=n_max, batch=b)
+    ck, cv = _latents(prob, lens, 20)
+    cache, k, v, sl = H.contiguous_cache(sess, b, n_max, lens, ck, cv)
+    for q_scale in (1.0, 64.0):
+        q = synth.queries(b, GEOM["H_q"], GEOM["d_h"], 20, int(q_scale), q_scale).astype(np.float64)
+        got = H.host_f64(_run(sess, cache, q))
+        want = H.oracle_decode(prob, ck, cv, q)
+        assert O.rel_l2_rows(got, want) <= TOL
+    sess.close()
+
+
+def test_tc_decode_matches_plain_kernels_and_split_counts():
+    import torch
+    prob = _prob(160, 224, layer=21)
+    lens = [1500, 70, 640]
+    b = len(lens)
+    ck, cv = _latents(prob, lens, 21)
+    q = synth.queries(b, GEOM["H_q"], GEOM["d_h"], 21, 0, 16.0).astype(np.float64)
+    want = H.oracle_decode(prob, ck, cv, q)
+    sess = H.Session(prob, max_pos=1536, batch=b)
+    cache, k, v, sl = H.contiguous_cache(sess, b, 1536, lens, ck, cv)
+    res = []
+    for S in (0, 1, 2, 5, 12):
+        res.append(H.host_f64(_run(sess, cache, q, n_splits=S)))
+        assert O.rel_l2_rows(res[-1], want) <= TOL
+    for r_ in res[1:]:
+        assert O.rel_l2_rows(r_, res[0]) <= TOL        # same scores; p rounded against another max, output rounded to bf16
+    sess.close()
+    # the plain fp32 kernels agree with the tensor-core kernels within the bf16 tolerance
+    dbg = H.Session(prob, max_pos=1536, batch=b, flags=1)
+    cache, k, v, sl = H.contiguous_cache(dbg, b, 1536, lens, ck, cv)
+    out = torch.zeros(b, GEOM["H_q"], GEOM["d_h"], dtype=torch.bfloat16, device="cuda")
+    dbg.L.lorc_decode_attn(dbg.ctx, 0, cache, H.dev_bf16(q), out)
+    assert dbg.L.lorc_last_path(dbg.ctx) == 1
+    assert O.rel_l2_rows(res[0], H.host_f64(out)) <= TOL
+    dbg.close()
+
+
+@pytest.mark.parametrize("page_size", [64, 16, 128])
+def test_tc_decode_paged_and_page_permutation(page_size):
+    import torch
+    prob = _prob(96, 72, layer=22)
+    lens = [200, 65, 64, 449]
+    b = len(lens)
+    sess = H.Session(prob, max_pos=512, batch=b)
+    ck, cv = _latents(prob, lens, 22)
+    q = synth.queries(b, GEOM["H_q"], GEOM["d_h"], 22, 0, 8.0).astype(np.float64)
+    want = H.oracle_decode(prob, ck, cv, q)
+    outs = []
+    for order_seed in (11, 12):
+        cache, k, v, sl, ptd, pt = H.paged_cache(sess, b, lens, page_size, order_seed, ck, cv)
+        out = _run(sess, cache, q)
+        assert O.rel_l2_rows(H.host_f64(out), want) <= TOL
+        outs.append(out.clone())
+    assert torch.equal(outs[0], outs[1])                # physical page order changes nothing
+    cache, k, v, sl = H.contiguous_cache(sess, b, 512, lens, ck, cv)
+    assert torch.equal(_run(sess, cache, q), outs[0])   # paged == contiguous, bit for bit
+    sess.close()
+
+
+def test_tc_ragged_batch_equals_each_sequence_alone_and_empty_sequence():
+    import torch
+    prob = _prob(96, 72, layer=23)
+    lens = [17, 390, 128]
+    sess = H.Session(prob, max_pos=512, batch=3)
+    ck, cv = _latents(prob, lens, 23)
+    q = synth.queries(3, GEOM["H_q"], GEOM["d_h"], 23, 0, 4.0)
+    cache, k, v, sl = H.contiguous_cache(sess, 3, 512, lens, ck, cv)
+    out = _run(sess, cache, q)
+    for s in range(3):
+        c1, k1, v1, sl1 = H.contiguous_cache(sess, 1, 512, [lens[s]], [ck[s]], [cv[s]])
+        c1.max_seq_len = max(lens)
+        o1 = _run(sess, c1, q[s:s + 1])
+        assert torch.equal(o1[0], out[s])
+    # an empty sequence gives zeros and status EMPTY; the others are unaffected
+    sl[0] = 0
+    o2 = torch.ones(3, GEOM["H_q"], GEOM["d_h"], dtype=torch.bfloat16, device="cuda")
+    sess.L.lorc_decode_attn(sess.ctx, 0, cache, H.dev_bf16(q), o2)
+    assert sess.L.lorc_sync_status(sess.ctx) == sess.L.LORC_ERR_EMPTY
+    assert float(o2[0].abs().max()) == 0.0 and torch.equal(o2[1:], out[1:])
+    # a page index outside the pool is reported, not dereferenced
+    cache, k, v, sl, ptd, pt = H.paged_cache(sess, 3, lens, 64, 31, ck, cv)
+    ptd[1, 2] = 10 ** 6
+    sess.L.lorc_decode_attn(sess.ctx, 0, cache, H.dev_bf16(q), o2)
+    assert sess.L.lorc_sync_status(sess.ctx) == sess.L.LORC_ERR_CAPACITY
+    sess.close()
+
+
+def test_tc_append_then_decode_chain_and_host_entry():
+    import torch
+    prob = _prob(96, 72, layer=24)
+    b, N = 2, 300
+    sess = H.Session(prob, max_pos=384, batch=b)
+    xs = [synth.hidden_states(N + 1, prob.D, 24, chunk=300 + s).astype(np.float64) for s in range(b)]
+    cache, k, v, sl = H.contiguous_cache(sess, b, 384, [N] * b)
+    cache.max_seq_len = 384
+    sess.L.lorc_append(sess.ctx, 0, cache, H.dev_bf16(np.stack([x[:N] for x in xs])), T=N)
+    sl += 1
+    q = synth.queries(b, GEOM["H_q"], GEOM["d_h"], 24, 0, 8.0)
+    xh = torch.from_numpy(np.stack([x[N] for x in xs]).astype(np.float32)).to(torch.bfloat16).pin_memory()
+    qh = torch.from_numpy(q).to(torch.bfloat16).pin_memory()
+    oh = torch.zeros(b, GEOM["H_q"], GEOM["d_h"], dtype=torch.bfloat16).pin_memory()
+    sess.L.lorc_decode_step_host(sess.ctx, 0, cache, xh, qh, oh)
+    assert sess.L.lorc_sync_status(sess.ctx) == 0
+    assert sess.L.lorc_last_path(sess.ctx) == 2
+    ck, cv = H.oracle_latents(prob, xs)
+    want = H.oracle_decode(prob, ck, cv, q.astype(np.float64))
+    assert O.rel_l2_rows(H.host_f64(oh), want) <= TOL
+    sess.close()
