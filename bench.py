@@ -40,6 +40,9 @@ def parse_args():
     ap.add_argument("--debug-fp32", action="store_true", help="time the plain fp32 kernels")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch call by call instead of replaying a CUDA graph")
+    ap.add_argument("--stages", action="store_true",
+                    help="call-by-call launches with per-kernel CUDA events; adds a 'stages' object (ms per step)")
     return ap.parse_args()
 
 
@@ -172,20 +175,50 @@ class Workload:
         L.lorc_set_workspace(self.ctx, self.ws)
         self.step_index = 0
 
-    def step(self, attn_events=None):
-        """One decode step on the device: all layers, inputs already in HBM."""
-        L, i = self.L, self.step_index
-        self.seq_lens += 1
+    def _layers(self, xs, qs, append=True, attn=True):
+        L = self.L
         for l in range(self.n_layers):
-            L.lorc_append(self.ctx, l, self.caches[l], self.x[l][i], T=1)
-            if attn_events is not None:
-                e0 = self.torch.cuda.Event(enable_timing=True)
-                e1 = self.torch.cuda.Event(enable_timing=True)
-                e0.record()
-            L.lorc_decode_attn(self.ctx, l, self.caches[l], self.q[l][i], self.out[l])
-            if attn_events is not None:
-                e1.record()
-                attn_events.append((l, e0, e1))
+            if append:
+                L.lorc_append(self.ctx, l, self.caches[l], xs[l], T=1)
+            if attn:
+                L.lorc_decode_attn(self.ctx, l, self.caches[l], qs[l], self.out[l])
+
+    def step(self):
+        """One decode step on the device, launched call by call: all layers, inputs already in HBM."""
+        i = self.step_index
+        self.seq_lens += 1
+        self._layers([x[i] for x in self.x], [q[i] for q in self.q])
+        self.step_index += 1
+
+    def capture(self):
+        """Capture one decode step (and, separately, the attention calls alone) into CUDA graphs.
+        The step's inputs are read from fixed buffers that step_graph() refills before each replay."""
+        torch = self.torch
+        self.x_cur = torch.stack([x[0] for x in self.x]).contiguous()
+        self.q_cur = torch.stack([q[0] for q in self.q]).contiguous()
+        self.x_all = torch.stack(self.x).transpose(0, 1).contiguous()      # [steps, L, b, D]
+        self.q_all = torch.stack(self.q).transpose(0, 1).contiguous()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            self.g_attn = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(self.g_attn, stream=side):
+                self._layers(self.x_cur, self.q_cur, append=False)
+            # (work issued during capture is recorded, not executed: the cache does not advance here)
+            self.g_step = torch.cuda.CUDAGraph()
+            n0 = self.L.lorc_launch_count(self.ctx)
+            with torch.cuda.graph(self.g_step, stream=side):
+                self.seq_lens += 1
+                self._layers(self.x_cur, self.q_cur)
+            self.launches_per_step = self.L.lorc_launch_count(self.ctx) - n0
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+
+    def step_graph(self):
+        i = self.step_index
+        self.x_cur.copy_(self.x_all[i])
+        self.q_cur.copy_(self.q_all[i])
+        self.g_step.replay()
         self.step_index += 1
 
     def step_host(self, xh, qh, oh):
@@ -303,8 +336,11 @@ def main():
 
     peaks = load_peaks()
     flags = L.LORC_FLAG_DEBUG_FP32 if args.debug_fp32 else 0
+    if args.stages:
+        flags |= L.LORC_FLAG_PROFILE
+        args.no_graph = True
     e2e_steps = 0 if args.no_e2e else max(2, min(args.steps, 8))
-    total_steps = args.warmup + args.steps + e2e_steps + 2
+    total_steps = args.warmup + args.steps + e2e_steps + 4
     wl = Workload(L, shape, n_layers, total_steps, device, flags)
     b = shape.batch
 
@@ -313,28 +349,59 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    use_graph = not args.no_graph
+    wl.step()                      # first call of every kernel outside any capture
+    torch.cuda.synchronize()
+    if use_graph:
+        try:
+            wl.capture()
+        except Exception as exc:   # keep the benchmark alive on the call-by-call path
+            sys.stderr.write(f"graph capture failed ({exc}); timing call-by-call launches\n")
+            use_graph = False
+    do_step = wl.step_graph if use_graph else wl.step
     for _ in range(args.warmup):
-        wl.step()
+        do_step()
     barrier()
     launches0 = L.lorc_launch_count(wl.ctx)
+    if args.stages:
+        L.lorc_profile_read(wl.ctx)          # drop what set-up and warm-up recorded
     sampler = ClockSampler(local_rank)
     sampler.start()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    attn_events = []
-    n_ctx_start = shape.context + args.warmup
+    n_ctx_start = shape.context + 1 + args.warmup
     ev0.record()
     for _ in range(args.steps):
-        wl.step(attn_events)
+        do_step()
     ev1.record()
     barrier()
+    ms = ev0.elapsed_time(ev1)
+    stages = None
+    if args.stages:
+        stages = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps}
+                  for k, v in L.lorc_profile_read(wl.ctx).items()}
+    launches_per_step = wl.launches_per_step if use_graph else (L.lorc_launch_count(wl.ctx) - launches0) / args.steps
+    # the attention calls alone (all layers), on the cache as it stands after the timed steps
+    ea0, ea1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    attn_reps = max(3, min(args.steps, 16))
+    def attn_only():
+        if use_graph:
+            wl.g_attn.replay()
+        else:
+            wl._layers(None, [q[0] for q in wl.q], append=False)
+    attn_only()
+    torch.cuda.synchronize()
+    ea0.record()
+    for _ in range(attn_reps):
+        attn_only()
+    ea1.record()
+    barrier()
     clocks = sampler.stop()
-    launches = L.lorc_launch_count(wl.ctx) - launches0
+    attn_ms = ea0.elapsed_time(ea1) / attn_reps * args.steps
     path = L.lorc_last_path(wl.ctx)
     rc = L.lorc_sync_status(wl.ctx)
     if rc:
         raise RuntimeError(f"device status {rc}: {L.lorc_last_error(wl.ctx)}")
-    ms = ev0.elapsed_time(ev1)
-    attn_ms = sum(e0.elapsed_time(e1) for _, e0, e1 in attn_events)
+    launches = int(round(launches_per_step * args.steps))
 
     # end-to-end: host buffers in, host buffers out, every step
     e2e = None
@@ -365,7 +432,7 @@ def main():
     if rank == 0:
         tokens = b * args.steps * world
         value = tokens / (ms * 1e-3)
-        n_ctx_mid = n_ctx_start + (args.steps + 1) / 2.0
+        n_ctx_mid = n_ctx_start + args.steps      # context the attention-only pass sees
         flops, byts = algorithmic_counts(shape, wl.ranks, b, n_ctx_mid)
         attn_ms_step = attn_ms / args.steps
         t_tc = flops / (peaks["bf16_tflops_sustained"] * 1e12)
@@ -379,7 +446,7 @@ def main():
                        "ranks_mean": sum(wl.ranks) / len(wl.ranks), "l2": "inputs larger than L2 (latent cache %.1f GB)" %
                        (sum(2 * 2 * r for r in wl.ranks) * b * n_ctx_mid / 1e9),
                        "kernel_path": {1: "plain fp32 CUDA-core", 2: "tcgen05"}.get(path, str(path)),
-                       "replicas": world},
+                       "replicas": world, "launch": "cuda graph per step" if use_graph else "call by call"},
             "decode_attn": {"ms_per_step": attn_ms_step, "tokens_per_s": b * world / (attn_ms_step * 1e-3),
                             "roofline_ms": max(t_tc, t_hbm) * 1e3, "frac_of_roofline": max(t_tc, t_hbm) * 1e3 / attn_ms_step,
                             "hbm_gbs": byts / (attn_ms_step * 1e-3) / 1e9},
@@ -390,6 +457,8 @@ def main():
                          "flops_per_step": flops, "bytes_per_step": byts},
             "clocks": clocks, "gpu_launches": launches,
         }
+        if stages:
+            line["stages"] = stages
         if e2e:
             line["e2e"] = {"value": b * e2e_steps * world / e2e_s, "unit": UNIT, "h2d_bytes_per_step": e2e[1],
                            "d2h_bytes_per_step": e2e[2], "steps": e2e_steps}

@@ -56,6 +56,14 @@ extern "C" {
 
 /* context flags */
 #define LORC_FLAG_DEBUG_FP32 1  /* run the plain fp32 CUDA-core kernels everywhere (debug path) */
+#define LORC_FLAG_PROFILE 2     /* bracket every kernel with CUDA events (see lorc_profile_read) */
+
+/* stages reported by lorc_profile_read */
+#define LORC_STAGE_APPEND 0     /* cache write */
+#define LORC_STAGE_SCORE 1      /* key reconstruction + RoPE + scores (tensor-core path) or the whole plain kernel */
+#define LORC_STAGE_PV 2         /* softmax + P.C_V */
+#define LORC_STAGE_COMBINE 3    /* split merge + value up-projection */
+#define LORC_N_STAGES 4
 
 typedef struct lorc_ctx lorc_ctx;
 
@@ -209,6 +217,13 @@ const char* lorc_last_error(const lorc_ctx* ctx);
  * context used: 0 = none yet, 1 = plain fp32 CUDA-core kernels, 2 = tensor-core
  * (tcgen05) kernels.  For tests and benchmarks. */
 int lorc_last_path(const lorc_ctx* ctx);
+
+/* Contexts created with LORC_FLAG_PROFILE record a CUDA event before and after every
+ * kernel they launch (do not use together with stream capture).  This call waits for the
+ * recorded events, adds up the device time per stage since the previous call and writes
+ * ms[LORC_N_STAGES] (milliseconds) and launches[LORC_N_STAGES]; either may be NULL.
+ * Without the flag it returns zeros. */
+int lorc_profile_read(lorc_ctx* ctx, float* ms, int64_t* launches);
 
 /* Number of kernel launches the library has enqueued on this context so far. */
 int64_t lorc_launch_count(const lorc_ctx* ctx);

@@ -27,6 +27,9 @@ LORC_MODE_FULL = 1
 LORC_ROPE_HALF_SPLIT = 0
 LORC_ROPE_INTERLEAVED = 1
 LORC_FLAG_DEBUG_FP32 = 1
+LORC_FLAG_PROFILE = 2
+LORC_N_STAGES = 4
+LORC_STAGE_NAMES = ("append", "score", "pv", "combine")
 LORC_STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -69,6 +72,7 @@ def _signatures():
         "lorc_sync_status": ([vp, vp], i32),
         "lorc_last_error": ([vp], C.c_char_p),
         "lorc_last_path": ([vp], i32),
+        "lorc_profile_read": ([vp, C.POINTER(C.c_float), C.POINTER(i64)], i32),
         "lorc_launch_count": ([vp], i64),
     }
 
@@ -186,6 +190,14 @@ def lorc_last_error(ctx):
 
 def lorc_last_path(ctx):
     return int(_lib.lorc_last_path(ctx))
+
+
+def lorc_profile_read(ctx):
+    """Device milliseconds and launch counts per stage since the last call (LORC_FLAG_PROFILE contexts)."""
+    ms = (C.c_float * LORC_N_STAGES)()
+    cnt = (C.c_int64 * LORC_N_STAGES)()
+    _check(ctx, _lib.lorc_profile_read(ctx, ms, cnt))
+    return {name: (float(ms[i]), int(cnt[i])) for i, name in enumerate(LORC_STAGE_NAMES)}
 
 
 def lorc_launch_count(ctx):

@@ -31,6 +31,19 @@ struct LorcLayer {
 
 struct LorcTcState;            // tensor-core path's private per-context state
 
+// Event pairs recorded around kernels when LORC_FLAG_PROFILE is set.
+struct LorcProfile {
+    struct Rec { int stage; cudaEvent_t e0, e1; };
+    std::vector<Rec> pending;
+    std::vector<cudaEvent_t> pool;
+    cudaEvent_t get() {
+        if (!pool.empty()) { cudaEvent_t e = pool.back(); pool.pop_back(); return e; }
+        cudaEvent_t e = nullptr;
+        cudaEventCreate(&e);
+        return e;
+    }
+};
+
 struct lorc_ctx {
     lorc_model_desc desc;
     int device = 0;
@@ -46,6 +59,26 @@ struct lorc_ctx {
     int last_path = 0;
     int64_t launches = 0;
     LorcTcState* tc = nullptr;
+    LorcProfile* prof = nullptr;   // non-null iff LORC_FLAG_PROFILE
+};
+
+// RAII bracket: records an event pair around the launches issued in its scope (no-op unless profiling).
+struct LorcStageTimer {
+    LorcProfile* p;
+    LorcProfile::Rec rec;
+    cudaStream_t st;
+    LorcStageTimer(const lorc_ctx* ctx, int stage, cudaStream_t stream) : p(ctx->prof), st(stream) {
+        if (!p) return;
+        rec.stage = stage;
+        rec.e0 = p->get();
+        rec.e1 = p->get();
+        cudaEventRecord(rec.e0, st);
+    }
+    ~LorcStageTimer() {
+        if (!p) return;
+        cudaEventRecord(rec.e1, st);
+        p->pending.push_back(rec);
+    }
 };
 
 // Where rows of a cache live: contiguous or paged (mirrors lorc_cache, device-usable).

@@ -429,6 +429,7 @@ cudaError_t lorc_generic_combine(const lorc_ctx* ctx, const LorcLayer& L, int ba
     const int W = latent ? L.r_v : d.d_head;
     dim3 cgrid(d.n_q_heads, batch);
     size_t smem = (size_t)W * sizeof(float);
+    LorcStageTimer timer(ctx, LORC_STAGE_COMBINE, st);
     if (latent)
         combine_generic_kernel<true><<<cgrid, 128, smem, st>>>(part_ml, part_o, L.B_v, out, W, ctx->n,
                                                               d.d_head, ctx->group, n_splits,
@@ -448,6 +449,8 @@ cudaError_t lorc_generic_decode(const lorc_ctx* ctx, const LorcLayer& L, const C
     const int G = ctx->group;
     const bool latent = (L.mode == LORC_MODE_LATENT);
     dim3 grid(n_splits, d.n_kv_heads, cv.batch);
+    {
+    LorcStageTimer timer(ctx, LORC_STAGE_SCORE, st);
 #define LAUNCH_DEC(DHV, LAT)                                                                      \
     decode_generic_kernel<DHV, LAT><<<grid, 128, 0, st>>>(                                        \
         q, cv, L.B_k, L.r_k, L.r_v, ctx->n, G, n_splits, d.rope_style, ctx->rope_table, d.max_pos, \
@@ -458,6 +461,7 @@ cudaError_t lorc_generic_decode(const lorc_ctx* ctx, const LorcLayer& L, const C
         if (latent) LAUNCH_DEC(64, true); else LAUNCH_DEC(64, false);
     }
 #undef LAUNCH_DEC
+    }
     *launches += 1;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;

@@ -129,6 +129,7 @@ int lorc_create(const lorc_model_desc* desc, lorc_ctx** out) {
     ctx->n = desc->n_kv_heads * desc->d_head;
     ctx->group = desc->n_q_heads / desc->n_kv_heads;
     ctx->layers.resize(desc->n_layers);
+    if (desc->flags & LORC_FLAG_PROFILE) ctx->prof = new (std::nothrow) LorcProfile();
     cudaError_t e = cudaGetDevice(&ctx->device);
     if (e == cudaSuccess)
         e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device);
@@ -142,6 +143,7 @@ int lorc_create(const lorc_model_desc* desc, lorc_ctx** out) {
     if (e != cudaSuccess) {
         cudaFree(ctx->status_dev);
         cudaFree(ctx->rope_table);
+        delete ctx->prof;
         delete ctx;
         return LORC_ERR_CUDA;
     }
@@ -153,6 +155,14 @@ int lorc_destroy(lorc_ctx* ctx) {
     if (!ctx) return LORC_ERR_ARG;
     for (auto& L : ctx->layers) free_layer(L);
     lorc_tc_release(ctx);
+    if (ctx->prof) {
+        for (auto& r : ctx->prof->pending) {
+            cudaEventDestroy(r.e0);
+            cudaEventDestroy(r.e1);
+        }
+        for (auto e : ctx->prof->pool) cudaEventDestroy(e);
+        delete ctx->prof;
+    }
     cudaFree(ctx->status_dev);
     cudaFree(ctx->rope_table);
     delete ctx;
@@ -242,6 +252,7 @@ int lorc_append(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* x
     int launches = 0;
     cudaError_t e;
     int path = 1;
+    LorcStageTimer timer(ctx, LORC_STAGE_APPEND, st);
     if (!(ctx->desc.flags & LORC_FLAG_DEBUG_FP32) && lorc_tc_append_supported(ctx, *L, cv, T)) {
         e = lorc_tc_append(ctx, layer, *L, cv, (const bf16*)x, T, st, &launches);
         path = 2;
@@ -361,6 +372,32 @@ int lorc_sync_status(lorc_ctx* ctx, void* stream) {
 const char* lorc_last_error(const lorc_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
 
 int lorc_last_path(const lorc_ctx* ctx) { return ctx ? ctx->last_path : 0; }
+
+int lorc_profile_read(lorc_ctx* ctx, float* ms, int64_t* launches) {
+    if (!ctx) return LORC_ERR_ARG;
+    float acc[LORC_N_STAGES] = {0.f, 0.f, 0.f, 0.f};
+    int64_t cnt[LORC_N_STAGES] = {0, 0, 0, 0};
+    if (ctx->prof) {
+        for (auto& r : ctx->prof->pending) {
+            float t = 0.f;
+            cudaError_t e = cudaEventSynchronize(r.e1);
+            if (e == cudaSuccess) e = cudaEventElapsedTime(&t, r.e0, r.e1);
+            if (e != cudaSuccess) return fail_cuda(ctx, e, "lorc_profile_read");
+            if (r.stage >= 0 && r.stage < LORC_N_STAGES) {
+                acc[r.stage] += t;
+                cnt[r.stage] += 1;
+            }
+            ctx->prof->pool.push_back(r.e0);
+            ctx->prof->pool.push_back(r.e1);
+        }
+        ctx->prof->pending.clear();
+    }
+    for (int i = 0; i < LORC_N_STAGES; ++i) {
+        if (ms) ms[i] = acc[i];
+        if (launches) launches[i] = cnt[i];
+    }
+    return LORC_OK;
+}
 
 int64_t lorc_launch_count(const lorc_ctx* ctx) { return ctx ? ctx->launches : 0; }
 

@@ -14,7 +14,7 @@
 //                 bf16 into shared memory, and O_lat^T[r_V, H_q] += C_V^T . P^T on the tensor cores with
 //                 C_V consumed straight from its row-major TMA tiles (MN-major operand).
 //                 Partials (m, l, O_lat) go to scratch.
-//  combine        merges the splits and applies B_V (generic_kernels.cu).
+//  combine        merges the splits and applies B_V (fast_aux.cu).
 //
 // Keys and values never exist in memory; only the 4*H_q bytes of scores per token are written.
 #include <math.h>
@@ -589,12 +589,6 @@ bool lorc_tc_decode_supported(const lorc_ctx* ctx, const LorcLayer& L, const Cac
     return lorc_get_tmap_encode() != nullptr;
 }
 
-bool lorc_tc_append_supported(const lorc_ctx*, const LorcLayer&, const CacheView&, int) { return false; }
-
-cudaError_t lorc_tc_append(lorc_ctx*, int, const LorcLayer&, const CacheView&, const bf16*, int, cudaStream_t, int*) {
-    return cudaErrorNotSupported;
-}
-
 static int tc_tiles_per_split(int max_seq_len, int n_splits_hint) {
     int tiles = (max_seq_len + TILE - 1) / TILE;
     if (n_splits_hint > 0) {
@@ -703,10 +697,13 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
     const int total_units = cv.batch * tiles * sp.n_hp;
     int grid1 = total_units < ctx->sm_count ? total_units : ctx->sm_count;
     const size_t smem1 = sizeof(ScoreSmem) + 1024;
-    if (ctx->group == 4)
-        lorc_score_kernel<4><<<grid1, S_THREADS, smem1, st>>>(TL.mapCK, TL.mapBKT, sp);
-    else
-        lorc_score_kernel<8><<<grid1, S_THREADS, smem1, st>>>(TL.mapCK, TL.mapBKT, sp);
+    {
+        LorcStageTimer timer(ctx, LORC_STAGE_SCORE, st);
+        if (ctx->group == 4)
+            lorc_score_kernel<4><<<grid1, S_THREADS, smem1, st>>>(TL.mapCK, TL.mapBKT, sp);
+        else
+            lorc_score_kernel<8><<<grid1, S_THREADS, smem1, st>>>(TL.mapCK, TL.mapBKT, sp);
+    }
     *launches += 1;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -718,12 +715,15 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
     pp.tiles_per_split = tps; pp.max_pos = d.max_pos;
     pp.page_size = cv.page_size; pp.max_pages_per_seq = cv.max_pages_per_seq; pp.n_pages = cv.n_pages;
     dim3 grid2(S, cv.batch);
-    if (d.n_q_heads == 32)
-        lorc_pv_kernel<32><<<grid2, V_THREADS, sizeof(PvSmem<32>) + 1024, st>>>(TL.mapCV, pp);
-    else
-        lorc_pv_kernel<64><<<grid2, V_THREADS, sizeof(PvSmem<64>) + 1024, st>>>(TL.mapCV, pp);
+    {
+        LorcStageTimer timer(ctx, LORC_STAGE_PV, st);
+        if (d.n_q_heads == 32)
+            lorc_pv_kernel<32><<<grid2, V_THREADS, sizeof(PvSmem<32>) + 1024, st>>>(TL.mapCV, pp);
+        else
+            lorc_pv_kernel<64><<<grid2, V_THREADS, sizeof(PvSmem<64>) + 1024, st>>>(TL.mapCV, pp);
+    }
     *launches += 1;
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    return lorc_generic_combine(ctx, L, cv.batch, S, part_ml, part_o, out, st, launches);
+    return lorc_fast_combine(ctx, L, cv.batch, S, part_ml, part_o, out, st, launches);
 }

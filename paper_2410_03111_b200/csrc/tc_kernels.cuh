@@ -16,6 +16,12 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
 cudaError_t lorc_tc_append(lorc_ctx* ctx, int layer, const LorcLayer& L, const CacheView& cv,
                            const bf16* x, int T, cudaStream_t st, int* launches);
 
+// Merge of split partials + value up-projection for LATENT layers with d_head = 128
+// (same inputs and result as lorc_generic_combine).
+cudaError_t lorc_fast_combine(const lorc_ctx* ctx, const LorcLayer& L, int batch, int n_splits,
+                              const float* part_ml, const float* part_o, bf16* out, cudaStream_t st,
+                              int* launches);
+
 // Drop cached per-layer state (tensor maps) when factors are reloaded / the context dies.
 void lorc_tc_invalidate_layer(lorc_ctx* ctx, int layer);
 void lorc_tc_release(lorc_ctx* ctx);
