@@ -42,7 +42,7 @@ struct ScoreSmem {
     bf16 A[S_STAGES][TILE * KC];          // latent slice  [128 tokens][64]       16 KiB
     bf16 B[S_STAGES][256 * KC];           // B_K^T slice   [256 features][64]     32 KiB
     float2 trigT[64][TILE];               // (cos, sin)(t * theta_j), [j][t]      64 KiB
-    float qrot[2][2][8][128];             // [buffer][head of pair][g][dim]       16 KiB
+    float qrot[2][2][64][16];             // [buffer][head of pair][pair j][qa_0..qa_G-1, qb_0..qb_G-1]  16 KiB
     uint64_t full[S_STAGES], empty[S_STAGES], acc_full[2], acc_empty[2];
     uint32_t tmem_base;
     int abort_flag;
@@ -209,8 +209,8 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
                 const float2 cs = p.rope_table[(long long)delta * 64 + j];
                 const bf16* qp = p.q + ((long long)un.s * p.H_q + h) * 128;
                 const float a = __bfloat162float(qp[j]), b = __bfloat162float(qp[j + 64]);
-                sm.qrot[qb][hip][g][j] = (a * cs.x - b * cs.y) * scale;
-                sm.qrot[qb][hip][g][j + 64] = (a * cs.y + b * cs.x) * scale;
+                sm.qrot[qb][hip][j][g] = (a * cs.x - b * cs.y) * scale;
+                sm.qrot[qb][hip][j][G + g] = (a * cs.y + b * cs.x) * scale;
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");
             if (!mbar_wait(&sm.acc_full[buf], (uc >> 1) & 1)) { ok = false; break; }
@@ -232,9 +232,16 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
                     const float a = __uint_as_float(ra[i]), b = __uint_as_float(rb[i]);
                     const float ka = a * cs.x - b * cs.y;
                     const float kb = a * cs.y + b * cs.x;
+                    const float4* qv = reinterpret_cast<const float4*>(sm.qrot[qb][grp][j]);
+                    float qa[G], qbv[G];
 #pragma unroll
-                    for (int g = 0; g < G; ++g)
-                        acc[g] = fmaf(sm.qrot[qb][grp][g][j + 64], kb, fmaf(sm.qrot[qb][grp][g][j], ka, acc[g]));
+                    for (int g4 = 0; g4 < G / 4; ++g4) {
+                        const float4 x = qv[g4], y = qv[G / 4 + g4];
+                        qa[g4 * 4 + 0] = x.x; qa[g4 * 4 + 1] = x.y; qa[g4 * 4 + 2] = x.z; qa[g4 * 4 + 3] = x.w;
+                        qbv[g4 * 4 + 0] = y.x; qbv[g4 * 4 + 1] = y.y; qbv[g4 * 4 + 2] = y.z; qbv[g4 * 4 + 3] = y.w;
+                    }
+#pragma unroll
+                    for (int g = 0; g < G; ++g) acc[g] = fmaf(qbv[g], kb, fmaf(qa[g], ka, acc[g]));
                 }
             }
             tc_fence_before_sync();
