@@ -23,7 +23,7 @@ struct LorcLayer {
     int mode = LORC_MODE_LATENT;
     int r_k = 0, r_v = 0;      // FULL mode: both equal n
     bf16* A_cat = nullptr;     // [D, r_k + r_v]   columns of A_K then A_V (FULL: W_k then W_v)
-    bf16* A_catT = nullptr;    // [r_k + r_v, D]   transposed copy (K-major operand of the tensor-core append)
+    bf16* A_tiled = nullptr;   // [(r_k+r_v)/8][D/32][32 lanes][8]: A_cat in mma fragment order (fast append), D % 32 == 0
     bf16* B_k = nullptr;       // [r_k, n]   (LATENT)
     bf16* B_v = nullptr;       // [r_v, n]   (LATENT)
     bf16* B_kT = nullptr;      // [n, r_k]   transposed copy (K-major operand of the key reconstruction)

@@ -21,7 +21,7 @@ int fail_cuda(lorc_ctx* ctx, cudaError_t e, const char* where) {
 
 void free_layer(LorcLayer& L) {
     cudaFree(L.A_cat);
-    cudaFree(L.A_catT);
+    cudaFree(L.A_tiled);
     cudaFree(L.B_k);
     cudaFree(L.B_v);
     cudaFree(L.B_kT);
@@ -190,7 +190,7 @@ int lorc_load_factors(lorc_ctx* ctx, int layer, int mode, int r_k, int r_v, cons
     lorc_tc_invalidate_layer(ctx, layer);
     const int R = r_k + r_v;
     cudaError_t e = cudaMalloc(&L.A_cat, (size_t)D * R * sizeof(bf16));
-    if (e == cudaSuccess) e = cudaMalloc(&L.A_catT, (size_t)D * R * sizeof(bf16));
+    if (e == cudaSuccess && D % 32 == 0) e = cudaMalloc(&L.A_tiled, (size_t)D * R * sizeof(bf16));
     if (e == cudaSuccess && mode == LORC_MODE_LATENT) {
         e = cudaMalloc(&L.B_k, (size_t)r_k * n * sizeof(bf16));
         if (e == cudaSuccess) e = cudaMalloc(&L.B_v, (size_t)r_v * n * sizeof(bf16));
@@ -202,7 +202,7 @@ int lorc_load_factors(lorc_ctx* ctx, int layer, int mode, int r_k, int r_v, cons
     if (e == cudaSuccess)
         e = cudaMemcpy2DAsync(L.A_cat + r_k, (size_t)R * sizeof(bf16), A_v, (size_t)r_v * sizeof(bf16),
                               (size_t)r_v * sizeof(bf16), D, cudaMemcpyDeviceToDevice, st);
-    if (e == cudaSuccess) e = lorc_generic_transpose(L.A_cat, L.A_catT, D, R, st);
+    if (e == cudaSuccess && L.A_tiled) e = lorc_fast_retile_factor(L.A_cat, L.A_tiled, D, R, st);
     if (e == cudaSuccess && mode == LORC_MODE_LATENT) {
         e = cudaMemcpyAsync(L.B_k, B_k, (size_t)r_k * n * sizeof(bf16), cudaMemcpyDeviceToDevice, st);
         if (e == cudaSuccess)

@@ -223,9 +223,10 @@ static inline lorc_tmap_encode_fn lorc_get_tmap_encode() {
 }
 
 // bf16 tensor of `rank` dims (dims[0] innermost, strides in bytes for dims 1..rank-1), box of box[] elements,
-// 128-byte swizzle (box[0] must be 64 elements), out-of-bounds elements read as zero.
+// 128-byte swizzle (box[0] must be 64 elements) unless swizzle128 is false (plain rows, box[0] <= 256 elements);
+// out-of-bounds elements read as zero.
 static inline bool lorc_make_tmap_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
-                                       const uint64_t* strides_bytes, const uint32_t* box) {
+                                       const uint64_t* strides_bytes, const uint32_t* box, bool swizzle128 = true) {
     lorc_tmap_encode_fn enc = lorc_get_tmap_encode();
     if (!enc) return false;
     cuuint64_t gd[5];
@@ -238,7 +239,7 @@ static inline bool lorc_make_tmap_bf16(CUtensorMap* map, const void* base, int r
     }
     for (int i = 0; i + 1 < rank; ++i) gs[i] = strides_bytes[i];
     CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gd, gs, bx,
-                     es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     es, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }

@@ -438,7 +438,15 @@ lorc_pv_kernel(const __grid_constant__ CUtensorMap mapCV, const PvParams p) {
                 float mx[HQ];
 #pragma unroll
                 for (int h = 0; h < HQ; ++h) mx[h] = -INFINITY;
-                for (int n = t_begin + t; n < t_end; n += TILE) {
+                // (two tiles per iteration: twice as many independent loads in flight)
+                int n = t_begin + t;
+                for (; n + TILE < t_end; n += 2 * TILE) {
+                    const float* sp = p.scores + (long long)s * p.H_q * p.n_pad + n;
+#pragma unroll
+                    for (int h = 0; h < HQ; ++h)
+                        mx[h] = fmaxf(mx[h], fmaxf(sp[(long long)h * p.n_pad], sp[(long long)h * p.n_pad + TILE]));
+                }
+                if (n < t_end) {
                     const float* sp = p.scores + (long long)s * p.H_q * p.n_pad + n;
 #pragma unroll
                     for (int h = 0; h < HQ; ++h) mx[h] = fmaxf(mx[h], sp[(long long)h * p.n_pad]);
@@ -546,7 +554,7 @@ __global__ void rope_tile_kernel(float2* out, double theta) {
 // ------------------------------------------------------------------------------------------------
 struct LorcTcLayer {
     bool has_bkt = false;
-    CUtensorMap mapBKT;
+    CUtensorMap mapBKT, mapBV;          // B_K^T in 64 x 256 swizzled boxes; B_V in plain 64-row x 128-column boxes
     // cache maps are rebuilt only when the cache geometry or pointers change
     const void* k_ptr = nullptr;
     const void* v_ptr = nullptr;
@@ -672,6 +680,9 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
         uint64_t dims[2] = {(uint64_t)L.r_k, (uint64_t)ctx->n}, str[1] = {(uint64_t)L.r_k * 2};
         uint32_t box[2] = {KC, 256};
         if (!lorc_make_tmap_bf16(&TL.mapBKT, L.B_kT, 2, dims, str, box)) return cudaErrorInvalidValue;
+        uint64_t d2[2] = {(uint64_t)ctx->n, (uint64_t)L.r_v}, s2[1] = {(uint64_t)ctx->n * 2};
+        uint32_t b2[2] = {128, 64};
+        if (!lorc_make_tmap_bf16(&TL.mapBV, L.B_v, 2, d2, s2, b2, false)) return cudaErrorInvalidValue;
         TL.has_bkt = true;
     }
     if (!build_cache_maps(TL, L, cv)) return cudaErrorInvalidValue;
@@ -732,5 +743,5 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
     *launches += 1;
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    return lorc_fast_combine(ctx, L, cv.batch, S, part_ml, part_o, out, st, launches);
+    return lorc_fast_combine(ctx, L, &TL.mapBV, cv.batch, S, part_ml, part_o, out, st, launches);
 }

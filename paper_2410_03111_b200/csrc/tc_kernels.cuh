@@ -1,6 +1,8 @@
 // Tensor-core (tcgen05 / TMA) kernels of the library: interface used by the C ABI.
 #pragma once
 
+#include <cuda.h>
+
 #include "common.cuh"
 
 // Whether the tensor-core kernels cover this layer / cache combination.
@@ -18,9 +20,13 @@ cudaError_t lorc_tc_append(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
 
 // Merge of split partials + value up-projection for LATENT layers with d_head = 128
 // (same inputs and result as lorc_generic_combine).
-cudaError_t lorc_fast_combine(const lorc_ctx* ctx, const LorcLayer& L, int batch, int n_splits,
-                              const float* part_ml, const float* part_o, bf16* out, cudaStream_t st,
+// mapBV: B_V [r_v, n] as a 2-D tensor map with plain (unswizzled) boxes of 64 rows x 128 columns.
+cudaError_t lorc_fast_combine(const lorc_ctx* ctx, const LorcLayer& L, const CUtensorMap* mapBV, int batch,
+                              int n_splits, const float* part_ml, const float* part_o, bf16* out, cudaStream_t st,
                               int* launches);
+
+// A_cat [D, R] (row-major) -> fragment order [R/8][D/32][32 lanes][8] used by the fast append kernel.
+cudaError_t lorc_fast_retile_factor(const bf16* A_cat, bf16* A_tiled, int D, int R, cudaStream_t st);
 
 // Drop cached per-layer state (tensor maps) when factors are reloaded / the context dies.
 void lorc_tc_invalidate_layer(lorc_ctx* ctx, int layer);
