@@ -25,6 +25,16 @@ cudaError_t lorc_fast_combine(const lorc_ctx* ctx, const LorcLayer& L, const CUt
                               int n_splits, const float* part_ml, const float* part_o, bf16* out, cudaStream_t st,
                               int* launches);
 
+// Softmax + P.C_V + value up-projection (tc_pv.cu).  scores [b, H_q, n_pad] (log2 units) and
+// tmax [b, H_q, tiles, 4] (maxima of each 32-token quarter tile) come from the score kernel.
+// mapCV: C_V cache in 64-column x 128-row (or page-sized) swizzled boxes; mapBV: B_V [r_v, n] in plain
+// 128 x 128 boxes.  Launches the PV kernel and the kernel that adds its pieces into `out`.
+size_t lorc_tc_pv_scratch_bytes(const lorc_ctx* ctx, int batch, int max_seq_len);
+cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, const CUtensorMap& mapCV,
+                              const CUtensorMap& mapBV, const float* scores, const float* tmax, int n_pad, int tiles,
+                              int n_splits_hint, void* scratch, size_t scratch_bytes, bf16* out, cudaStream_t st,
+                              int* launches);
+
 // A_cat [D, R] (row-major) -> fragment order [R/8][D/32][32 lanes][8] used by the fast append kernel.
 cudaError_t lorc_fast_retile_factor(const bf16* A_cat, bf16* A_tiled, int D, int R, cudaStream_t st);
 
