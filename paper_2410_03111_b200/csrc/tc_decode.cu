@@ -1,6 +1,6 @@
 // Tensor-core decode attention over the latent cache (sm_100a: TMA + tcgen05 + TMEM).
 //
-// Two kernels per layer, followed by the merge / value-up-projection kernel:
+// Two kernels per layer, followed by a small kernel that adds up the output pieces:
 //
 //  score kernel   persistent CTAs walk (sequence, 128-token tile, KV-head pair) units.  Per unit the
 //                 key tile of two KV heads is reconstructed on the tensor cores,
@@ -10,11 +10,9 @@
 //                 with the G rotated queries of its KV head; the scores (log2 units) go to scratch.
 //                 RoPE is split as R(n0 + t) = R(n0) R(t): R(t), t < 128, is a constant table in shared
 //                 memory and R(n0) is folded into the query once per unit (q' = R(m - n0) q).
-//  PV kernel      one CTA per (sequence, context split): exact row max of the split, p = 2^(s - m) as
-//                 bf16 into shared memory, and O_lat^T[r_V, H_q] += C_V^T . P^T on the tensor cores with
-//                 C_V consumed straight from its row-major TMA tiles (MN-major operand).
-//                 Partials (m, l, O_lat) go to scratch.
-//  combine        merges the splits and applies B_V (fast_aux.cu).
+//                 It also leaves the maximum of every 32-token quarter tile, so that the next kernel knows
+//                 the exact row maximum of the softmax without a pass over the scores.
+//  PV kernel      softmax + P.C_V + value up-projection, split by latent columns (tc_pv.cu).
 //
 // Keys and values never exist in memory; only the 4*H_q bytes of scores per token are written.
 #include <math.h>
@@ -51,6 +49,7 @@ struct ScoreSmem {
 struct ScoreParams {
     const bf16* q;                 // [b, H_q, 128]
     float* scores;                 // [b, H_q, n_pad]
+    float* tmax;                   // [b, H_q, tiles_per_seq, 4]  maxima per 32-token quarter tile
     const int32_t* seq_lens;
     const int32_t* page_table;     // NULL: contiguous
     const float2* rope_table;      // [max_pos][64]
@@ -247,12 +246,16 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
             tc_fence_before_sync();
             mbar_arrive(&sm.acc_empty[buf]);
             const int n = n0 + t;
-            if (n < p.n_pad) {
 #pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    const int h = (un.hp * 2 + grp) * G + g;
-                    p.scores[((long long)un.s * p.H_q + h) * p.n_pad + n] = acc[g];
-                }
+            for (int g = 0; g < G; ++g) {
+                const int h = (un.hp * 2 + grp) * G + g;
+                if (n < p.n_pad) p.scores[((long long)un.s * p.H_q + h) * p.n_pad + n] = acc[g];
+                // maximum over the 32 tokens of this warp (tokens past the end of the sequence do not count)
+                float mxv = (n < un.len) ? acc[g] : -INFINITY;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) mxv = fmaxf(mxv, __shfl_xor_sync(0xffffffffu, mxv, o));
+                if (lane == 0)
+                    p.tmax[(((long long)un.s * p.H_q + h) * p.tiles_per_seq + un.tile) * 4 + quarter] = mxv;
             }
             ++uc;
         }
@@ -264,276 +267,6 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, 512);
-}
-
-// ------------------------------------------------------------------------------------------------
-// PV kernel
-// ------------------------------------------------------------------------------------------------
-constexpr int V_STAGES = 4;
-constexpr int V_THREADS = 192;       // warp 0 TMA, warp 1 MMA, warps 2..5 softmax
-constexpr int V_SOFT = 128;
-
-template <int HQ>
-struct PvSmem {
-    bf16 V[V_STAGES][2][TILE * KC];       // C_V slice: two 64-column blocks of [128 tokens][64]   32 KiB/stage
-    bf16 P[2][2][HQ * KC];                // probabilities [HQ heads][128 tokens] as two 64-token chunks
-    float red[4][HQ];
-    float m_s[HQ];
-    uint64_t full[V_STAGES], empty[V_STAGES], p_full[2], p_empty[2], o_full;
-    uint32_t tmem_base;
-    int abort_flag;
-};
-
-struct PvParams {
-    const float* scores;           // [b, H_q, n_pad]  (log2 units)
-    float* part_ml;                // [b, H_q, S, 2]   (max in natural-log units, sum)
-    float* part_o;                 // [b, H_q, S, r_v]
-    const int32_t* seq_lens;
-    const int32_t* page_table;
-    int* status;
-    int batch, H_q, r_v, n_pad, n_splits, tiles_per_split, max_pos;
-    int page_size, max_pages_per_seq, n_pages;
-};
-
-template <int HQ>
-__global__ void __launch_bounds__(V_THREADS, 1)
-lorc_pv_kernel(const __grid_constant__ CUtensorMap mapCV, const PvParams p) {
-    extern __shared__ uint8_t raw[];
-    typedef PvSmem<HQ> S;
-    S& sm = *reinterpret_cast<S*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
-    const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
-    const int split = blockIdx.x, s = blockIdx.y;
-    const int nblk = (p.r_v + 127) / 128;
-    constexpr uint32_t TM_COLS = (HQ * 8 <= 256) ? 256 : 512;
-
-    int len = p.seq_lens[s];
-    if (len > p.max_pos) {
-        if (tid == 0) lorc_set_status(p.status, LORC_ERR_CAPACITY);
-        len = 0;
-    }
-    if (len < 0) len = 0;
-    const int t_begin = min(len, split * p.tiles_per_split * TILE);
-    const int t_end = min(len, (split + 1) * p.tiles_per_split * TILE);
-    const int ntiles = (t_end - t_begin + TILE - 1) / TILE;
-
-    if (tid == 0) {
-        for (int i = 0; i < V_STAGES; ++i) {
-            mbar_init(&sm.full[i], 1);
-            mbar_init(&sm.empty[i], 1);
-        }
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(&sm.p_full[i], V_SOFT);
-            mbar_init(&sm.p_empty[i], 1);
-        }
-        mbar_init(&sm.o_full, 1);
-        sm.abort_flag = 0;
-        fence_barrier_init();
-        prefetch_tensormap(&mapCV);
-    }
-    if (warp == 1) {
-        tmem_alloc(&sm.tmem_base, TM_COLS);
-        tmem_relinquish();
-    }
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    const uint32_t tmem = sm.tmem_base;
-
-    if (warp == 0) {
-        if (lane == 0 && ntiles > 0) {
-            uint32_t it = 0;
-            bool ok = true;
-            for (int i = 0; i < ntiles && ok; ++i) {
-                const int n0 = t_begin + i * TILE;
-                for (int blk = 0; blk < nblk; ++blk, ++it) {
-                    const int st = it % V_STAGES;
-                    if (!mbar_wait(&sm.empty[st], ((it / V_STAGES) & 1) ^ 1)) { ok = false; break; }
-                    if (p.page_table == nullptr) {
-                        mbar_arrive_expect_tx(&sm.full[st], 2 * TILE * KC * 2);
-                        tma_load_3d(sm.V[st][0], &mapCV, &sm.full[st], blk * 128, n0, s);
-                        tma_load_3d(sm.V[st][1], &mapCV, &sm.full[st], blk * 128 + 64, n0, s);
-                    } else {
-                        const int ppt = TILE / p.page_size;
-                        int pages[8];
-                        uint32_t bytes = 0;
-                        for (int pg = 0; pg < ppt; ++pg) {
-                            int lp = n0 / p.page_size + pg;
-                            int page = -1;
-                            if (lp * p.page_size < len && lp < p.max_pages_per_seq) {
-                                page = p.page_table[(long long)s * p.max_pages_per_seq + lp];
-                                if (page < 0 || page >= p.n_pages) {
-                                    lorc_set_status(p.status, LORC_ERR_CAPACITY);
-                                    page = -1;
-                                }
-                            }
-                            pages[pg] = page;
-                            if (page >= 0) bytes += 2 * p.page_size * KC * 2;
-                        }
-                        if (bytes == 0) {
-                            mbar_arrive(&sm.full[st]);
-                        } else {
-                            mbar_arrive_expect_tx(&sm.full[st], bytes);
-                            for (int pg = 0; pg < ppt; ++pg)
-                                if (pages[pg] >= 0) {
-                                    tma_load_3d(sm.V[st][0] + pg * p.page_size * KC, &mapCV, &sm.full[st], blk * 128,
-                                                0, pages[pg]);
-                                    tma_load_3d(sm.V[st][1] + pg * p.page_size * KC, &mapCV, &sm.full[st],
-                                                blk * 128 + 64, 0, pages[pg]);
-                                }
-                        }
-                    }
-                }
-            }
-            if (!ok) {
-                lorc_set_status(p.status, LORC_ERR_TIMEOUT);
-                sm.abort_flag = 1;
-            }
-        }
-    } else if (warp == 1) {
-        if (lane == 0 && ntiles > 0) {
-            const uint32_t idesc = make_idesc_bf16(128, HQ, 1, 0);
-            uint32_t it = 0;
-            bool ok = true;
-            for (int i = 0; i < ntiles && ok; ++i) {
-                const int buf = i & 1;
-                if (!mbar_wait(&sm.p_full[buf], (i >> 1) & 1)) { ok = false; break; }
-                tc_fence_after_sync();
-                const uint32_t p0 = smem_u32(sm.P[buf][0]);
-                for (int blk = 0; blk < nblk; ++blk, ++it) {
-                    const int st = it % V_STAGES;
-                    if (!mbar_wait(&sm.full[st], (it / V_STAGES) & 1)) { ok = false; break; }
-                    tc_fence_after_sync();
-                    const uint32_t v0 = smem_u32(sm.V[st][0]);
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        // A: C_V^T block, MN-major: 16 token rows per step, two 64-column blocks 16 KiB apart
-                        const uint64_t ad = make_smem_desc_sw128(v0 + k * 2048, TILE * KC * 2, 1024);
-                        // B: P [HQ][128 tokens], K-major: 64-token chunks of HQ*128 bytes
-                        const uint64_t bd =
-                            make_smem_desc_sw128(p0 + (k >> 2) * (HQ * KC * 2) + (k & 3) * 32, 0, 1024);
-                        tc_mma_bf16(tmem + blk * HQ, ad, bd, idesc, (i | k) != 0);
-                    }
-                    tc_commit(&sm.empty[st]);
-                }
-                if (!ok) break;
-                tc_commit(&sm.p_empty[buf]);
-            }
-            tc_commit(&sm.o_full);
-            if (!ok) {
-                lorc_set_status(p.status, LORC_ERR_TIMEOUT);
-                sm.abort_flag = 1;
-            }
-        }
-    } else {
-        // ------------------------------------------------------------------ softmax warps
-        const int t = tid - 64;                   // 0..127: token inside the tile, and TMEM lane later
-        const int wq = warp - 2;                  // 0..3 == warp % 4 - 2 .. careful below
-        float l[HQ];
-#pragma unroll
-        for (int h = 0; h < HQ; ++h) l[h] = 0.f;
-        bool ok = true;
-        if (ntiles > 0) {
-            // phase A: exact maximum of every head over this split
-            {
-                float mx[HQ];
-#pragma unroll
-                for (int h = 0; h < HQ; ++h) mx[h] = -INFINITY;
-                // (two tiles per iteration: twice as many independent loads in flight)
-                int n = t_begin + t;
-                for (; n + TILE < t_end; n += 2 * TILE) {
-                    const float* sp = p.scores + (long long)s * p.H_q * p.n_pad + n;
-#pragma unroll
-                    for (int h = 0; h < HQ; ++h)
-                        mx[h] = fmaxf(mx[h], fmaxf(sp[(long long)h * p.n_pad], sp[(long long)h * p.n_pad + TILE]));
-                }
-                if (n < t_end) {
-                    const float* sp = p.scores + (long long)s * p.H_q * p.n_pad + n;
-#pragma unroll
-                    for (int h = 0; h < HQ; ++h) mx[h] = fmaxf(mx[h], sp[(long long)h * p.n_pad]);
-                }
-#pragma unroll
-                for (int h = 0; h < HQ; ++h) {
-                    float v = mx[h];
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-                    if (lane == 0) sm.red[wq][h] = v;
-                }
-                asm volatile("bar.sync 2, 128;" ::: "memory");
-                if (t < HQ) sm.m_s[t] = fmaxf(fmaxf(sm.red[0][t], sm.red[1][t]), fmaxf(sm.red[2][t], sm.red[3][t]));
-                asm volatile("bar.sync 2, 128;" ::: "memory");
-            }
-            // phase B: probabilities of each tile into shared memory (bf16, K-major, 128-byte swizzle)
-            for (int i = 0; i < ntiles; ++i) {
-                const int buf = i & 1;
-                if (!mbar_wait(&sm.p_empty[buf], ((i >> 1) & 1) ^ 1)) { ok = false; break; }
-                const int n = t_begin + i * TILE + t;
-                const bool valid = n < t_end;
-                const float* sp = p.scores + (long long)s * p.H_q * p.n_pad + n;
-                uint8_t* pb = reinterpret_cast<uint8_t*>(sm.P[buf][t >> 6]);
-                const int tc = t & 63;
-#pragma unroll
-                for (int h = 0; h < HQ; ++h) {
-                    float pv = 0.f;
-                    if (valid) pv = exp2f(sp[(long long)h * p.n_pad] - sm.m_s[h]);
-                    const bf16 pr = __float2bfloat16_rn(pv);
-                    l[h] += __bfloat162float(pr);
-                    const int off = h * 128 + ((((tc >> 3) ^ (h & 7)) << 4) | ((tc & 7) << 1));
-                    *reinterpret_cast<bf16*>(pb + off) = pr;
-                }
-                fence_proxy_async_smem();
-                mbar_arrive(&sm.p_full[buf]);
-            }
-        }
-        // sum of probabilities per head over the CTA
-        float lsum = 0.f;
-#pragma unroll
-        for (int h = 0; h < HQ; ++h) {
-            float v = l[h];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-            if (lane == 0) sm.red[wq][h] = v;
-        }
-        asm volatile("bar.sync 2, 128;" ::: "memory");
-        if (t < HQ) {
-            lsum = sm.red[0][t] + sm.red[1][t] + sm.red[2][t] + sm.red[3][t];
-            const long long unit = ((long long)s * p.H_q + t) * p.n_splits + split;
-            p.part_ml[unit * 2 + 0] = (ntiles > 0) ? sm.m_s[t] * LN2 : -INFINITY;
-            p.part_ml[unit * 2 + 1] = (ntiles > 0 && ok) ? lsum : 0.f;
-        }
-        if (ntiles > 0 && ok) {
-            if (mbar_wait(&sm.o_full, 0)) {
-                tc_fence_after_sync();
-                // TMEM lane = latent row inside a 128-row block; this warp may read quarter (warp % 4)
-                const int quarter = warp % 4;
-                const int row = quarter * 32 + lane;
-                for (int blk = 0; blk < nblk; ++blk) {
-                    const int rr = blk * 128 + row;
-#pragma unroll
-                    for (int c0 = 0; c0 < HQ; c0 += 32) {
-                        uint32_t r[32];
-                        tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + blk * HQ + c0, r);
-                        tmem_wait_ld();
-                        if (rr < p.r_v) {
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) {
-                                const long long unit = ((long long)s * p.H_q + c0 + i) * p.n_splits + split;
-                                p.part_o[unit * p.r_v + rr] = __uint_as_float(r[i]);
-                            }
-                        }
-                    }
-                }
-            } else {
-                ok = false;
-            }
-        }
-        if (!ok && lane == 0) {
-            lorc_set_status(p.status, LORC_ERR_TIMEOUT);
-            sm.abort_flag = 1;
-        }
-    }
-    tc_fence_before_sync();
-    __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem, TM_COLS);
 }
 
 // constant table (cos, sin)(t * theta_j) laid out [j][t], t < 128
@@ -554,7 +287,7 @@ __global__ void rope_tile_kernel(float2* out, double theta) {
 // ------------------------------------------------------------------------------------------------
 struct LorcTcLayer {
     bool has_bkt = false;
-    CUtensorMap mapBKT, mapBV;          // B_K^T in 64 x 256 swizzled boxes; B_V in plain 64-row x 128-column boxes
+    CUtensorMap mapBKT, mapBV;          // B_K^T in 64 x 256 swizzled boxes; B_V in plain 128-row x 128-column boxes
     // cache maps are rebuilt only when the cache geometry or pointers change
     const void* k_ptr = nullptr;
     const void* v_ptr = nullptr;
@@ -604,28 +337,20 @@ bool lorc_tc_decode_supported(const lorc_ctx* ctx, const LorcLayer& L, const Cac
     return lorc_get_tmap_encode() != nullptr;
 }
 
-static int tc_tiles_per_split(int max_seq_len, int n_splits_hint) {
-    int tiles = (max_seq_len + TILE - 1) / TILE;
-    if (n_splits_hint > 0) {
-        int S = n_splits_hint < tiles ? n_splits_hint : tiles;
-        return (tiles + S - 1) / S;
-    }
-    return tiles < 4 ? tiles : 4;
-}
-
 static size_t tc_scores_bytes(const lorc_ctx* ctx, int batch, int max_seq_len) {
     size_t n_pad = (size_t)((max_seq_len + TILE - 1) / TILE) * TILE;
     return lorc_align_up((size_t)batch * ctx->desc.n_q_heads * n_pad * sizeof(float), 256);
 }
 
+static size_t tc_tmax_bytes(const lorc_ctx* ctx, int batch, int max_seq_len) {
+    size_t tiles = (size_t)((max_seq_len + TILE - 1) / TILE);
+    return lorc_align_up((size_t)batch * ctx->desc.n_q_heads * tiles * 4 * sizeof(float), 256);
+}
+
 size_t lorc_tc_workspace_bytes(const lorc_ctx* ctx, int batch, int max_seq_len) {
     if (!tc_shape_ok(ctx)) return 0;
-    // worst case over split hints: one tile per split
-    int tiles = (max_seq_len + TILE - 1) / TILE;
-    int S = (tiles + 3) / 4;
-    size_t units = (size_t)batch * ctx->desc.n_q_heads * S;
-    return tc_scores_bytes(ctx, batch, max_seq_len) + lorc_align_up(units * 2 * sizeof(float), 256) +
-           lorc_align_up(units * (size_t)ctx->n * sizeof(float), 256);
+    return tc_scores_bytes(ctx, batch, max_seq_len) + tc_tmax_bytes(ctx, batch, max_seq_len) +
+           lorc_tc_pv_scratch_bytes(ctx, batch, max_seq_len);
 }
 
 static bool build_cache_maps(LorcTcLayer& T, const LorcLayer& L, const CacheView& cv) {
@@ -671,8 +396,6 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
         cudaError_t e;
         e = cudaFuncSetAttribute(lorc_score_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ScoreSmem) + 1024);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(lorc_score_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ScoreSmem) + 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(lorc_pv_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(PvSmem<32>) + 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(lorc_pv_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(PvSmem<64>) + 1024);
         if (e != cudaSuccess) return e;
         T->attrs_set = true;
     }
@@ -681,7 +404,7 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
         uint32_t box[2] = {KC, 256};
         if (!lorc_make_tmap_bf16(&TL.mapBKT, L.B_kT, 2, dims, str, box)) return cudaErrorInvalidValue;
         uint64_t d2[2] = {(uint64_t)ctx->n, (uint64_t)L.r_v}, s2[1] = {(uint64_t)ctx->n * 2};
-        uint32_t b2[2] = {128, 64};
+        uint32_t b2[2] = {128, 128};
         if (!lorc_make_tmap_bf16(&TL.mapBV, L.B_v, 2, d2, s2, b2, false)) return cudaErrorInvalidValue;
         TL.has_bkt = true;
     }
@@ -689,25 +412,16 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
 
     const int tiles = (cv.max_seq_len + TILE - 1) / TILE;
     const int n_pad = tiles * TILE;
-    int tps = tc_tiles_per_split(cv.max_seq_len, n_splits);
     const size_t sc_bytes = tc_scores_bytes(ctx, cv.batch, cv.max_seq_len);
-    int S;
-    size_t units, ml_bytes, o_bytes;
-    // fewer, longer splits until the partial results fit the workspace and the merge kernel's limit
-    for (;; ++tps) {
-        S = (tiles + tps - 1) / tps;
-        units = (size_t)cv.batch * d.n_q_heads * S;
-        ml_bytes = lorc_align_up(units * 2 * sizeof(float), 256);
-        o_bytes = lorc_align_up(units * (size_t)L.r_v * sizeof(float), 256);
-        if (S <= LORC_MAX_SPLITS && sc_bytes + ml_bytes + o_bytes <= ws_bytes) break;
-        if (S == 1) return cudaErrorMemoryAllocation;
-    }
+    const size_t tm_bytes = tc_tmax_bytes(ctx, cv.batch, cv.max_seq_len);
+    if (sc_bytes + tm_bytes >= ws_bytes) return cudaErrorMemoryAllocation;
     float* scores = (float*)ws;
-    float* part_ml = (float*)((char*)ws + sc_bytes);
-    float* part_o = (float*)((char*)ws + sc_bytes + ml_bytes);
+    float* tmax = (float*)((char*)ws + sc_bytes);
+    void* pv_scratch = (char*)ws + sc_bytes + tm_bytes;
+    const size_t pv_bytes = ws_bytes - sc_bytes - tm_bytes;
 
     ScoreParams sp;
-    sp.q = q; sp.scores = scores; sp.seq_lens = cv.seq_lens; sp.page_table = cv.page_table;
+    sp.q = q; sp.scores = scores; sp.tmax = tmax; sp.seq_lens = cv.seq_lens; sp.page_table = cv.page_table;
     sp.rope_table = ctx->rope_table; sp.rope_tile = T->rope_tile; sp.status = ctx->status_dev;
     sp.batch = cv.batch; sp.H_q = d.n_q_heads; sp.n_hp = d.n_kv_heads / 2; sp.r_k = L.r_k; sp.n_pad = n_pad;
     sp.tiles_per_seq = tiles; sp.max_pos = d.max_pos;
@@ -725,23 +439,6 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
     *launches += 1;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-
-    PvParams pp;
-    pp.scores = scores; pp.part_ml = part_ml; pp.part_o = part_o; pp.seq_lens = cv.seq_lens;
-    pp.page_table = cv.page_table; pp.status = ctx->status_dev;
-    pp.batch = cv.batch; pp.H_q = d.n_q_heads; pp.r_v = L.r_v; pp.n_pad = n_pad; pp.n_splits = S;
-    pp.tiles_per_split = tps; pp.max_pos = d.max_pos;
-    pp.page_size = cv.page_size; pp.max_pages_per_seq = cv.max_pages_per_seq; pp.n_pages = cv.n_pages;
-    dim3 grid2(S, cv.batch);
-    {
-        LorcStageTimer timer(ctx, LORC_STAGE_PV, st);
-        if (d.n_q_heads == 32)
-            lorc_pv_kernel<32><<<grid2, V_THREADS, sizeof(PvSmem<32>) + 1024, st>>>(TL.mapCV, pp);
-        else
-            lorc_pv_kernel<64><<<grid2, V_THREADS, sizeof(PvSmem<64>) + 1024, st>>>(TL.mapCV, pp);
-    }
-    *launches += 1;
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    return lorc_fast_combine(ctx, L, &TL.mapBV, cv.batch, S, part_ml, part_o, out, st, launches);
+    return lorc_tc_pv_launch(ctx, L, cv, TL.mapCV, TL.mapBV, scores, tmax, n_pad, tiles, n_splits, pv_scratch, pv_bytes,
+                             out, st, launches);
 }

@@ -18,13 +18,6 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
 cudaError_t lorc_tc_append(lorc_ctx* ctx, int layer, const LorcLayer& L, const CacheView& cv,
                            const bf16* x, int T, cudaStream_t st, int* launches);
 
-// Merge of split partials + value up-projection for LATENT layers with d_head = 128
-// (same inputs and result as lorc_generic_combine).
-// mapBV: B_V [r_v, n] as a 2-D tensor map with plain (unswizzled) boxes of 64 rows x 128 columns.
-cudaError_t lorc_fast_combine(const lorc_ctx* ctx, const LorcLayer& L, const CUtensorMap* mapBV, int batch,
-                              int n_splits, const float* part_ml, const float* part_o, bf16* out, cudaStream_t st,
-                              int* launches);
-
 // Softmax + P.C_V + value up-projection (tc_pv.cu).  scores [b, H_q, n_pad] (log2 units) and
 // tmax [b, H_q, tiles, 4] (maxima of each 32-token quarter tile) come from the score kernel.
 // mapCV: C_V cache in 64-column x 128-row (or page-sized) swizzled boxes; mapBV: B_V [r_v, n] in plain
