@@ -209,16 +209,28 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const __grid_constant
             const int n = t_begin + i * TILE + t;
             const bool valid = n < t_end;
             const float* sp = p.scores + (long long)s * p.H_q * p.n_pad + n;
-            uint8_t* pb = reinterpret_cast<uint8_t*>(sm.P[buf][t >> 6]);
+            const uint32_t pb = smem_u32(sm.P[buf][t >> 6]);
             const int tc = t & 63;
+            // all scores of this token first, so that the loads are in flight together: a load scheduled after
+            // one of the (generic-address) stores below would have to wait for it, one memory latency per head
+            float sv[HQ];
+#pragma unroll
+            for (int h = 0; h < HQ; ++h) sv[h] = valid ? __ldg(sp + (long long)h * p.n_pad) : -INFINITY;
+            {
+                // every loaded value is consumed before the first store is issued; a NaN among the scores means
+                // non-finite numbers in the cache, the factors or the query
+                float ssum = 0.f;
+#pragma unroll
+                for (int h = 0; h < HQ; ++h) ssum += valid ? sv[h] : 0.f;
+                if (ssum != ssum) lorc_set_status(p.status, LORC_ERR_ARG);
+            }
 #pragma unroll
             for (int h = 0; h < HQ; ++h) {
-                float pv = 0.f;
-                if (valid) pv = exp2f(sp[(long long)h * p.n_pad] - sm.m_s[h]);
+                const float pv = valid ? exp2f(sv[h] - sm.m_s[h]) : 0.f;
                 const bf16 pr = __float2bfloat16_rn(pv);
                 l[h] += __bfloat162float(pr);
                 const int off = h * 128 + ((((tc >> 3) ^ (h & 7)) << 4) | ((tc & 7) << 1));
-                *reinterpret_cast<bf16*>(pb + off) = pr;
+                asm volatile("st.shared.b16 [%0], %1;" ::"r"(pb + off), "h"(__bfloat16_as_ushort(pr)) : "memory");
             }
             fence_proxy_async_smem();
             mbar_arrive(&sm.p_full[buf]);
