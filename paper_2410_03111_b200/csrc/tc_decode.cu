@@ -287,7 +287,7 @@ __global__ void rope_tile_kernel(float2* out, double theta) {
 // ------------------------------------------------------------------------------------------------
 struct LorcTcLayer {
     bool has_bkt = false;
-    CUtensorMap mapBKT, mapBV;          // B_K^T in 64 x 256 swizzled boxes; B_V in plain 128-row x 128-column boxes
+    CUtensorMap mapBKT, mapBV;          // B_K^T in 64 x 256 swizzled boxes; B_V in plain 64-row x 128-column boxes
     // cache maps are rebuilt only when the cache geometry or pointers change
     const void* k_ptr = nullptr;
     const void* v_ptr = nullptr;
@@ -404,7 +404,7 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
         uint32_t box[2] = {KC, 256};
         if (!lorc_make_tmap_bf16(&TL.mapBKT, L.B_kT, 2, dims, str, box)) return cudaErrorInvalidValue;
         uint64_t d2[2] = {(uint64_t)ctx->n, (uint64_t)L.r_v}, s2[1] = {(uint64_t)ctx->n * 2};
-        uint32_t b2[2] = {128, 128};
+        uint32_t b2[2] = {128, 64};
         if (!lorc_make_tmap_bf16(&TL.mapBV, L.B_v, 2, d2, s2, b2, false)) return cudaErrorInvalidValue;
         TL.has_bkt = true;
     }

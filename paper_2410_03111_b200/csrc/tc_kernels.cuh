@@ -21,7 +21,7 @@ cudaError_t lorc_tc_append(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
 // Softmax + P.C_V + value up-projection (tc_pv.cu).  scores [b, H_q, n_pad] (log2 units) and
 // tmax [b, H_q, tiles, 4] (maxima of each 32-token quarter tile) come from the score kernel.
 // mapCV: C_V cache in 64-column x 128-row (or page-sized) swizzled boxes; mapBV: B_V [r_v, n] in plain
-// 128 x 128 boxes.  Launches the PV kernel and the kernel that adds its pieces into `out`.
+// boxes of 64 rows x 128 columns.  Launches the PV kernel and the kernel that adds its pieces into `out`.
 size_t lorc_tc_pv_scratch_bytes(const lorc_ctx* ctx, int batch, int max_seq_len);
 cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, const CUtensorMap& mapCV,
                               const CUtensorMap& mapBV, const float* scores, const float* tmax, int n_pad, int tiles,

@@ -26,16 +26,24 @@ constexpr int KC = 64;
 constexpr int P_STAGES = 2;          // 2 x 32 KiB: two CTAs fit on an SM
 constexpr int P_THREADS = 192;       // warp 0 TMA, warp 1 MMA, warps 2..5 softmax / epilogue
 constexpr int P_SOFT = 128;
+constexpr int BV_SLOTS = 5;           // B_V pieces of 64 rows (16 KiB): four in the C_V stages, one in the P buffers
+
+// read-only global load that the compiler keeps in program order with the other volatile asm of this file
+__device__ __forceinline__ float ldg_nc_f32(const float* p) {
+    float v;
+    asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    return v;
+}
 
 template <int HQ>
 struct Pv2Smem {
     bf16 V[P_STAGES][2][TILE * KC];       // C_V block: two 64-column halves of [128 tokens][64]; 32 KiB / stage.
-                                          // After the last MMA: B_V[128 rho of this block][128 columns of one KV head]
+                                          // After the last MMA: ring of B_V pieces [64 rho][128 columns of one KV head]
     bf16 P[2][2][HQ * KC];                // probabilities [HQ][128 tokens] as two 64-token chunks, 128-byte swizzle
     float o_sm[128][HQ];                  // O_lat block [rho][head] after the last MMA
     float m_s[HQ];
     float red[4][HQ];
-    uint64_t full[P_STAGES], empty[P_STAGES], p_full[2], p_empty[2], o_full, bv_full[P_STAGES], bv_empty[P_STAGES];
+    uint64_t full[P_STAGES], empty[P_STAGES], p_full[2], p_empty[2], o_full, bv_full[BV_SLOTS], bv_empty[BV_SLOTS];
     uint32_t tmem_base;
 };
 
@@ -78,12 +86,14 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const __grid_constant
     const int t_begin = tile_lo * TILE, t_end = min(len, tile_hi * TILE);
     const int rho0 = blk * 128;
     const int rows_valid = min(128, p.r_v - rho0);       // latent rows of this block that exist
-    const int n_bv = (ntiles > 0) ? p.n_kv : 0;          // B_V pieces to stream (one per KV head)
+    const int n_bv = (ntiles > 0) ? 2 * p.n_kv : 0;      // B_V pieces to stream: (KV head, half of the block's rows)
 
     if (tid == 0) {
         for (int i = 0; i < P_STAGES; ++i) {
             mbar_init(&sm.full[i], 1);
             mbar_init(&sm.empty[i], 1);
+        }
+        for (int i = 0; i < BV_SLOTS; ++i) {
             mbar_init(&sm.bv_full[i], 1);
             mbar_init(&sm.bv_empty[i], P_SOFT);
         }
@@ -137,14 +147,15 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const __grid_constant
                     }
                 }
             }
-            // the rows of B_V this block multiplies with, one 128-column piece per KV head, into the C_V stages
-            // (free once every MMA has retired)
+            // the rows of B_V this block multiplies with, in pieces of 64 rows x 128 columns (one KV head), through a
+            // ring that reuses the C_V stages and the P buffers (all free once every MMA has retired)
             if (n_bv > 0 && ok && !mbar_wait(&sm.o_full, 0)) ok = false;
             for (int c = 0; c < n_bv && ok; ++c) {
-                const int slot = c % P_STAGES;
-                if (!mbar_wait(&sm.bv_empty[slot], ((c / P_STAGES) & 1) ^ 1)) { ok = false; break; }
-                mbar_arrive_expect_tx(&sm.bv_full[slot], 128 * 128 * 2);
-                tma_load_2d(sm.V[slot][0], &mapBV, &sm.bv_full[slot], c * 128, rho0);
+                const int slot = c % BV_SLOTS;
+                if (!mbar_wait(&sm.bv_empty[slot], ((c / BV_SLOTS) & 1) ^ 1)) { ok = false; break; }
+                bf16* dst = (slot < 4) ? (&sm.V[0][0][0] + slot * 64 * 128) : &sm.P[0][0][0];
+                mbar_arrive_expect_tx(&sm.bv_full[slot], 64 * 128 * 2);
+                tma_load_2d(dst, &mapBV, &sm.bv_full[slot], (c >> 1) * 128, rho0 + (c & 1) * 64);
             }
             if (!ok) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
         }
@@ -203,34 +214,42 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const __grid_constant
         if (t < HQ) sm.m_s[t] = fmaxf(fmaxf(sm.red[0][t], sm.red[1][t]), fmaxf(sm.red[2][t], sm.red[3][t]));
         asm volatile("bar.sync 2, 128;" ::: "memory");
 
+        // Scores of a tile are loaded one tile ahead, all heads at once.  The loads and the shared-memory stores are
+        // volatile asm, which keeps them in program order: loads of tile i + 1, then stores of tile i.
+        float sv[HQ];
+        {
+            const int n = t_begin + t;
+            const float* sp = p.scores + (long long)s * p.H_q * p.n_pad + n;
+#pragma unroll
+            for (int h = 0; h < HQ; ++h) sv[h] = (ntiles > 0 && n < t_end) ? ldg_nc_f32(sp + (long long)h * p.n_pad) : 0.f;
+        }
         for (int i = 0; i < ntiles; ++i) {
             const int buf = i & 1;
             if (!mbar_wait(&sm.p_empty[buf], ((i >> 1) & 1) ^ 1)) { ok = false; break; }
-            const int n = t_begin + i * TILE + t;
-            const bool valid = n < t_end;
-            const float* sp = p.scores + (long long)s * p.H_q * p.n_pad + n;
-            const uint32_t pb = smem_u32(sm.P[buf][t >> 6]);
-            const int tc = t & 63;
-            // all scores of this token first, so that the loads are in flight together: a load scheduled after
-            // one of the (generic-address) stores below would have to wait for it, one memory latency per head
-            float sv[HQ];
-#pragma unroll
-            for (int h = 0; h < HQ; ++h) sv[h] = valid ? __ldg(sp + (long long)h * p.n_pad) : -INFINITY;
-            {
-                // every loaded value is consumed before the first store is issued; a NaN among the scores means
-                // non-finite numbers in the cache, the factors or the query
-                float ssum = 0.f;
-#pragma unroll
-                for (int h = 0; h < HQ; ++h) ssum += valid ? sv[h] : 0.f;
-                if (ssum != ssum) lorc_set_status(p.status, LORC_ERR_ARG);
-            }
+            const bool valid = t_begin + i * TILE + t < t_end;
+            // p = 2^(s - m), rounded to bf16 (the same rounded value enters the denominator)
+            bf16 pr[HQ];
+            float ssum = 0.f;
 #pragma unroll
             for (int h = 0; h < HQ; ++h) {
-                const float pv = valid ? exp2f(sv[h] - sm.m_s[h]) : 0.f;
-                const bf16 pr = __float2bfloat16_rn(pv);
-                l[h] += __bfloat162float(pr);
+                ssum += sv[h];
+                pr[h] = __float2bfloat16_rn(valid ? exp2f(sv[h] - sm.m_s[h]) : 0.f);
+                l[h] += __bfloat162float(pr[h]);
+            }
+            // a NaN among the scores means non-finite numbers in the cache, the factors or the query
+            if (ssum != ssum) lorc_set_status(p.status, LORC_ERR_ARG);
+            {
+                const int nn = t_begin + (i + 1) * TILE + t;
+                const float* sp = p.scores + (long long)s * p.H_q * p.n_pad + nn;
+#pragma unroll
+                for (int h = 0; h < HQ; ++h) sv[h] = (i + 1 < ntiles && nn < t_end) ? ldg_nc_f32(sp + (long long)h * p.n_pad) : 0.f;
+            }
+            const uint32_t pb = smem_u32(sm.P[buf][t >> 6]);
+            const int tc = t & 63;
+#pragma unroll
+            for (int h = 0; h < HQ; ++h) {
                 const int off = h * 128 + ((((tc >> 3) ^ (h & 7)) << 4) | ((tc & 7) << 1));
-                asm volatile("st.shared.b16 [%0], %1;" ::"r"(pb + off), "h"(__bfloat16_as_ushort(pr)) : "memory");
+                asm volatile("st.shared.b16 [%0], %1;" ::"r"(pb + off), "h"(__bfloat16_as_ushort(pr[h])));
             }
             fence_proxy_async_smem();
             mbar_arrive(&sm.p_full[buf]);
@@ -271,43 +290,50 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const __grid_constant
         }
         asm volatile("bar.sync 2, 128;" ::: "memory");
         // out_part[h][j] = sum_rho O_lat[rho][h] * B_V[rho0 + rho][g(h) * 128 + j], thread = column j
-        for (int c = 0; c < n_bv; ++c) {
-            const int slot = c % P_STAGES;
+        {
             float acc[G_MAX];
+            for (int c = 0; c < n_bv; ++c) {
+                const int slot = c % BV_SLOTS, g = c >> 1, half = c & 1;
+                if (half == 0) {
 #pragma unroll
-            for (int i = 0; i < G_MAX; ++i) acc[i] = 0.f;
-            if (ok && !mbar_wait(&sm.bv_full[slot], (c / P_STAGES) & 1)) ok = false;
-            if (ok) {
-                const bf16* bv = sm.V[slot][0] + t;
-                if (G == 4) {
-#pragma unroll 8
-                    for (int r = 0; r < rows_valid; ++r) {
-                        const float b = __bfloat162float(bv[r * 128]);
-                        const float4 o = *reinterpret_cast<const float4*>(&sm.o_sm[r][c * 4]);
-                        acc[0] = fmaf(o.x, b, acc[0]);
-                        acc[1] = fmaf(o.y, b, acc[1]);
-                        acc[2] = fmaf(o.z, b, acc[2]);
-                        acc[3] = fmaf(o.w, b, acc[3]);
-                    }
-                } else {
-#pragma unroll 4
-                    for (int r = 0; r < rows_valid; ++r) {
-                        const float b = __bfloat162float(bv[r * 128]);
-                        const float4 o0 = *reinterpret_cast<const float4*>(&sm.o_sm[r][c * 8]);
-                        const float4 o1 = *reinterpret_cast<const float4*>(&sm.o_sm[r][c * 8 + 4]);
-                        acc[0] = fmaf(o0.x, b, acc[0]);
-                        acc[1] = fmaf(o0.y, b, acc[1]);
-                        acc[2] = fmaf(o0.z, b, acc[2]);
-                        acc[3] = fmaf(o0.w, b, acc[3]);
-                        acc[4] = fmaf(o1.x, b, acc[4]);
-                        acc[5] = fmaf(o1.y, b, acc[5]);
-                        acc[6] = fmaf(o1.z, b, acc[6]);
-                        acc[7] = fmaf(o1.w, b, acc[7]);
-                    }
+                    for (int i = 0; i < G_MAX; ++i) acc[i] = 0.f;
                 }
-                mbar_arrive(&sm.bv_empty[slot]);
+                if (ok && !mbar_wait(&sm.bv_full[slot], (c / BV_SLOTS) & 1)) ok = false;
+                if (ok) {
+                    const bf16* bv = ((slot < 4) ? (&sm.V[0][0][0] + slot * 64 * 128) : &sm.P[0][0][0]) + t;
+                    const int r_lo = half * 64;
+                    const int rows = max(0, min(64, rows_valid - r_lo));
+                    if (G == 4) {
+#pragma unroll 8
+                        for (int r = 0; r < rows; ++r) {
+                            const float b = __bfloat162float(bv[r * 128]);
+                            const float4 o = *reinterpret_cast<const float4*>(&sm.o_sm[r_lo + r][g * 4]);
+                            acc[0] = fmaf(o.x, b, acc[0]);
+                            acc[1] = fmaf(o.y, b, acc[1]);
+                            acc[2] = fmaf(o.z, b, acc[2]);
+                            acc[3] = fmaf(o.w, b, acc[3]);
+                        }
+                    } else {
+#pragma unroll 4
+                        for (int r = 0; r < rows; ++r) {
+                            const float b = __bfloat162float(bv[r * 128]);
+                            const float4 o0 = *reinterpret_cast<const float4*>(&sm.o_sm[r_lo + r][g * 8]);
+                            const float4 o1 = *reinterpret_cast<const float4*>(&sm.o_sm[r_lo + r][g * 8 + 4]);
+                            acc[0] = fmaf(o0.x, b, acc[0]);
+                            acc[1] = fmaf(o0.y, b, acc[1]);
+                            acc[2] = fmaf(o0.z, b, acc[2]);
+                            acc[3] = fmaf(o0.w, b, acc[3]);
+                            acc[4] = fmaf(o1.x, b, acc[4]);
+                            acc[5] = fmaf(o1.y, b, acc[5]);
+                            acc[6] = fmaf(o1.z, b, acc[6]);
+                            acc[7] = fmaf(o1.w, b, acc[7]);
+                        }
+                    }
+                    mbar_arrive(&sm.bv_empty[slot]);
+                }
+                if (half == 1)
+                    for (int i = 0; i < G; ++i) op[(long long)(g * G + i) * 128 + t] = ok ? acc[i] : 0.f;
             }
-            for (int i = 0; i < G; ++i) op[(long long)(c * G + i) * 128 + t] = ok ? acc[i] : 0.f;
         }
         if (ntiles == 0) {
             for (int h = 0; h < HQ; ++h) op[(long long)h * 128 + t] = 0.f;
