@@ -27,6 +27,7 @@ struct LorcLayer {
     bf16* B_k = nullptr;       // [r_k, n]   (LATENT)
     bf16* B_v = nullptr;       // [r_v, n]   (LATENT)
     bf16* B_kT = nullptr;      // [n, r_k]   transposed copy (K-major operand of the key reconstruction)
+    bf16* B_vT = nullptr;      // [n, r_v]   transposed copy (K-major operand of the value up-projection)
 };
 
 struct LorcTcState;            // tensor-core path's private per-context state

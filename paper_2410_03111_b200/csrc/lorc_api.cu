@@ -25,6 +25,7 @@ void free_layer(LorcLayer& L) {
     cudaFree(L.B_k);
     cudaFree(L.B_v);
     cudaFree(L.B_kT);
+    cudaFree(L.B_vT);
     L = LorcLayer();
 }
 
@@ -195,6 +196,7 @@ int lorc_load_factors(lorc_ctx* ctx, int layer, int mode, int r_k, int r_v, cons
         e = cudaMalloc(&L.B_k, (size_t)r_k * n * sizeof(bf16));
         if (e == cudaSuccess) e = cudaMalloc(&L.B_v, (size_t)r_v * n * sizeof(bf16));
         if (e == cudaSuccess) e = cudaMalloc(&L.B_kT, (size_t)r_k * n * sizeof(bf16));
+        if (e == cudaSuccess) e = cudaMalloc(&L.B_vT, (size_t)r_v * n * sizeof(bf16));
     }
     if (e == cudaSuccess)
         e = cudaMemcpy2DAsync(L.A_cat, (size_t)R * sizeof(bf16), A_k, (size_t)r_k * sizeof(bf16),
@@ -208,6 +210,7 @@ int lorc_load_factors(lorc_ctx* ctx, int layer, int mode, int r_k, int r_v, cons
         if (e == cudaSuccess)
             e = cudaMemcpyAsync(L.B_v, B_v, (size_t)r_v * n * sizeof(bf16), cudaMemcpyDeviceToDevice, st);
         if (e == cudaSuccess) e = lorc_generic_transpose(L.B_k, L.B_kT, r_k, n, st);
+        if (e == cudaSuccess) e = lorc_generic_transpose(L.B_v, L.B_vT, r_v, n, st);
     }
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) {

@@ -27,7 +27,6 @@ namespace {
 constexpr int TILE = 128;            // tokens per tile
 constexpr int KC = 64;               // latent columns per pipeline stage
 constexpr float LOG2E = 1.4426950408889634f;
-constexpr float LN2 = 0.6931471805599453f;
 
 // ------------------------------------------------------------------------------------------------
 // score kernel
@@ -287,7 +286,7 @@ __global__ void rope_tile_kernel(float2* out, double theta) {
 // ------------------------------------------------------------------------------------------------
 struct LorcTcLayer {
     bool has_bkt = false;
-    CUtensorMap mapBKT, mapBV;          // B_K^T in 64 x 256 swizzled boxes; B_V in plain 64-row x 128-column boxes
+    CUtensorMap mapBKT, mapBVT;         // B_K^T in 64 x 256 swizzled boxes; B_V^T in 64 x 128 swizzled boxes
     // cache maps are rebuilt only when the cache geometry or pointers change
     const void* k_ptr = nullptr;
     const void* v_ptr = nullptr;
@@ -403,9 +402,9 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
         uint64_t dims[2] = {(uint64_t)L.r_k, (uint64_t)ctx->n}, str[1] = {(uint64_t)L.r_k * 2};
         uint32_t box[2] = {KC, 256};
         if (!lorc_make_tmap_bf16(&TL.mapBKT, L.B_kT, 2, dims, str, box)) return cudaErrorInvalidValue;
-        uint64_t d2[2] = {(uint64_t)ctx->n, (uint64_t)L.r_v}, s2[1] = {(uint64_t)ctx->n * 2};
-        uint32_t b2[2] = {128, 64};
-        if (!lorc_make_tmap_bf16(&TL.mapBV, L.B_v, 2, d2, s2, b2, false)) return cudaErrorInvalidValue;
+        uint64_t d2[2] = {(uint64_t)L.r_v, (uint64_t)ctx->n}, s2[1] = {(uint64_t)L.r_v * 2};
+        uint32_t b2[2] = {KC, 128};
+        if (!lorc_make_tmap_bf16(&TL.mapBVT, L.B_vT, 2, d2, s2, b2)) return cudaErrorInvalidValue;
         TL.has_bkt = true;
     }
     if (!build_cache_maps(TL, L, cv)) return cudaErrorInvalidValue;
@@ -439,6 +438,6 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
     *launches += 1;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    return lorc_tc_pv_launch(ctx, L, cv, TL.mapCV, TL.mapBV, scores, tmax, n_pad, tiles, n_splits, pv_scratch, pv_bytes,
+    return lorc_tc_pv_launch(ctx, L, cv, TL.mapCV, TL.mapBVT, scores, tmax, n_pad, tiles, n_splits, pv_scratch, pv_bytes,
                              out, st, launches);
 }

@@ -18,13 +18,13 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
 cudaError_t lorc_tc_append(lorc_ctx* ctx, int layer, const LorcLayer& L, const CacheView& cv,
                            const bf16* x, int T, cudaStream_t st, int* launches);
 
-// Softmax + P.C_V + value up-projection (tc_pv.cu).  scores [b, H_q, n_pad] (log2 units) and
+// Softmax + P.C_V and value up-projection (tc_pv.cu).  scores [b, H_q, n_pad] (log2 units) and
 // tmax [b, H_q, tiles, 4] (maxima of each 32-token quarter tile) come from the score kernel.
-// mapCV: C_V cache in 64-column x 128-row (or page-sized) swizzled boxes; mapBV: B_V [r_v, n] in plain
-// boxes of 64 rows x 128 columns.  Launches the PV kernel and the kernel that adds its pieces into `out`.
+// mapCV: C_V cache in 64-column x 128-row (or page-sized) swizzled boxes; mapBVT: B_V^T [n, r_v] in swizzled
+// boxes of 64 latent columns x 128 rows.  Launches the PV kernel and the up-projection kernel that writes `out`.
 size_t lorc_tc_pv_scratch_bytes(const lorc_ctx* ctx, int batch, int max_seq_len);
 cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, const CUtensorMap& mapCV,
-                              const CUtensorMap& mapBV, const float* scores, const float* tmax, int n_pad, int tiles,
+                              const CUtensorMap& mapBVT, const float* scores, const float* tmax, int n_pad, int tiles,
                               int n_splits_hint, void* scratch, size_t scratch_bytes, bf16* out, cudaStream_t st,
                               int* launches);
 

@@ -1,17 +1,18 @@
-// Softmax + P.C_V + value up-projection on the tensor cores, split by LATENT COLUMNS.
+// Softmax + P.C_V, split by LATENT COLUMNS, and the value up-projection, both on the tensor cores.
 //
-// A CTA owns one 128-column block of C_V (rho in [128 blk, 128 blk + 128)) of one sequence and one
-// share of its context.  Because a block of latent columns is disjoint from every other block, the
-// CTA's accumulator O_lat^T[128 rho, H_q] (fp32 in TMEM) needs no merge with other column blocks;
-// and because every CTA uses the same exact row maximum (taken from the quarter-tile maxima the score
-// kernel leaves behind), context shares of the same block add up directly.  The CTA therefore
-// finishes its own piece of the output, out_part[h, :] = sum_rho O_lat[h, rho] B_V[rho, g(h)], against
-// the 128 rows of B_V it owns, and writes 16 KiB (H_q = 32) instead of a full latent-space partial.
-// A small kernel adds the pieces in a fixed order and divides by the softmax denominator, so results
-// do not depend on scheduling.
+// PV kernel.  A CTA owns one 128-column block of C_V (rho in [128 blk, 128 blk + 128)) of one sequence
+// and one share of its context.  A block of latent columns is disjoint from every other block, so the
+// CTA's accumulator O_lat^T[128 rho, H_q] (fp32 in TMEM) needs no merge with other column blocks; and
+// every CTA uses the same exact row maximum (from the quarter-tile maxima the score kernel leaves
+// behind), so the context shares of a block simply add.  Each CTA writes its 128 x H_q piece of the
+// un-normalised latent output and, for block 0, its share of the softmax denominator.
 //
 //   per tile of 128 tokens:  p = 2^(s - m) (bf16, K-major in shared memory)        softmax warps
 //                            O_lat^T += C_V[tile, block]^T . P^T                    tcgen05, MN-major A
+//
+// Up-projection kernel.  One CTA per (KV head g, 128 output rows = 128 / G sequences): builds the
+// normalised latent rows o[(s, i), rho] = sum_shares O_lat / l in bf16, 64 columns at a time, and
+// multiplies by B_V[:, g] (TMA-staged from a transposed copy): out = o . B_V[:, g] in TMEM, then bf16.
 #include <math.h>
 
 #include "sm100_ptx.cuh"
@@ -26,7 +27,6 @@ constexpr int KC = 64;
 constexpr int P_STAGES = 2;          // 2 x 32 KiB: two CTAs fit on an SM
 constexpr int P_THREADS = 192;       // warp 0 TMA, warp 1 MMA, warps 2..5 softmax / epilogue
 constexpr int P_SOFT = 128;
-constexpr int BV_SLOTS = 5;           // B_V pieces of 64 rows (16 KiB): four in the C_V stages, one in the P buffers
 
 // read-only global load that the compiler keeps in program order with the other volatile asm of this file
 __device__ __forceinline__ float ldg_nc_f32(const float* p) {
@@ -37,20 +37,18 @@ __device__ __forceinline__ float ldg_nc_f32(const float* p) {
 
 template <int HQ>
 struct Pv2Smem {
-    bf16 V[P_STAGES][2][TILE * KC];       // C_V block: two 64-column halves of [128 tokens][64]; 32 KiB / stage.
-                                          // After the last MMA: ring of B_V pieces [64 rho][128 columns of one KV head]
+    bf16 V[P_STAGES][2][TILE * KC];       // C_V block: two 64-column halves of [128 tokens][64]; 32 KiB / stage
     bf16 P[2][2][HQ * KC];                // probabilities [HQ][128 tokens] as two 64-token chunks, 128-byte swizzle
-    float o_sm[128][HQ];                  // O_lat block [rho][head] after the last MMA
     float m_s[HQ];
     float red[4][HQ];
-    uint64_t full[P_STAGES], empty[P_STAGES], p_full[2], p_empty[2], o_full, bv_full[BV_SLOTS], bv_empty[BV_SLOTS];
+    uint64_t full[P_STAGES], empty[P_STAGES], p_full[2], p_empty[2], o_full;
     uint32_t tmem_base;
 };
 
 struct Pv2Params {
     const float* scores;           // [b, H_q, n_pad]      log2 units
     const float* tmax;             // [b, H_q, tiles, 4]   maxima of every 32-token quarter tile
-    float* out_part;               // [b, n_blk * n_csplit, H_q, 128]
+    float* o_part;                 // [b, n_csplit, H_q, r_pad]   un-normalised latent output, r_pad = 128 n_blk
     float* l_part;                 // [b, n_csplit, H_q]
     const int32_t* seq_lens;
     const int32_t* page_table;
@@ -61,16 +59,13 @@ struct Pv2Params {
 
 template <int HQ>
 __global__ void __launch_bounds__(P_THREADS, 2)
-lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const __grid_constant__ CUtensorMap mapBV,
-                const Pv2Params p) {
+lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
     extern __shared__ uint8_t raw[];
     typedef Pv2Smem<HQ> S;
     S& sm = *reinterpret_cast<S*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
-    constexpr int G_MAX = 8;
     constexpr uint32_t TM_COLS = HQ <= 32 ? 32 : 64;
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
     const int blk = blockIdx.x, cs = blockIdx.y, s = blockIdx.z;
-    const int G = HQ / p.n_kv;
 
     int len = p.seq_lens[s];
     if (len > p.max_pos) {
@@ -85,17 +80,11 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const __grid_constant
     const int ntiles = tile_hi - tile_lo;
     const int t_begin = tile_lo * TILE, t_end = min(len, tile_hi * TILE);
     const int rho0 = blk * 128;
-    const int rows_valid = min(128, p.r_v - rho0);       // latent rows of this block that exist
-    const int n_bv = (ntiles > 0) ? 2 * p.n_kv : 0;      // B_V pieces to stream: (KV head, half of the block's rows)
 
     if (tid == 0) {
         for (int i = 0; i < P_STAGES; ++i) {
             mbar_init(&sm.full[i], 1);
             mbar_init(&sm.empty[i], 1);
-        }
-        for (int i = 0; i < BV_SLOTS; ++i) {
-            mbar_init(&sm.bv_full[i], 1);
-            mbar_init(&sm.bv_empty[i], P_SOFT);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&sm.p_full[i], P_SOFT);
@@ -104,7 +93,6 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const __grid_constant
         mbar_init(&sm.o_full, 1);
         fence_barrier_init();
         prefetch_tensormap(&mapCV);
-        prefetch_tensormap(&mapBV);
     }
     if (warp == 1) {
         tmem_alloc(&sm.tmem_base, TM_COLS);
@@ -146,16 +134,6 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const __grid_constant
                         tma_load_3d(sm.V[st][1] + pg * p.page_size * KC, &mapCV, &sm.full[st], rho0 + 64, 0, page);
                     }
                 }
-            }
-            // the rows of B_V this block multiplies with, in pieces of 64 rows x 128 columns (one KV head), through a
-            // ring that reuses the C_V stages and the P buffers (all free once every MMA has retired)
-            if (n_bv > 0 && ok && !mbar_wait(&sm.o_full, 0)) ok = false;
-            for (int c = 0; c < n_bv && ok; ++c) {
-                const int slot = c % BV_SLOTS;
-                if (!mbar_wait(&sm.bv_empty[slot], ((c / BV_SLOTS) & 1) ^ 1)) { ok = false; break; }
-                bf16* dst = (slot < 4) ? (&sm.V[0][0][0] + slot * 64 * 128) : &sm.P[0][0][0];
-                mbar_arrive_expect_tx(&sm.bv_full[slot], 64 * 128 * 2);
-                tma_load_2d(dst, &mapBV, &sm.bv_full[slot], (c >> 1) * 128, rho0 + (c & 1) * 64);
             }
             if (!ok) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
         }
@@ -267,76 +245,28 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const __grid_constant
             p.l_part[((long long)s * p.n_csplit + cs) * p.H_q + t] =
                 (ntiles > 0 && ok) ? sm.red[0][t] + sm.red[1][t] + sm.red[2][t] + sm.red[3][t] : 0.f;
 
-        float* op = p.out_part + (((long long)s * (p.n_blk * p.n_csplit) + blk * p.n_csplit + cs) * p.H_q) * 128;
+        // this CTA's piece of the un-normalised latent output: TMEM lane = latent row of the block
         if (ntiles > 0 && ok) {
             if (!mbar_wait(&sm.o_full, 0)) ok = false;
         }
-        if (ntiles > 0 && ok) {
-            tc_fence_after_sync();
-            // TMEM lane = latent row of the block; this warp reads lane quarter (warp % 4)
+        {
             const int quarter = warp % 4;
-            const int row = quarter * 32 + lane;
+            const int r_pad = p.n_blk * 128;
+            float* op = p.o_part + (((long long)s * p.n_csplit + cs) * p.H_q) * r_pad + rho0 + quarter * 32 + lane;
+            if (ntiles > 0 && ok) tc_fence_after_sync();
 #pragma unroll
             for (int c0 = 0; c0 < HQ; c0 += 32) {
                 uint32_t r[32];
-                tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + c0, r);
-                tmem_wait_ld();
+                if (ntiles > 0 && ok) {
+                    tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + c0, r);
+                    tmem_wait_ld();
+                } else {
 #pragma unroll
-                for (int i4 = 0; i4 < 8; ++i4)
-                    *reinterpret_cast<float4*>(&sm.o_sm[row][c0 + i4 * 4]) =
-                        make_float4(__uint_as_float(r[i4 * 4]), __uint_as_float(r[i4 * 4 + 1]),
-                                    __uint_as_float(r[i4 * 4 + 2]), __uint_as_float(r[i4 * 4 + 3]));
-            }
-        }
-        asm volatile("bar.sync 2, 128;" ::: "memory");
-        // out_part[h][j] = sum_rho O_lat[rho][h] * B_V[rho0 + rho][g(h) * 128 + j], thread = column j
-        {
-            float acc[G_MAX];
-            for (int c = 0; c < n_bv; ++c) {
-                const int slot = c % BV_SLOTS, g = c >> 1, half = c & 1;
-                if (half == 0) {
+                    for (int i = 0; i < 32; ++i) r[i] = 0u;
+                }
 #pragma unroll
-                    for (int i = 0; i < G_MAX; ++i) acc[i] = 0.f;
-                }
-                if (ok && !mbar_wait(&sm.bv_full[slot], (c / BV_SLOTS) & 1)) ok = false;
-                if (ok) {
-                    const bf16* bv = ((slot < 4) ? (&sm.V[0][0][0] + slot * 64 * 128) : &sm.P[0][0][0]) + t;
-                    const int r_lo = half * 64;
-                    const int rows = max(0, min(64, rows_valid - r_lo));
-                    if (G == 4) {
-#pragma unroll 8
-                        for (int r = 0; r < rows; ++r) {
-                            const float b = __bfloat162float(bv[r * 128]);
-                            const float4 o = *reinterpret_cast<const float4*>(&sm.o_sm[r_lo + r][g * 4]);
-                            acc[0] = fmaf(o.x, b, acc[0]);
-                            acc[1] = fmaf(o.y, b, acc[1]);
-                            acc[2] = fmaf(o.z, b, acc[2]);
-                            acc[3] = fmaf(o.w, b, acc[3]);
-                        }
-                    } else {
-#pragma unroll 4
-                        for (int r = 0; r < rows; ++r) {
-                            const float b = __bfloat162float(bv[r * 128]);
-                            const float4 o0 = *reinterpret_cast<const float4*>(&sm.o_sm[r_lo + r][g * 8]);
-                            const float4 o1 = *reinterpret_cast<const float4*>(&sm.o_sm[r_lo + r][g * 8 + 4]);
-                            acc[0] = fmaf(o0.x, b, acc[0]);
-                            acc[1] = fmaf(o0.y, b, acc[1]);
-                            acc[2] = fmaf(o0.z, b, acc[2]);
-                            acc[3] = fmaf(o0.w, b, acc[3]);
-                            acc[4] = fmaf(o1.x, b, acc[4]);
-                            acc[5] = fmaf(o1.y, b, acc[5]);
-                            acc[6] = fmaf(o1.z, b, acc[6]);
-                            acc[7] = fmaf(o1.w, b, acc[7]);
-                        }
-                    }
-                    mbar_arrive(&sm.bv_empty[slot]);
-                }
-                if (half == 1)
-                    for (int i = 0; i < G; ++i) op[(long long)(g * G + i) * 128 + t] = ok ? acc[i] : 0.f;
+                for (int i = 0; i < 32; ++i) op[(long long)(c0 + i) * r_pad] = __uint_as_float(r[i]);
             }
-        }
-        if (ntiles == 0) {
-            for (int h = 0; h < HQ; ++h) op[(long long)h * 128 + t] = 0.f;
         }
         if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
     }
@@ -349,35 +279,170 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const __grid_constant
 
 namespace {
 
-// out[s][h][:] = (sum over pieces of out_part) / (sum over context shares of l), pieces added in index order.
-// grid (H_q / 4, batch), 512 threads = 4 heads x 128 columns.
-__global__ void __launch_bounds__(512)
-lorc_pv_finalize_kernel(const float* __restrict__ out_part, const float* __restrict__ l_part, bf16* __restrict__ out,
-                        int H_q, int n_parts, int n_csplit, int* status) {
-    const int s = blockIdx.y;
-    const int h = blockIdx.x * 4 + (threadIdx.x >> 7), j = threadIdx.x & 127;
-    float L = 0.f;
-    for (int c = 0; c < n_csplit; ++c) L += l_part[((long long)s * n_csplit + c) * H_q + h];
-    const float* op = out_part + ((long long)s * n_parts * H_q + h) * 128 + j;
-    float a = 0.f;
-    int c = 0;
-    for (; c + 8 <= n_parts; c += 8) {
-        float v[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) v[u] = op[(long long)(c + u) * H_q * 128];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) a += v[u];
+// ------------------------------------------------------------------------------------------------
+// value up-projection: out[(s, h), :] = (sum_shares O_lat[s, share, h, :] / l[s, h]) . B_V[:, g(h)]
+// grid (n_kv_heads, ceil(batch * G / 128)); warp 0 TMA (B_V^T slices), warp 1 MMA, warps 2..5 build
+// the A operand (one output row per thread) and write the result.
+// ------------------------------------------------------------------------------------------------
+constexpr int U_BSTAGES = 4;
+constexpr int U_THREADS = 192;
+
+struct UpSmem {
+    bf16 A[2][128 * KC];                  // normalised latent rows [128 rows][64 rho], K-major, 128-byte swizzle
+    bf16 B[U_BSTAGES][128 * KC];          // B_V^T slice [128 columns j][64 rho] by TMA
+    uint64_t a_full[2], a_empty[2], b_full[U_BSTAGES], b_empty[U_BSTAGES], d_full;
+    uint32_t tmem_base;
+};
+
+struct UpParams {
+    const float* o_part;           // [b, n_csplit, H_q, r_pad]
+    const float* l_part;           // [b, n_csplit, H_q]
+    bf16* out;                     // [b, H_q, 128]
+    int* status;
+    int batch, H_q, G, r_v, r_pad, n_csplit;
+};
+
+__global__ void __launch_bounds__(U_THREADS, 1)
+lorc_upproj_kernel(const __grid_constant__ CUtensorMap mapBVT, const UpParams p) {
+    extern __shared__ uint8_t raw[];
+    UpSmem& sm = *reinterpret_cast<UpSmem*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
+    const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
+    const int g = blockIdx.x, chunk = blockIdx.y;
+    const int nkc = (p.r_v + KC - 1) / KC;
+    if (tid == 0) {
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&sm.a_full[i], 128);
+            mbar_init(&sm.a_empty[i], 1);
+        }
+        for (int i = 0; i < U_BSTAGES; ++i) {
+            mbar_init(&sm.b_full[i], 1);
+            mbar_init(&sm.b_empty[i], 1);
+        }
+        mbar_init(&sm.d_full, 1);
+        fence_barrier_init();
+        prefetch_tensormap(&mapBVT);
     }
-    for (; c < n_parts; ++c) a += op[(long long)c * H_q * 128];
-    if (!(L > 0.f)) {
-        if (j == 0) lorc_set_status(status, LORC_ERR_EMPTY);
-        a = 0.f;
-        L = 1.f;
+    if (warp == 1) {
+        tmem_alloc(&sm.tmem_base, 128);
+        tmem_relinquish();
     }
-    out[((long long)s * H_q + h) * 128 + j] = __float2bfloat16_rn(a / L);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = sm.tmem_base;
+    bool ok = true;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int kc = 0; kc < nkc; ++kc) {
+                const int st = kc % U_BSTAGES;
+                if (!mbar_wait(&sm.b_empty[st], ((kc / U_BSTAGES) & 1) ^ 1)) { ok = false; break; }
+                mbar_arrive_expect_tx(&sm.b_full[st], 128 * KC * 2);
+                tma_load_2d(sm.B[st], &mapBVT, &sm.b_full[st], kc * KC, g * 128);
+            }
+            if (!ok) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc_bf16(128, 128, 0, 0);
+            for (int kc = 0; kc < nkc; ++kc) {
+                const int sa = kc & 1, sb = kc % U_BSTAGES;
+                if (!mbar_wait(&sm.a_full[sa], (kc >> 1) & 1)) { ok = false; break; }
+                if (!mbar_wait(&sm.b_full[sb], (kc / U_BSTAGES) & 1)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t a0 = smem_u32(sm.A[sa]), b0 = smem_u32(sm.B[sb]);
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    tc_mma_bf16(tmem, make_smem_desc_sw128(a0 + k * 32, 0, 1024), make_smem_desc_sw128(b0 + k * 32, 0, 1024),
+                                idesc, (kc | k) != 0);
+                tc_commit(&sm.a_empty[sa]);
+                tc_commit(&sm.b_empty[sb]);
+            }
+            tc_commit(&sm.d_full);
+            if (!ok) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
+        }
+    } else {
+        const int t = tid - 64;                        // output row inside this CTA
+        const int R = chunk * 128 + t;                 // (sequence, head of the group)
+        const int s = R / p.G, i = R - s * p.G;
+        const int h = g * p.G + i;
+        const bool live = s < p.batch;
+        float inv = 0.f;
+        if (live) {
+            float L = 0.f;
+            for (int c = 0; c < p.n_csplit; ++c) L += p.l_part[((long long)s * p.n_csplit + c) * p.H_q + h];
+            if (L > 0.f) inv = 1.f / L;
+            else if (i == 0) lorc_set_status(p.status, LORC_ERR_EMPTY);
+        }
+        const float* orow = p.o_part + ((long long)s * p.n_csplit * p.H_q + h) * p.r_pad;
+        const long long share_stride = (long long)p.H_q * p.r_pad;
+        for (int kc = 0; kc < nkc; ++kc) {
+            const int sa = kc & 1;
+            // the 64 latent columns of this row, summed over the context shares (loads first, then the wait)
+            float4 v[16];
+#pragma unroll
+            for (int q4 = 0; q4 < 16; ++q4) v[q4] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (live && inv != 0.f) {
+                for (int c = 0; c < p.n_csplit; ++c) {
+                    const float4* src = reinterpret_cast<const float4*>(orow + c * share_stride + kc * KC);
+#pragma unroll
+                    for (int q4 = 0; q4 < 16; ++q4) {
+                        const float4 x = __ldg(src + q4);
+                        v[q4].x += x.x; v[q4].y += x.y; v[q4].z += x.z; v[q4].w += x.w;
+                    }
+                }
+            }
+            if (!mbar_wait(&sm.a_empty[sa], ((kc >> 1) & 1) ^ 1)) { ok = false; break; }
+            const uint32_t arow = smem_u32(sm.A[sa]) + t * 128;
+#pragma unroll
+            for (int c8 = 0; c8 < 8; ++c8) {           // 16-byte chunks of the 128-byte row
+                const float4 x = v[2 * c8], y = v[2 * c8 + 1];
+                __nv_bfloat162 b0 = __floats2bfloat162_rn(x.x * inv, x.y * inv), b1 = __floats2bfloat162_rn(x.z * inv, x.w * inv);
+                __nv_bfloat162 b2 = __floats2bfloat162_rn(y.x * inv, y.y * inv), b3 = __floats2bfloat162_rn(y.z * inv, y.w * inv);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(arow + ((c8 ^ (t & 7)) << 4)),
+                             "r"(*reinterpret_cast<uint32_t*>(&b0)), "r"(*reinterpret_cast<uint32_t*>(&b1)),
+                             "r"(*reinterpret_cast<uint32_t*>(&b2)), "r"(*reinterpret_cast<uint32_t*>(&b3)));
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(&sm.a_full[sa]);
+        }
+        if (ok && !mbar_wait(&sm.d_full, 0)) ok = false;
+        if (ok) {
+            tc_fence_after_sync();
+            const int quarter = warp % 4;
+            // TMEM lane = output row; the warp's lane quarter decides which rows it can read
+            const int row = quarter * 32 + lane;
+            const int R2 = chunk * 128 + row;
+            const int s2 = R2 / p.G, h2 = g * p.G + (R2 - s2 * p.G);
+#pragma unroll
+            for (int c0 = 0; c0 < 128; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + c0, r);
+                tmem_wait_ld();
+                if (s2 < p.batch) {
+                    uint4* dst = reinterpret_cast<uint4*>(p.out + ((long long)s2 * p.H_q + h2) * 128 + c0);
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(r[q4 * 8 + 2 * e]),
+                                                                     __uint_as_float(r[q4 * 8 + 2 * e + 1]));
+                            w[e] = *reinterpret_cast<uint32_t*>(&b);
+                        }
+                        dst[q4] = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                }
+            }
+        }
+        if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, 128);
 }
 
-// Column blocks and context shares of one launch: two CTAs fit on an SM, so aim at filling those slots once.
+// Column blocks and context shares of one PV launch: two CTAs fit on an SM, so aim at filling those slots once.
 void pv_plan(const lorc_ctx* ctx, const LorcLayer& L, int batch, int max_seq_len, int n_splits_hint, int* n_blk,
              int* n_csplit) {
     const int tiles = (max_seq_len + TILE - 1) / TILE;
@@ -396,19 +461,19 @@ void pv_plan(const lorc_ctx* ctx, const LorcLayer& L, int batch, int max_seq_len
 // host side
 // ------------------------------------------------------------------------------------------------
 size_t lorc_tc_pv_scratch_bytes(const lorc_ctx* ctx, int batch, int max_seq_len) {
-    // any layer (up to n / 128 column blocks) with the number of context shares the plan picks for it, or a
-    // forced share count as far as it fits (the launch lowers the count until the pieces fit)
+    // the planned number of context shares for the narrowest layer (one column block), which is the largest
     const int tiles = (max_seq_len + TILE - 1) / TILE;
-    const int n_blk_max = (ctx->n + 127) / 128;
-    int cs = 2 * ctx->sm_count / batch;          // n_blk * n_csplit <= slots / batch for every n_blk
-    if (cs < n_blk_max) cs = n_blk_max;
-    int cs_l = tiles < 64 ? tiles : 64;
-    return lorc_align_up((size_t)batch * cs * ctx->desc.n_q_heads * 128 * sizeof(float), 256) +
-           lorc_align_up((size_t)batch * cs_l * ctx->desc.n_q_heads * sizeof(float), 256);
+    int cs = 2 * ctx->sm_count / batch;
+    if (cs > tiles) cs = tiles;
+    if (cs > 64) cs = 64;
+    if (cs < 1) cs = 1;
+    const size_t r_pad = (size_t)((ctx->n + 127) / 128) * 128;
+    return lorc_align_up((size_t)batch * cs * ctx->desc.n_q_heads * r_pad * sizeof(float), 256) +
+           lorc_align_up((size_t)batch * cs * ctx->desc.n_q_heads * sizeof(float), 256);
 }
 
 cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, const CUtensorMap& mapCV,
-                              const CUtensorMap& mapBV, const float* scores, const float* tmax, int n_pad, int tiles,
+                              const CUtensorMap& mapBVT, const float* scores, const float* tmax, int n_pad, int tiles,
                               int n_splits_hint, void* scratch, size_t scratch_bytes, bf16* out, cudaStream_t st,
                               int* launches) {
     const lorc_model_desc& d = ctx->desc;
@@ -419,21 +484,25 @@ cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(lorc_pv2_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)sizeof(Pv2Smem<64>) + 1024);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(lorc_upproj_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)sizeof(UpSmem) + 1024);
         if (e != cudaSuccess) return e;
         attr = true;
     }
     int n_blk, n_csplit;
     pv_plan(ctx, L, cv.batch, cv.max_seq_len, n_splits_hint, &n_blk, &n_csplit);
+    const int r_pad = n_blk * 128;
     size_t part_bytes, l_bytes;
     for (;; --n_csplit) {
-        part_bytes = lorc_align_up((size_t)cv.batch * n_blk * n_csplit * d.n_q_heads * 128 * sizeof(float), 256);
+        part_bytes = lorc_align_up((size_t)cv.batch * n_csplit * d.n_q_heads * r_pad * sizeof(float), 256);
         l_bytes = lorc_align_up((size_t)cv.batch * n_csplit * d.n_q_heads * sizeof(float), 256);
         if (part_bytes + l_bytes <= scratch_bytes) break;
         if (n_csplit == 1) return cudaErrorMemoryAllocation;
     }
     Pv2Params p;
     p.scores = scores; p.tmax = tmax;
-    p.out_part = (float*)scratch;
+    p.o_part = (float*)scratch;
     p.l_part = (float*)((char*)scratch + part_bytes);
     p.seq_lens = cv.seq_lens; p.page_table = cv.page_table; p.status = ctx->status_dev;
     p.batch = cv.batch; p.H_q = d.n_q_heads; p.n_kv = d.n_kv_heads; p.r_v = L.r_v; p.n_pad = n_pad; p.tiles = tiles;
@@ -443,17 +512,20 @@ cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView
     {
         LorcStageTimer timer(ctx, LORC_STAGE_PV, st);
         if (d.n_q_heads == 32)
-            lorc_pv2_kernel<32><<<grid, P_THREADS, sizeof(Pv2Smem<32>) + 1024, st>>>(mapCV, mapBV, p);
+            lorc_pv2_kernel<32><<<grid, P_THREADS, sizeof(Pv2Smem<32>) + 1024, st>>>(mapCV, p);
         else
-            lorc_pv2_kernel<64><<<grid, P_THREADS, sizeof(Pv2Smem<64>) + 1024, st>>>(mapCV, mapBV, p);
+            lorc_pv2_kernel<64><<<grid, P_THREADS, sizeof(Pv2Smem<64>) + 1024, st>>>(mapCV, p);
     }
     *launches += 1;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    UpParams u;
+    u.o_part = p.o_part; u.l_part = p.l_part; u.out = out; u.status = ctx->status_dev;
+    u.batch = cv.batch; u.H_q = d.n_q_heads; u.G = ctx->group; u.r_v = L.r_v; u.r_pad = r_pad; u.n_csplit = n_csplit;
     {
         LorcStageTimer timer(ctx, LORC_STAGE_COMBINE, st);
-        lorc_pv_finalize_kernel<<<dim3(d.n_q_heads / 4, cv.batch), 512, 0, st>>>(
-            p.out_part, p.l_part, out, d.n_q_heads, n_blk * n_csplit, n_csplit, ctx->status_dev);
+        dim3 ugrid(d.n_kv_heads, (cv.batch * ctx->group + 127) / 128);
+        lorc_upproj_kernel<<<ugrid, U_THREADS, sizeof(UpSmem) + 1024, st>>>(mapBVT, u);
     }
     *launches += 1;
     return cudaGetLastError();
