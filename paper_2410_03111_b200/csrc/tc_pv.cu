@@ -280,46 +280,88 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
 namespace {
 
 // ------------------------------------------------------------------------------------------------
-// value up-projection: out[(s, h), :] = (sum_shares O_lat[s, share, h, :] / l[s, h]) . B_V[:, g(h)]
-// grid (n_kv_heads, ceil(batch * G / 128)); warp 0 TMA (B_V^T slices), warp 1 MMA, warps 2..5 build
-// the A operand (one output row per thread) and write the result.
+// normalise: o_norm[s, h, rho] = bf16( sum_shares O_lat[s, share, h, rho] / sum_shares l[s, share, h] )
+// one thread per 4 latent columns
 // ------------------------------------------------------------------------------------------------
-constexpr int U_BSTAGES = 4;
+__global__ void __launch_bounds__(256)
+lorc_normalize_kernel(const float* __restrict__ o_part, const float* __restrict__ l_part, bf16* __restrict__ o_norm,
+                      int H_q, int r_pad, int n_csplit, long long total4, int* status) {
+    const long long i4 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i4 >= total4) return;
+    const int r4n = r_pad >> 2;
+    const long long row = i4 / r4n;                   // s * H_q + h
+    const int r4 = (int)(i4 - row * r4n);
+    const int s = (int)(row / H_q), h = (int)(row - (long long)s * H_q);
+    const long long share_stride4 = (long long)H_q * r4n;
+    const float4* src = reinterpret_cast<const float4*>(o_part) + ((long long)s * n_csplit * H_q + h) * r4n + r4;
+    const float* lp = l_part + (long long)s * n_csplit * H_q + h;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    float L = 0.f;
+    int c = 0;
+    for (; c + 4 <= n_csplit; c += 4) {
+        float4 v[4];
+        float l[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            v[u] = __ldg(src + (c + u) * share_stride4);
+            l[u] = __ldg(lp + (long long)(c + u) * H_q);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            a.x += v[u].x; a.y += v[u].y; a.z += v[u].z; a.w += v[u].w;
+            L += l[u];
+        }
+    }
+    for (; c < n_csplit; ++c) {
+        const float4 v = __ldg(src + c * share_stride4);
+        a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+        L += __ldg(lp + (long long)c * H_q);
+    }
+    float inv = 0.f;
+    if (L > 0.f) inv = 1.f / L;
+    else if (r4 == 0) lorc_set_status(status, LORC_ERR_EMPTY);
+    __nv_bfloat162 b0 = __floats2bfloat162_rn(a.x * inv, a.y * inv), b1 = __floats2bfloat162_rn(a.z * inv, a.w * inv);
+    uint2 w = make_uint2(*reinterpret_cast<uint32_t*>(&b0), *reinterpret_cast<uint32_t*>(&b1));
+    reinterpret_cast<uint2*>(o_norm)[i4] = w;
+}
+
+// ------------------------------------------------------------------------------------------------
+// value up-projection: out[(s, h), :] = o_norm[s, h, :] . B_V[:, g(h)], a plain TMA-fed tcgen05 GEMM.
+// grid (n_kv_heads, ceil(batch * G / 128)): 128 output rows (s, i) x 128 columns, K = r_v in slices of 64.
+// ------------------------------------------------------------------------------------------------
+constexpr int U_STAGES = 6;
 constexpr int U_THREADS = 192;
 
 struct UpSmem {
-    bf16 A[2][128 * KC];                  // normalised latent rows [128 rows][64 rho], K-major, 128-byte swizzle
-    bf16 B[U_BSTAGES][128 * KC];          // B_V^T slice [128 columns j][64 rho] by TMA
-    uint64_t a_full[2], a_empty[2], b_full[U_BSTAGES], b_empty[U_BSTAGES], d_full;
+    bf16 A[U_STAGES][128 * KC];           // o_norm rows [128 rows (s, i)][64 rho]
+    bf16 B[U_STAGES][128 * KC];           // B_V^T slice [128 columns j][64 rho]
+    uint64_t full[U_STAGES], empty[U_STAGES], d_full;
     uint32_t tmem_base;
 };
 
 struct UpParams {
-    const float* o_part;           // [b, n_csplit, H_q, r_pad]
-    const float* l_part;           // [b, n_csplit, H_q]
     bf16* out;                     // [b, H_q, 128]
     int* status;
-    int batch, H_q, G, r_v, r_pad, n_csplit;
+    int batch, H_q, G, r_v;
 };
 
 __global__ void __launch_bounds__(U_THREADS, 1)
-lorc_upproj_kernel(const __grid_constant__ CUtensorMap mapBVT, const UpParams p) {
+lorc_upproj_kernel(const __grid_constant__ CUtensorMap mapON, const __grid_constant__ CUtensorMap mapBVT,
+                   const UpParams p) {
     extern __shared__ uint8_t raw[];
     UpSmem& sm = *reinterpret_cast<UpSmem*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
     const int g = blockIdx.x, chunk = blockIdx.y;
     const int nkc = (p.r_v + KC - 1) / KC;
+    const int seqs_per_cta = 128 / p.G;
     if (tid == 0) {
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(&sm.a_full[i], 128);
-            mbar_init(&sm.a_empty[i], 1);
-        }
-        for (int i = 0; i < U_BSTAGES; ++i) {
-            mbar_init(&sm.b_full[i], 1);
-            mbar_init(&sm.b_empty[i], 1);
+        for (int i = 0; i < U_STAGES; ++i) {
+            mbar_init(&sm.full[i], 1);
+            mbar_init(&sm.empty[i], 1);
         }
         mbar_init(&sm.d_full, 1);
         fence_barrier_init();
+        prefetch_tensormap(&mapON);
         prefetch_tensormap(&mapBVT);
     }
     if (warp == 1) {
@@ -335,10 +377,12 @@ lorc_upproj_kernel(const __grid_constant__ CUtensorMap mapBVT, const UpParams p)
     if (warp == 0) {
         if (lane == 0) {
             for (int kc = 0; kc < nkc; ++kc) {
-                const int st = kc % U_BSTAGES;
-                if (!mbar_wait(&sm.b_empty[st], ((kc / U_BSTAGES) & 1) ^ 1)) { ok = false; break; }
-                mbar_arrive_expect_tx(&sm.b_full[st], 128 * KC * 2);
-                tma_load_2d(sm.B[st], &mapBVT, &sm.b_full[st], kc * KC, g * 128);
+                const int st = kc % U_STAGES;
+                if (!mbar_wait(&sm.empty[st], ((kc / U_STAGES) & 1) ^ 1)) { ok = false; break; }
+                mbar_arrive_expect_tx(&sm.full[st], 2 * 128 * KC * 2);
+                // rows (s, i): box of G heads x 128/G sequences (sequences past the batch read as zero)
+                tma_load_3d(sm.A[st], &mapON, &sm.full[st], kc * KC, g * p.G, chunk * seqs_per_cta);
+                tma_load_2d(sm.B[st], &mapBVT, &sm.full[st], kc * KC, g * 128);
             }
             if (!ok) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
         }
@@ -346,81 +390,34 @@ lorc_upproj_kernel(const __grid_constant__ CUtensorMap mapBVT, const UpParams p)
         if (lane == 0) {
             const uint32_t idesc = make_idesc_bf16(128, 128, 0, 0);
             for (int kc = 0; kc < nkc; ++kc) {
-                const int sa = kc & 1, sb = kc % U_BSTAGES;
-                if (!mbar_wait(&sm.a_full[sa], (kc >> 1) & 1)) { ok = false; break; }
-                if (!mbar_wait(&sm.b_full[sb], (kc / U_BSTAGES) & 1)) { ok = false; break; }
+                const int st = kc % U_STAGES;
+                if (!mbar_wait(&sm.full[st], (kc / U_STAGES) & 1)) { ok = false; break; }
                 tc_fence_after_sync();
-                const uint32_t a0 = smem_u32(sm.A[sa]), b0 = smem_u32(sm.B[sb]);
+                const uint32_t a0 = smem_u32(sm.A[st]), b0 = smem_u32(sm.B[st]);
 #pragma unroll
                 for (int k = 0; k < 4; ++k)
                     tc_mma_bf16(tmem, make_smem_desc_sw128(a0 + k * 32, 0, 1024), make_smem_desc_sw128(b0 + k * 32, 0, 1024),
                                 idesc, (kc | k) != 0);
-                tc_commit(&sm.a_empty[sa]);
-                tc_commit(&sm.b_empty[sb]);
+                tc_commit(&sm.empty[st]);
             }
             tc_commit(&sm.d_full);
             if (!ok) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
         }
     } else {
-        const int t = tid - 64;                        // output row inside this CTA
-        const int R = chunk * 128 + t;                 // (sequence, head of the group)
-        const int s = R / p.G, i = R - s * p.G;
-        const int h = g * p.G + i;
-        const bool live = s < p.batch;
-        float inv = 0.f;
-        if (live) {
-            float L = 0.f;
-            for (int c = 0; c < p.n_csplit; ++c) L += p.l_part[((long long)s * p.n_csplit + c) * p.H_q + h];
-            if (L > 0.f) inv = 1.f / L;
-            else if (i == 0) lorc_set_status(p.status, LORC_ERR_EMPTY);
-        }
-        const float* orow = p.o_part + ((long long)s * p.n_csplit * p.H_q + h) * p.r_pad;
-        const long long share_stride = (long long)p.H_q * p.r_pad;
-        for (int kc = 0; kc < nkc; ++kc) {
-            const int sa = kc & 1;
-            // the 64 latent columns of this row, summed over the context shares (loads first, then the wait)
-            float4 v[16];
-#pragma unroll
-            for (int q4 = 0; q4 < 16; ++q4) v[q4] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (live && inv != 0.f) {
-                for (int c = 0; c < p.n_csplit; ++c) {
-                    const float4* src = reinterpret_cast<const float4*>(orow + c * share_stride + kc * KC);
-#pragma unroll
-                    for (int q4 = 0; q4 < 16; ++q4) {
-                        const float4 x = __ldg(src + q4);
-                        v[q4].x += x.x; v[q4].y += x.y; v[q4].z += x.z; v[q4].w += x.w;
-                    }
-                }
-            }
-            if (!mbar_wait(&sm.a_empty[sa], ((kc >> 1) & 1) ^ 1)) { ok = false; break; }
-            const uint32_t arow = smem_u32(sm.A[sa]) + t * 128;
-#pragma unroll
-            for (int c8 = 0; c8 < 8; ++c8) {           // 16-byte chunks of the 128-byte row
-                const float4 x = v[2 * c8], y = v[2 * c8 + 1];
-                __nv_bfloat162 b0 = __floats2bfloat162_rn(x.x * inv, x.y * inv), b1 = __floats2bfloat162_rn(x.z * inv, x.w * inv);
-                __nv_bfloat162 b2 = __floats2bfloat162_rn(y.x * inv, y.y * inv), b3 = __floats2bfloat162_rn(y.z * inv, y.w * inv);
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(arow + ((c8 ^ (t & 7)) << 4)),
-                             "r"(*reinterpret_cast<uint32_t*>(&b0)), "r"(*reinterpret_cast<uint32_t*>(&b1)),
-                             "r"(*reinterpret_cast<uint32_t*>(&b2)), "r"(*reinterpret_cast<uint32_t*>(&b3)));
-            }
-            fence_proxy_async_smem();
-            mbar_arrive(&sm.a_full[sa]);
-        }
-        if (ok && !mbar_wait(&sm.d_full, 0)) ok = false;
+        if (!mbar_wait(&sm.d_full, 0)) ok = false;
         if (ok) {
             tc_fence_after_sync();
+            // TMEM lane = output row (s_local * G + i); the warp's lane quarter decides which rows it reads
             const int quarter = warp % 4;
-            // TMEM lane = output row; the warp's lane quarter decides which rows it can read
             const int row = quarter * 32 + lane;
-            const int R2 = chunk * 128 + row;
-            const int s2 = R2 / p.G, h2 = g * p.G + (R2 - s2 * p.G);
+            const int s = chunk * seqs_per_cta + row / p.G, h = g * p.G + row % p.G;
 #pragma unroll
             for (int c0 = 0; c0 < 128; c0 += 32) {
                 uint32_t r[32];
                 tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + c0, r);
                 tmem_wait_ld();
-                if (s2 < p.batch) {
-                    uint4* dst = reinterpret_cast<uint4*>(p.out + ((long long)s2 * p.H_q + h2) * 128 + c0);
+                if (s < p.batch) {
+                    uint4* dst = reinterpret_cast<uint4*>(p.out + ((long long)s * p.H_q + h) * 128 + c0);
 #pragma unroll
                     for (int q4 = 0; q4 < 4; ++q4) {
                         uint32_t w[4];
@@ -469,7 +466,8 @@ size_t lorc_tc_pv_scratch_bytes(const lorc_ctx* ctx, int batch, int max_seq_len)
     if (cs < 1) cs = 1;
     const size_t r_pad = (size_t)((ctx->n + 127) / 128) * 128;
     return lorc_align_up((size_t)batch * cs * ctx->desc.n_q_heads * r_pad * sizeof(float), 256) +
-           lorc_align_up((size_t)batch * cs * ctx->desc.n_q_heads * sizeof(float), 256);
+           lorc_align_up((size_t)batch * cs * ctx->desc.n_q_heads * sizeof(float), 256) +
+           lorc_align_up((size_t)batch * ctx->desc.n_q_heads * r_pad * sizeof(bf16), 256);
 }
 
 cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, const CUtensorMap& mapCV,
@@ -494,12 +492,14 @@ cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView
     pv_plan(ctx, L, cv.batch, cv.max_seq_len, n_splits_hint, &n_blk, &n_csplit);
     const int r_pad = n_blk * 128;
     size_t part_bytes, l_bytes;
+    const size_t on_bytes = lorc_align_up((size_t)cv.batch * d.n_q_heads * r_pad * sizeof(bf16), 256);
     for (;; --n_csplit) {
         part_bytes = lorc_align_up((size_t)cv.batch * n_csplit * d.n_q_heads * r_pad * sizeof(float), 256);
         l_bytes = lorc_align_up((size_t)cv.batch * n_csplit * d.n_q_heads * sizeof(float), 256);
-        if (part_bytes + l_bytes <= scratch_bytes) break;
+        if (part_bytes + l_bytes + on_bytes <= scratch_bytes) break;
         if (n_csplit == 1) return cudaErrorMemoryAllocation;
     }
+    bf16* o_norm = (bf16*)((char*)scratch + part_bytes + l_bytes);
     Pv2Params p;
     p.scores = scores; p.tmax = tmax;
     p.o_part = (float*)scratch;
@@ -519,14 +519,26 @@ cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView
     *launches += 1;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    UpParams u;
-    u.o_part = p.o_part; u.l_part = p.l_part; u.out = out; u.status = ctx->status_dev;
-    u.batch = cv.batch; u.H_q = d.n_q_heads; u.G = ctx->group; u.r_v = L.r_v; u.r_pad = r_pad; u.n_csplit = n_csplit;
+    LorcStageTimer timer(ctx, LORC_STAGE_COMBINE, st);
+    const long long total4 = (long long)cv.batch * d.n_q_heads * (r_pad / 4);
+    lorc_normalize_kernel<<<(unsigned)((total4 + 255) / 256), 256, 0, st>>>(p.o_part, p.l_part, o_norm, d.n_q_heads, r_pad,
+                                                                        n_csplit, total4, ctx->status_dev);
+    *launches += 1;
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    // o_norm [b, H_q, r_pad] as (rho, head, sequence) with boxes of 64 rho x G heads x 128/G sequences
+    CUtensorMap mapON;
     {
-        LorcStageTimer timer(ctx, LORC_STAGE_COMBINE, st);
-        dim3 ugrid(d.n_kv_heads, (cv.batch * ctx->group + 127) / 128);
-        lorc_upproj_kernel<<<ugrid, U_THREADS, sizeof(UpSmem) + 1024, st>>>(mapBVT, u);
+        uint64_t dims[3] = {(uint64_t)r_pad, (uint64_t)d.n_q_heads, (uint64_t)cv.batch};
+        uint64_t str[2] = {(uint64_t)r_pad * 2, (uint64_t)d.n_q_heads * r_pad * 2};
+        uint32_t box[3] = {KC, (uint32_t)ctx->group, (uint32_t)(128 / ctx->group)};
+        if (!lorc_make_tmap_bf16(&mapON, o_norm, 3, dims, str, box)) return cudaErrorInvalidValue;
     }
+    UpParams u;
+    u.out = out; u.status = ctx->status_dev;
+    u.batch = cv.batch; u.H_q = d.n_q_heads; u.G = ctx->group; u.r_v = L.r_v;
+    dim3 ugrid(d.n_kv_heads, (cv.batch * ctx->group + 127) / 128);
+    lorc_upproj_kernel<<<ugrid, U_THREADS, sizeof(UpSmem) + 1024, st>>>(mapON, mapBVT, u);
     *launches += 1;
     return cudaGetLastError();
 }
