@@ -2,9 +2,11 @@
 //
 // Two kernels per layer, followed by a small kernel that adds up the output pieces:
 //
-//  score kernel   persistent CTAs walk (sequence, 128-token tile, KV-head pair) units.  Per unit the
-//                 key tile of two KV heads is reconstructed on the tensor cores,
-//                     K[128 tokens, 256] = C_K[tile, :] . B_K[:, pair]          (fp32 in TMEM),
+//  score kernel   persistent CTA PAIRS (clusters of two, cta_group::2 MMAs) walk (sequence, two consecutive
+//                 128-token tiles, KV-head pair) units.  Per unit the key tiles of two KV heads are
+//                 reconstructed on the tensor cores, each CTA holding its own 128 tokens and HALF of the
+//                 B_K^T slice (the pair shares it, which halves the shared-memory traffic per FLOP),
+//                     K[256 tokens, 256] = C_K[tiles, :] . B_K[:, pair]         (fp32 in both CTAs' TMEM),
 //                 from TMA-staged 64-wide slices of the latent tile and of B_K^T.  Eight epilogue warps
 //                 (thread = token row) read the accumulator, rotate each key at its position and dot it
 //                 with the G rotated queries of its KV head; the scores (log2 units) go to scratch.
@@ -17,6 +19,7 @@
 // Keys and values never exist in memory; only the 4*H_q bytes of scores per token are written.
 #include <math.h>
 
+#include "sm100_pair.cuh"
 #include "sm100_ptx.cuh"
 #include "tc_kernels.cuh"
 
@@ -31,18 +34,17 @@ constexpr float LOG2E = 1.4426950408889634f;
 // ------------------------------------------------------------------------------------------------
 // score kernel
 // ------------------------------------------------------------------------------------------------
-constexpr int S_STAGES = 3;
+constexpr int S_STAGES = 4;
 constexpr int S_THREADS = 320;       // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
 constexpr int S_EPI = 256;
 
 struct ScoreSmem {
     bf16 A[S_STAGES][TILE * KC];          // latent slice  [128 tokens][64]       16 KiB
-    bf16 B[S_STAGES][256 * KC];           // B_K^T slice   [256 features][64]     32 KiB
+    bf16 B[S_STAGES][128 * KC];           // this CTA's half of the B_K^T slice [128 features][64]   16 KiB
     float2 trigT[64][TILE];               // (cos, sin)(t * theta_j), [j][t]      64 KiB
     float qrot[2][2][64][16];             // [buffer][head of pair][pair j][qa_0..qa_G-1, qb_0..qb_G-1]  16 KiB
     uint64_t full[S_STAGES], empty[S_STAGES], acc_full[2], acc_empty[2];
     uint32_t tmem_base;
-    int abort_flag;
 };
 
 struct ScoreParams {
@@ -54,31 +56,36 @@ struct ScoreParams {
     const float2* rope_table;      // [max_pos][64]
     const float2* rope_tile;       // [64][128]  (cos, sin)(t * theta_j)
     int* status;
-    int batch, H_q, n_hp, r_k, n_pad, tiles_per_seq, max_pos;
+    int batch, H_q, n_hp, r_k, n_pad, tiles_per_seq, tile_pairs, max_pos;
     int page_size, max_pages_per_seq, n_pages;
 };
 
 struct Unit {
-    int s, tile, hp, len;
+    int s, tile, hp, len;     // tile = this CTA's own 128-token tile of the pair's two
 };
 
-__device__ __forceinline__ bool decode_unit(const ScoreParams& p, int u, Unit& un) {
+// Unit `u` of the pair: (sequence, tile pair, KV-head pair).  Valid when the pair's first tile starts inside the
+// sequence; the second CTA's tile may lie past the end (its rows are then masked or not written at all).
+__device__ __forceinline__ bool decode_unit(const ScoreParams& p, int u, int rank, Unit& un) {
     un.hp = u % p.n_hp;
     int r = u / p.n_hp;
-    un.tile = r % p.tiles_per_seq;
-    un.s = r / p.tiles_per_seq;
+    const int tp = r % p.tile_pairs;
+    un.s = r / p.tile_pairs;
+    un.tile = 2 * tp + rank;
     un.len = p.seq_lens[un.s];
-    return un.len > 0 && un.len <= p.max_pos && un.tile * TILE < un.len;
+    return un.len > 0 && un.len <= p.max_pos && 2 * tp * TILE < un.len;
 }
 
 template <int G>
-__global__ void __launch_bounds__(S_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(S_THREADS, 1)
 lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_constant__ CUtensorMap mapBKT,
                   const ScoreParams p) {
     extern __shared__ uint8_t raw[];
     ScoreSmem& sm = *reinterpret_cast<ScoreSmem*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
-    const int total_units = p.batch * p.tiles_per_seq * p.n_hp;
+    const int rank = (int)cluster_ctarank();           // 0 = leader (issues the MMAs, owns the full / acc_empty barriers)
+    const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    const int total_units = p.batch * p.tile_pairs * p.n_hp;
     const int nkc = (p.r_k + KC - 1) / KC;
 
     if (tid == 0) {
@@ -88,79 +95,72 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&sm.acc_full[i], 1);
-            mbar_init(&sm.acc_empty[i], S_EPI);
+            mbar_init(&sm.acc_empty[i], 2 * S_EPI);      // the epilogue threads of both CTAs
         }
-        sm.abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&mapCK);
         prefetch_tensormap(&mapBKT);
     }
     if (warp == 1) {
-        tmem_alloc(&sm.tmem_base, 512);
-        tmem_relinquish();
+        tmem_alloc_pair(&sm.tmem_base, 512);
+        tmem_relinquish_pair();
     }
     // constant in-tile rotation table
     for (int i = tid; i < 64 * TILE; i += S_THREADS) (&sm.trigT[0][0])[i] = p.rope_tile[i];
     tc_fence_before_sync();
     __syncthreads();
+    cluster_arrive_release();                            // the peer's barriers are initialised before anyone signals them
+    cluster_wait_acquire();
     tc_fence_after_sync();
     const uint32_t tmem = sm.tmem_base;
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------------ TMA producer (both CTAs)
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+            for (int u = pair_id; u < total_units && ok; u += n_pairs) {
                 Unit un;
-                if (!decode_unit(p, u, un)) continue;
+                if (!decode_unit(p, u, rank, un)) continue;
                 for (int kc = 0; kc < nkc; ++kc, ++it) {
                     const int st = it % S_STAGES;
-                    const uint32_t ph = (it / S_STAGES) & 1;
-                    if (!mbar_wait(&sm.empty[st], ph ^ 1)) { ok = false; break; }
+                    if (!mbar_wait(&sm.empty[st], ((it / S_STAGES) & 1) ^ 1)) { ok = false; break; }
+                    // all bytes of the stage, from both CTAs, are counted on the leader's barrier
+                    const uint32_t lead_bar = mapa_shared(smem_u32(&sm.full[st]), 0);
+                    if (rank == 0) mbar_arrive_expect_tx(&sm.full[st], 2 * 2 * TILE * KC * 2);
                     if (p.page_table == nullptr) {
-                        mbar_arrive_expect_tx(&sm.full[st], (TILE + 256) * KC * 2);
-                        tma_load_3d(sm.A[st], &mapCK, &sm.full[st], kc * KC, un.tile * TILE, un.s);
+                        tma_load_3d_pair(sm.A[st], &mapCK, lead_bar, kc * KC, un.tile * TILE, un.s);
                     } else {
-                        const int ppt = TILE / p.page_size;          // pages per tile
-                        int pages[8];
-                        uint32_t bytes = 256 * KC * 2;
+                        // one box per page; pages past the end of the sequence (or with a bad table entry) are read
+                        // from page 0: those rows are masked, but every box must deliver its bytes
+                        const int ppt = TILE / p.page_size;
                         for (int pg = 0; pg < ppt; ++pg) {
-                            int lp = un.tile * ppt + pg;
-                            int page = -1;
-                            if (lp * p.page_size < un.len && lp < p.max_pages_per_seq) {
+                            const int lp = un.tile * ppt + pg;
+                            int page = 0;
+                            if ((long long)lp * p.page_size < un.len && lp < p.max_pages_per_seq) {
                                 page = p.page_table[(long long)un.s * p.max_pages_per_seq + lp];
                                 if (page < 0 || page >= p.n_pages) {
                                     lorc_set_status(p.status, LORC_ERR_CAPACITY);
-                                    page = -1;
+                                    page = 0;
                                 }
                             }
-                            pages[pg] = page;
-                            if (page >= 0) bytes += p.page_size * KC * 2;
+                            tma_load_3d_pair(sm.A[st] + pg * p.page_size * KC, &mapCK, lead_bar, kc * KC, 0, page);
                         }
-                        mbar_arrive_expect_tx(&sm.full[st], bytes);
-                        for (int pg = 0; pg < ppt; ++pg)
-                            if (pages[pg] >= 0)
-                                tma_load_3d(sm.A[st] + pg * p.page_size * KC, &mapCK, &sm.full[st], kc * KC, 0,
-                                            pages[pg]);
                     }
-                    tma_load_2d(sm.B[st], &mapBKT, &sm.full[st], kc * KC, un.hp * 256);
+                    tma_load_2d_pair(sm.B[st], &mapBKT, lead_bar, kc * KC, un.hp * 256 + rank * 128);
                 }
             }
-            if (!ok) {
-                lorc_set_status(p.status, LORC_ERR_TIMEOUT);
-                sm.abort_flag = 1;
-            }
+            if (!ok) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            const uint32_t idesc = make_idesc_bf16(128, 256, 0, 0);
+        // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = make_idesc_bf16(256, 256, 0, 0);
             uint32_t it = 0, uc = 0;
             bool ok = true;
-            for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+            for (int u = pair_id; u < total_units && ok; u += n_pairs) {
                 Unit un;
-                if (!decode_unit(p, u, un)) continue;
+                if (!decode_unit(p, u, rank, un)) continue;
                 const int buf = uc & 1;
                 if (!mbar_wait(&sm.acc_empty[buf], ((uc >> 1) & 1) ^ 1)) { ok = false; break; }
                 tc_fence_after_sync();
@@ -171,19 +171,16 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
                     const uint32_t a0 = smem_u32(sm.A[st]), b0 = smem_u32(sm.B[st]);
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
-                        tc_mma_bf16(tmem + buf * 256, make_smem_desc_sw128(a0 + k * 32, 0, 1024),
-                                    make_smem_desc_sw128(b0 + k * 32, 0, 1024), idesc, (kc | k) != 0);
+                        tc_mma_bf16_pair(tmem + buf * 256, make_smem_desc_sw128(a0 + k * 32, 0, 1024),
+                                         make_smem_desc_sw128(b0 + k * 32, 0, 1024), idesc, (kc | k) != 0);
                     }
-                    tc_commit(&sm.empty[st]);
+                    tc_commit_pair(&sm.empty[st]);        // frees the stage in both CTAs
                 }
                 if (!ok) break;
-                tc_commit(&sm.acc_full[buf]);
+                tc_commit_pair(&sm.acc_full[buf]);        // both CTAs' epilogues may read their accumulators
                 ++uc;
             }
-            if (!ok) {
-                lorc_set_status(p.status, LORC_ERR_TIMEOUT);
-                sm.abort_flag = 1;
-            }
+            if (!ok) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
         }
     } else {
         // ------------------------------------------------------------------ epilogue: RoPE + scores
@@ -194,12 +191,15 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
         const float scale = rsqrtf(128.f) * LOG2E;
         uint32_t uc = 0;
         bool ok = true;
-        for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+        const uint32_t lead_acc_empty[2] = {mapa_shared(smem_u32(&sm.acc_empty[0]), 0),
+                                            mapa_shared(smem_u32(&sm.acc_empty[1]), 0)};
+        for (int u = pair_id; u < total_units && ok; u += n_pairs) {
             Unit un;
-            if (!decode_unit(p, u, un)) continue;
+            if (!decode_unit(p, u, rank, un)) continue;
             const int buf = uc & 1, qb = uc & 1;
             const int n0 = un.tile * TILE;
-            const int delta = un.len - 1 - n0;    // query position relative to the tile start
+            // query position relative to the tile start (a tile wholly past the sequence is masked anyway)
+            const int delta = max(un.len - 1 - n0, 0);
             for (int idx = te; idx < 2 * G * 64; idx += S_EPI) {
                 const int hh = idx >> 6, j = idx & 63;
                 const int hip = hh / G, g = hh - hip * G;
@@ -243,7 +243,7 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
                 }
             }
             tc_fence_before_sync();
-            mbar_arrive(&sm.acc_empty[buf]);
+            mbar_arrive_cluster(lead_acc_empty[buf]);
             const int n = n0 + t;
 #pragma unroll
             for (int g = 0; g < G; ++g) {
@@ -253,19 +253,19 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
                 float mxv = (n < un.len) ? acc[g] : -INFINITY;
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) mxv = fmaxf(mxv, __shfl_xor_sync(0xffffffffu, mxv, o));
-                if (lane == 0)
+                if (lane == 0 && un.tile < p.tiles_per_seq)
                     p.tmax[(((long long)un.s * p.H_q + h) * p.tiles_per_seq + un.tile) * 4 + quarter] = mxv;
             }
             ++uc;
         }
-        if (!ok && lane == 0) {
-            lorc_set_status(p.status, LORC_ERR_TIMEOUT);
-            sm.abort_flag = 1;
-        }
+        if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
     }
+    // both CTAs are done with tensor memory and with each other's barriers before either lets go
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem, 512);
+    cluster_arrive_release();
+    cluster_wait_acquire();
+    if (warp == 1) tmem_dealloc_pair(tmem, 512);
 }
 
 // constant table (cos, sin)(t * theta_j) laid out [j][t], t < 128
@@ -286,7 +286,7 @@ __global__ void rope_tile_kernel(float2* out, double theta) {
 // ------------------------------------------------------------------------------------------------
 struct LorcTcLayer {
     bool has_bkt = false;
-    CUtensorMap mapBKT, mapBVT;         // B_K^T in 64 x 256 swizzled boxes; B_V^T in 64 x 128 swizzled boxes
+    CUtensorMap mapBKT, mapBVT;         // B_K^T in 64 x 128 swizzled boxes; B_V^T in 64 x 128 swizzled boxes
     // cache maps are rebuilt only when the cache geometry or pointers change
     const void* k_ptr = nullptr;
     const void* v_ptr = nullptr;
@@ -400,7 +400,7 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
     }
     if (!TL.has_bkt) {
         uint64_t dims[2] = {(uint64_t)L.r_k, (uint64_t)ctx->n}, str[1] = {(uint64_t)L.r_k * 2};
-        uint32_t box[2] = {KC, 256};
+        uint32_t box[2] = {KC, 128};
         if (!lorc_make_tmap_bf16(&TL.mapBKT, L.B_kT, 2, dims, str, box)) return cudaErrorInvalidValue;
         uint64_t d2[2] = {(uint64_t)L.r_v, (uint64_t)ctx->n}, s2[1] = {(uint64_t)L.r_v * 2};
         uint32_t b2[2] = {KC, 128};
@@ -423,10 +423,12 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
     sp.q = q; sp.scores = scores; sp.tmax = tmax; sp.seq_lens = cv.seq_lens; sp.page_table = cv.page_table;
     sp.rope_table = ctx->rope_table; sp.rope_tile = T->rope_tile; sp.status = ctx->status_dev;
     sp.batch = cv.batch; sp.H_q = d.n_q_heads; sp.n_hp = d.n_kv_heads / 2; sp.r_k = L.r_k; sp.n_pad = n_pad;
-    sp.tiles_per_seq = tiles; sp.max_pos = d.max_pos;
+    sp.tiles_per_seq = tiles; sp.tile_pairs = (tiles + 1) / 2; sp.max_pos = d.max_pos;
     sp.page_size = cv.page_size; sp.max_pages_per_seq = cv.max_pages_per_seq; sp.n_pages = cv.n_pages;
-    const int total_units = cv.batch * tiles * sp.n_hp;
-    int grid1 = total_units < ctx->sm_count ? total_units : ctx->sm_count;
+    const int total_units = cv.batch * sp.tile_pairs * sp.n_hp;          // units of a CTA pair
+    int n_pairs = ctx->sm_count / 2;
+    if (total_units < n_pairs) n_pairs = total_units;
+    const int grid1 = 2 * n_pairs;
     const size_t smem1 = sizeof(ScoreSmem) + 1024;
     {
         LorcStageTimer timer(ctx, LORC_STAGE_SCORE, st);
