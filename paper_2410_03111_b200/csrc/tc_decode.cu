@@ -41,9 +41,9 @@ constexpr int S_EPI = 256;
 struct ScoreSmem {
     bf16 A[S_STAGES][TILE * KC];          // latent slice  [128 tokens][64]       16 KiB
     bf16 B[S_STAGES][128 * KC];           // this CTA's half of the B_K^T slice [128 features][64]   16 KiB
-    float2 trigT[64][TILE];               // (cos, sin)(t * theta_j), [j][t]      64 KiB
-    float qrot[2][2][64][16];             // [buffer][head of pair][pair j][qa_0..qa_G-1, qb_0..qb_G-1]  16 KiB
-    uint64_t full[S_STAGES], empty[S_STAGES], acc_full[2], acc_empty[2];
+    float4 trig[TILE][32];                // in-tile rotation table, see rope_tile_kernel                     64 KiB
+    float qrot[2][2][1024];               // [buffer][head of pair][rotated, scaled query; see qrot_index]    16 KiB
+    uint64_t full[S_STAGES], empty[S_STAGES], acc_full[2], acc_empty[2], trig_full;
     uint32_t tmem_base;
 };
 
@@ -54,7 +54,7 @@ struct ScoreParams {
     const int32_t* seq_lens;
     const int32_t* page_table;     // NULL: contiguous
     const float2* rope_table;      // [max_pos][64]
-    const float2* rope_tile;       // [64][128]  (cos, sin)(t * theta_j)
+    const float4* rope_tile;       // [128][32]  in-tile rotation table in its shared-memory layout
     int* status;
     int batch, H_q, n_hp, r_k, n_pad, tiles_per_seq, tile_pairs, max_pos;
     int page_size, max_pages_per_seq, n_pages;
@@ -74,6 +74,19 @@ __device__ __forceinline__ bool decode_unit(const ScoreParams& p, int u, int ran
     un.tile = 2 * tp + rank;
     un.len = p.seq_lens[un.s];
     return un.len > 0 && un.len <= p.max_pos && 2 * tp * TILE < un.len;
+}
+
+// Epilogue work split.  A warp reads its 32 accumulator lanes (tokens) with 16-lane x 256-bit loads, so lane
+// (r = lane / 4, c = lane % 4) holds, per 32-column chunk jc, the tokens r + 8m (m = 0..3) and the rotary pairs
+// j = 32 jc + 8k + 2c + e (k = 0..3, e = 0..1): four tokens share every query operand the thread loads, and the four
+// lanes of equal r add their partial dots at the end.
+//
+// Float index of query head g, pair j, component `half` (0: first half of the head, 1: second) in qrot[][]: the four
+// c of equal (jc, k, e, half, g / 4) are neighbouring 16-byte pieces, one conflict-free shared-memory access.
+template <int G>
+__device__ __forceinline__ int qrot_index(int j, int half, int g) {
+    const int jc = j >> 5, k = (j >> 3) & 3, c = (j >> 1) & 3, e = j & 1;
+    return ((((((jc * 4 + k) * 2 + e) * 2 + half) * (G / 4) + (g >> 2)) * 4 + c) << 2) + (g & 3);
 }
 
 template <int G>
@@ -97,6 +110,7 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
             mbar_init(&sm.acc_full[i], 1);
             mbar_init(&sm.acc_empty[i], 2 * S_EPI);      // the epilogue threads of both CTAs
         }
+        mbar_init(&sm.trig_full, 1);
         fence_barrier_init();
         prefetch_tensormap(&mapCK);
         prefetch_tensormap(&mapBKT);
@@ -105,8 +119,6 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
         tmem_alloc_pair(&sm.tmem_base, 512);
         tmem_relinquish_pair();
     }
-    // constant in-tile rotation table
-    for (int i = tid; i < 64 * TILE; i += S_THREADS) (&sm.trigT[0][0])[i] = p.rope_tile[i];
     tc_fence_before_sync();
     __syncthreads();
     cluster_arrive_release();                            // the peer's barriers are initialised before anyone signals them
@@ -117,6 +129,10 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
         if (lane == 0) {
+            // constant in-tile rotation table, fetched while the first stages fill
+            mbar_arrive_expect_tx(&sm.trig_full, (uint32_t)sizeof(sm.trig));
+            for (int i = 0; i < 4; ++i)
+                bulk_load(&sm.trig[i * 32][0], p.rope_tile + i * 32 * 32, (uint32_t)sizeof(sm.trig) / 4, &sm.trig_full);
             uint32_t it = 0;
             bool ok = true;
             for (int u = pair_id; u < total_units && ok; u += n_pairs) {
@@ -187,76 +203,140 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
         const int te = tid - 64;                  // 0..255
         const int grp = te / 128;                 // which head of the pair
         const int quarter = warp % 4;             // TMEM lane quarter this warp may read
-        const int t = quarter * 32 + lane;        // token row inside the tile
+        const int r = lane >> 2, c = lane & 3;
         const float scale = rsqrtf(128.f) * LOG2E;
+        constexpr int QL = 2 * G * 64 / S_EPI;    // (head, pair) items of the query rotation per thread
         uint32_t uc = 0;
-        bool ok = true;
+        bool ok = mbar_wait(&sm.trig_full, 0);
         const uint32_t lead_acc_empty[2] = {mapa_shared(smem_u32(&sm.acc_empty[0]), 0),
                                             mapa_shared(smem_u32(&sm.acc_empty[1]), 0)};
-        for (int u = pair_id; u < total_units && ok; u += n_pairs) {
-            Unit un;
-            if (!decode_unit(p, u, rank, un)) continue;
+        // The query of the NEXT unit is fetched while this unit's accumulators are processed.
+        float q_a[QL], q_b[QL];
+        float2 q_cs[QL];
+        auto fetch_query = [&](const Unit& un) {
+            // query position relative to the tile start (a tile wholly past the sequence is masked anyway)
+            const int delta = max(un.len - 1 - un.tile * TILE, 0);
+#pragma unroll
+            for (int i = 0; i < QL; ++i) {
+                const int idx = te + i * S_EPI;
+                const int hh = idx >> 6, j = idx & 63;
+                const int h = un.hp * 2 * G + hh;
+                const bf16* qp = p.q + ((long long)un.s * p.H_q + h) * 128;
+                q_cs[i] = p.rope_table[(long long)delta * 64 + j];
+                q_a[i] = __bfloat162float(qp[j]);
+                q_b[i] = __bfloat162float(qp[j + 64]);
+            }
+        };
+        Unit un;
+        int u = pair_id;
+        while (u < total_units && !decode_unit(p, u, rank, un)) u += n_pairs;
+        if (u < total_units) fetch_query(un);
+        while (u < total_units && ok) {
             const int buf = uc & 1, qb = uc & 1;
             const int n0 = un.tile * TILE;
-            // query position relative to the tile start (a tile wholly past the sequence is masked anyway)
-            const int delta = max(un.len - 1 - n0, 0);
-            for (int idx = te; idx < 2 * G * 64; idx += S_EPI) {
+#pragma unroll
+            for (int i = 0; i < QL; ++i) {
+                const int idx = te + i * S_EPI;
                 const int hh = idx >> 6, j = idx & 63;
                 const int hip = hh / G, g = hh - hip * G;
-                const int h = (un.hp * 2 + hip) * G + g;
-                const float2 cs = p.rope_table[(long long)delta * 64 + j];
-                const bf16* qp = p.q + ((long long)un.s * p.H_q + h) * 128;
-                const float a = __bfloat162float(qp[j]), b = __bfloat162float(qp[j + 64]);
-                sm.qrot[qb][hip][j][g] = (a * cs.x - b * cs.y) * scale;
-                sm.qrot[qb][hip][j][G + g] = (a * cs.y + b * cs.x) * scale;
+                sm.qrot[qb][hip][qrot_index<G>(j, 0, g)] = (q_a[i] * q_cs[i].x - q_b[i] * q_cs[i].y) * scale;
+                sm.qrot[qb][hip][qrot_index<G>(j, 1, g)] = (q_a[i] * q_cs[i].y + q_b[i] * q_cs[i].x) * scale;
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");
+            // next unit of this pair
+            Unit un_next;
+            int u_next = u + n_pairs;
+            while (u_next < total_units && !decode_unit(p, u_next, rank, un_next)) u_next += n_pairs;
+            if (u_next < total_units) fetch_query(un_next);
+
             if (!mbar_wait(&sm.acc_full[buf], (uc >> 1) & 1)) { ok = false; break; }
             tc_fence_after_sync();
-            float acc[G];
+            float acc[4][G];
 #pragma unroll
-            for (int g = 0; g < G; ++g) acc[g] = 0.f;
+            for (int m = 0; m < 4; ++m)
+#pragma unroll
+                for (int g = 0; g < G; ++g) acc[m][g] = 0.f;
             const uint32_t tbase = tmem + ((uint32_t)(quarter * 32) << 16) + buf * 256 + grp * 128;
+            const float4* q4 = reinterpret_cast<const float4*>(sm.qrot[qb][grp]) + c;
+            const float4* tr4 = &sm.trig[quarter * 32 + r][0];
+            const int tswz = (r & 1) << 2;                      // odd rows of the table swap 64-byte halves
 #pragma unroll 1
             for (int jc = 0; jc < 2; ++jc) {
-                uint32_t ra[32], rb[32];
-                tmem_ld32(tbase + jc * 32, ra);
-                tmem_ld32(tbase + 64 + jc * 32, rb);
+                uint32_t ra[2][16], rb[2][16];
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    tmem_ld16x256_x4(tbase + ((uint32_t)(hf * 16) << 16) + jc * 32, ra[hf]);
+                    tmem_ld16x256_x4(tbase + ((uint32_t)(hf * 16) << 16) + 64 + jc * 32, rb[hf]);
+                }
                 tmem_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const int j = jc * 32 + i;
-                    const float2 cs = sm.trigT[j][t];
-                    const float a = __uint_as_float(ra[i]), b = __uint_as_float(rb[i]);
-                    const float ka = a * cs.x - b * cs.y;
-                    const float kb = a * cs.y + b * cs.x;
-                    const float4* qv = reinterpret_cast<const float4*>(sm.qrot[qb][grp][j]);
-                    float qa[G], qbv[G];
+                for (int k = 0; k < 4; ++k) {
+                    float4 tr[4];
 #pragma unroll
-                    for (int g4 = 0; g4 < G / 4; ++g4) {
-                        const float4 x = qv[g4], y = qv[G / 4 + g4];
-                        qa[g4 * 4 + 0] = x.x; qa[g4 * 4 + 1] = x.y; qa[g4 * 4 + 2] = x.z; qa[g4 * 4 + 3] = x.w;
-                        qbv[g4 * 4 + 0] = y.x; qbv[g4 * 4 + 1] = y.y; qbv[g4 * 4 + 2] = y.z; qbv[g4 * 4 + 3] = y.w;
+                    for (int m = 0; m < 4; ++m) tr[m] = tr4[m * 8 * 32 + ((jc * 16 + k * 4 + c) ^ tswz)];
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        float qa[G], qbv[G];
+#pragma unroll
+                        for (int g4 = 0; g4 < G / 4; ++g4) {
+                            const float4 x = q4[((((jc * 4 + k) * 2 + e) * 2 + 0) * (G / 4) + g4) * 4];
+                            const float4 y = q4[((((jc * 4 + k) * 2 + e) * 2 + 1) * (G / 4) + g4) * 4];
+                            qa[g4 * 4 + 0] = x.x; qa[g4 * 4 + 1] = x.y; qa[g4 * 4 + 2] = x.z; qa[g4 * 4 + 3] = x.w;
+                            qbv[g4 * 4 + 0] = y.x; qbv[g4 * 4 + 1] = y.y; qbv[g4 * 4 + 2] = y.z; qbv[g4 * 4 + 3] = y.w;
+                        }
+#pragma unroll
+                        for (int m = 0; m < 4; ++m) {
+                            const float a = __uint_as_float(ra[m >> 1][4 * k + 2 * (m & 1) + e]);
+                            const float b = __uint_as_float(rb[m >> 1][4 * k + 2 * (m & 1) + e]);
+                            const float cs = e ? tr[m].z : tr[m].x, sn = e ? tr[m].w : tr[m].y;
+                            const float ka = a * cs - b * sn;
+                            const float kb = a * sn + b * cs;
+#pragma unroll
+                            for (int g = 0; g < G; ++g) acc[m][g] = fmaf(qbv[g], kb, fmaf(qa[g], ka, acc[m][g]));
+                        }
                     }
-#pragma unroll
-                    for (int g = 0; g < G; ++g) acc[g] = fmaf(qbv[g], kb, fmaf(qa[g], ka, acc[g]));
                 }
             }
             tc_fence_before_sync();
             mbar_arrive_cluster(lead_acc_empty[buf]);
-            const int n = n0 + t;
+            // add the four lanes' partial dots; lane c ends with the heads g = 4i + c
+            float tot[4][G / 4];
 #pragma unroll
-            for (int g = 0; g < G; ++g) {
-                const int h = (un.hp * 2 + grp) * G + g;
-                if (n < p.n_pad) p.scores[((long long)un.s * p.H_q + h) * p.n_pad + n] = acc[g];
+            for (int m = 0; m < 4; ++m) {
+                float h1[G / 2];
+#pragma unroll
+                for (int i = 0; i < G / 2; ++i) {
+                    const float keep = (c & 1) ? acc[m][2 * i + 1] : acc[m][2 * i];
+                    const float send = (c & 1) ? acc[m][2 * i] : acc[m][2 * i + 1];
+                    h1[i] = keep + __shfl_xor_sync(0xffffffffu, send, 1);
+                }
+#pragma unroll
+                for (int i = 0; i < G / 4; ++i) {
+                    const float keep = (c & 2) ? h1[2 * i + 1] : h1[2 * i];
+                    const float send = (c & 2) ? h1[2 * i] : h1[2 * i + 1];
+                    tot[m][i] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < G / 4; ++i) {
+                const int h = (un.hp * 2 + grp) * G + 4 * i + c;
+                float* srow = p.scores + ((long long)un.s * p.H_q + h) * p.n_pad;
                 // maximum over the 32 tokens of this warp (tokens past the end of the sequence do not count)
-                float mxv = (n < un.len) ? acc[g] : -INFINITY;
+                float mxv = -INFINITY;
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) mxv = fmaxf(mxv, __shfl_xor_sync(0xffffffffu, mxv, o));
-                if (lane == 0 && un.tile < p.tiles_per_seq)
+                for (int m = 0; m < 4; ++m) {
+                    const int n = n0 + quarter * 32 + r + 8 * m;
+                    if (n < p.n_pad) srow[n] = tot[m][i];
+                    if (n < un.len) mxv = fmaxf(mxv, tot[m][i]);
+                }
+#pragma unroll
+                for (int o = 4; o < 32; o <<= 1) mxv = fmaxf(mxv, __shfl_xor_sync(0xffffffffu, mxv, o));
+                if (r == 0 && un.tile < p.tiles_per_seq)
                     p.tmax[(((long long)un.s * p.H_q + h) * p.tiles_per_seq + un.tile) * 4 + quarter] = mxv;
             }
             ++uc;
+            u = u_next;
+            un = un_next;
         }
         if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
     }
@@ -268,15 +348,17 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
     if (warp == 1) tmem_dealloc_pair(tmem, 512);
 }
 
-// constant table (cos, sin)(t * theta_j) laid out [j][t], t < 128
+// Constant in-tile rotation table (cos, sin)(t * theta_j), t < 128, j < 64, in the layout the score kernel keeps in
+// shared memory: row t holds 32 pieces of 16 bytes, piece (j / 2) ^ (4 (t & 1)) = (cos_j, sin_j, cos_j+1, sin_j+1) for
+// even j.  (The swap of 64-byte halves on odd rows spreads the epilogue's accesses over all banks.)
 __global__ void rope_tile_kernel(float2* out, double theta) {
     int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= 64 * TILE) return;
-    int j = i / TILE, t = i % TILE;
+    int t = i / 64, j = i % 64;
     double inv = pow(theta, -(double)j / 64.0);
     double sn, cs;
     sincos((double)t * inv, &sn, &cs);
-    out[i] = make_float2((float)cs, (float)sn);
+    out[(t * 32 + ((j >> 1) ^ ((t & 1) << 2))) * 2 + (j & 1)] = make_float2((float)cs, (float)sn);
 }
 
 }  // namespace
@@ -421,7 +503,7 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
 
     ScoreParams sp;
     sp.q = q; sp.scores = scores; sp.tmax = tmax; sp.seq_lens = cv.seq_lens; sp.page_table = cv.page_table;
-    sp.rope_table = ctx->rope_table; sp.rope_tile = T->rope_tile; sp.status = ctx->status_dev;
+    sp.rope_table = ctx->rope_table; sp.rope_tile = reinterpret_cast<const float4*>(T->rope_tile); sp.status = ctx->status_dev;
     sp.batch = cv.batch; sp.H_q = d.n_q_heads; sp.n_hp = d.n_kv_heads / 2; sp.r_k = L.r_k; sp.n_pad = n_pad;
     sp.tiles_per_seq = tiles; sp.tile_pairs = (tiles + 1) / 2; sp.max_pos = d.max_pos;
     sp.page_size = cv.page_size; sp.max_pages_per_seq = cv.max_pages_per_seq; sp.n_pages = cv.n_pages;
