@@ -1,18 +1,21 @@
-// Softmax + P.C_V, split by LATENT COLUMNS, and the value up-projection, both on the tensor cores.
+// Softmax, P.C_V split by LATENT COLUMNS, and the value up-projection; the two contractions run on the tensor cores.
 //
-// PV kernel.  A CTA owns one 128-column block of C_V (rho in [128 blk, 128 blk + 128)) of one sequence
-// and one share of its context.  A block of latent columns is disjoint from every other block, so the
-// CTA's accumulator O_lat^T[128 rho, H_q] (fp32 in TMEM) needs no merge with other column blocks; and
-// every CTA uses the same exact row maximum (from the quarter-tile maxima the score kernel leaves
-// behind), so the context shares of a block simply add.  Each CTA writes its 128 x H_q piece of the
-// un-normalised latent output and, for block 0, its share of the softmax denominator.
+// Probability kernel.  One CTA per (sequence, group of 128-token tiles): finds the exact row maximum of every head
+// over the whole sequence (from the quarter-tile maxima the score kernel leaves behind), turns the scores of its
+// tiles into p = 2^(s - m) rounded to bf16 -- stored tile by tile as the 128-byte-swizzled K-major image the PV
+// kernel's MMA reads, so that kernel fetches a tile with one bulk copy -- and writes its share of the softmax
+// denominator.  The probabilities are computed once, not once per column block.
 //
-//   per tile of 128 tokens:  p = 2^(s - m) (bf16, K-major in shared memory)        softmax warps
-//                            O_lat^T += C_V[tile, block]^T . P^T                    tcgen05, MN-major A
+// PV kernel.  A CTA owns one 128-column block of C_V (rho in [128 blk, 128 blk + 128)) of one sequence and one share
+// of its context.  A block of latent columns is disjoint from every other block, so the CTA's accumulator
+// O_lat^T[128 rho, H_q] (fp32 in TMEM) needs no merge with other column blocks; and every tile uses the same exact
+// row maximum, so the context shares of a block simply add.  Per tile of 128 tokens
+//       O_lat^T += C_V[tile, block]^T . P^T                    tcgen05, MN-major A
+// and at the end the CTA writes its 128 x H_q piece of the un-normalised latent output.
 //
-// Up-projection kernel.  One CTA per (KV head g, 128 output rows = 128 / G sequences): builds the
-// normalised latent rows o[(s, i), rho] = sum_shares O_lat / l in bf16, 64 columns at a time, and
-// multiplies by B_V[:, g] (TMA-staged from a transposed copy): out = o . B_V[:, g] in TMEM, then bf16.
+// Up-projection.  A small kernel adds the context shares, divides by the denominator and rounds to bf16; then one
+// CTA per (KV head g, 128 output rows = 128 / G sequences) multiplies those rows by B_V[:, g] (TMA-staged from a
+// transposed copy): out = o . B_V[:, g] in TMEM, then bf16.
 #include <math.h>
 
 #include "sm100_ptx.cuh"
@@ -24,9 +27,8 @@ namespace {
 
 constexpr int TILE = 128;
 constexpr int KC = 64;
-constexpr int P_STAGES = 2;          // 2 x 32 KiB: two CTAs fit on an SM
-constexpr int P_THREADS = 192;       // warp 0 TMA, warp 1 MMA, warps 2..5 softmax / epilogue
-constexpr int P_SOFT = 128;
+constexpr int P_STAGES = 2;          // 2 x 40 KiB: two CTAs fit on an SM
+constexpr int P_THREADS = 192;       // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
 
 // read-only global load that the compiler keeps in program order with the other volatile asm of this file
 __device__ __forceinline__ float ldg_nc_f32(const float* p) {
@@ -35,25 +37,136 @@ __device__ __forceinline__ float ldg_nc_f32(const float* p) {
     return v;
 }
 
+// ------------------------------------------------------------------------------------------------
+// probability kernel
+// ------------------------------------------------------------------------------------------------
+struct ProbParams {
+    const float* scores;           // [b, H_q, n_pad]      log2 units
+    const float* tmax;             // [b, H_q, tiles, 4]   maxima of every 32-token quarter tile
+    bf16* probs;                   // [b, tiles, 2 chunks of 64 tokens, H_q, 64]   swizzled tile images
+    float* l_part;                 // [b, n_groups, H_q]
+    int* done;                     // [b, n_blk]  arrival counters of the PV kernel's context shares, zeroed here
+    const int32_t* seq_lens;
+    int* status;
+    int H_q, n_pad, tiles, tiles_per_group, n_groups, n_blk, max_pos;
+};
+
+// byte offset of (head h, token tc < 64) inside a 64-token chunk image: rows of 128 bytes, 16-byte pieces XOR-ed with
+// the row number (the 128-byte swizzle of the shared-memory matrix descriptors)
+__device__ __forceinline__ int prob_image_offset(int h, int tc) {
+    return h * 128 + ((((tc >> 3) ^ (h & 7)) << 4) | ((tc & 7) << 1));
+}
+
+template <int HQ>
+__global__ void __launch_bounds__(128)
+lorc_prob_kernel(const ProbParams p) {
+    __shared__ float m_s[HQ];
+    __shared__ float red[4][HQ];
+    const int t = threadIdx.x, warp = t / 32, lane = t % 32;
+    const int grp = blockIdx.x, s = blockIdx.y;
+    int len = p.seq_lens[s];
+    if (len > p.max_pos || len < 0) len = 0;        // the score kernel reports the capacity error
+    const int tiles_s = (len + TILE - 1) / TILE;
+    const int tile_lo = min(tiles_s, grp * p.tiles_per_group), tile_hi = min(tiles_s, tile_lo + p.tiles_per_group);
+    if (grp == 0 && t < p.n_blk) p.done[s * p.n_blk + t] = 0;
+    float l[HQ];
+#pragma unroll
+    for (int h = 0; h < HQ; ++h) l[h] = 0.f;
+    if (tile_lo < tile_hi) {
+        // the scores of the first tile are requested before the maxima, so the two round trips overlap
+        float sv[HQ];
+        const float* sbase = p.scores + (long long)s * p.H_q * p.n_pad + t;
+        {
+            const int n = tile_lo * TILE + t;
+#pragma unroll
+            for (int h = 0; h < HQ; ++h) sv[h] = n < len ? ldg_nc_f32(sbase + (long long)h * p.n_pad + tile_lo * TILE) : 0.f;
+        }
+        // exact maximum of every head over the WHOLE sequence ([tile][4 quarters] per head: one 16-byte load per
+        // tile, eight tiles in flight per thread)
+        for (int idx = t; idx < HQ * 4; idx += 128) {          // (head, tile phase)
+            const int h = idx >> 2, ph = idx & 3;
+            const float4* tp = reinterpret_cast<const float4*>(p.tmax + ((long long)s * p.H_q + h) * (4 * p.tiles));
+            float v = -INFINITY;
+            int i = ph;
+            for (; i + 28 < tiles_s; i += 32) {
+                float4 q[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) q[u] = tp[i + 4 * u];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) v = fmaxf(v, fmaxf(fmaxf(q[u].x, q[u].y), fmaxf(q[u].z, q[u].w)));
+            }
+            for (; i < tiles_s; i += 4) {
+                const float4 q = tp[i];
+                v = fmaxf(v, fmaxf(fmaxf(q.x, q.y), fmaxf(q.z, q.w)));
+            }
+            red[ph][h] = v;
+        }
+        __syncthreads();
+        if (t < HQ) m_s[t] = fmaxf(fmaxf(red[0][t], red[1][t]), fmaxf(red[2][t], red[3][t]));
+        __syncthreads();
+        for (int tile = tile_lo; tile < tile_hi; ++tile) {
+            const bool valid = tile * TILE + t < len;
+            uint8_t* img = reinterpret_cast<uint8_t*>(p.probs) +
+                           (((long long)s * p.tiles + tile) * 2 + (t >> 6)) * (HQ * KC * 2);
+            const int tc = t & 63;
+            float ssum = 0.f;
+            bf16 pr[HQ];
+#pragma unroll
+            for (int h = 0; h < HQ; ++h) {
+                ssum += sv[h];
+                // p = 2^(s - m), rounded to bf16 (the same rounded value enters the denominator)
+                pr[h] = __float2bfloat16_rn(valid ? exp2f(sv[h] - m_s[h]) : 0.f);
+                l[h] += __bfloat162float(pr[h]);
+            }
+            // a NaN among the scores means non-finite numbers in the cache, the factors or the query
+            if (ssum != ssum) lorc_set_status(p.status, LORC_ERR_ARG);
+            if (tile + 1 < tile_hi) {
+                const int n = (tile + 1) * TILE + t;
+#pragma unroll
+                for (int h = 0; h < HQ; ++h)
+                    sv[h] = n < len ? ldg_nc_f32(sbase + (long long)h * p.n_pad + (tile + 1) * TILE) : 0.f;
+            }
+#pragma unroll
+            for (int h = 0; h < HQ; ++h) *reinterpret_cast<bf16*>(img + prob_image_offset(h, tc)) = pr[h];
+        }
+    }
+    // this group's share of the softmax denominator (zero for a group past the end of the sequence)
+    __syncthreads();
+#pragma unroll
+    for (int h = 0; h < HQ; ++h) {
+        float v = l[h];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) red[warp][h] = v;
+    }
+    __syncthreads();
+    if (t < HQ) p.l_part[((long long)s * p.n_groups + grp) * p.H_q + t] = red[0][t] + red[1][t] + red[2][t] + red[3][t];
+}
+
+// ------------------------------------------------------------------------------------------------
+// PV kernel
+// ------------------------------------------------------------------------------------------------
 template <int HQ>
 struct Pv2Smem {
     bf16 V[P_STAGES][2][TILE * KC];       // C_V block: two 64-column halves of [128 tokens][64]; 32 KiB / stage
-    bf16 P[2][2][HQ * KC];                // probabilities [HQ][128 tokens] as two 64-token chunks, 128-byte swizzle
-    float m_s[HQ];
-    float red[4][HQ];
-    uint64_t full[P_STAGES], empty[P_STAGES], p_full[2], p_empty[2], o_full;
+    bf16 P[P_STAGES][2][HQ * KC];         // probabilities [HQ][128 tokens] as two 64-token chunks, 128-byte swizzle
+    float red[128 / HQ][HQ];
+    float l_inv[HQ];
+    uint64_t full[P_STAGES], empty[P_STAGES], o_full;
     uint32_t tmem_base;
+    int last;
 };
 
 struct Pv2Params {
-    const float* scores;           // [b, H_q, n_pad]      log2 units
-    const float* tmax;             // [b, H_q, tiles, 4]   maxima of every 32-token quarter tile
+    const bf16* probs;             // [b, tiles, 2, H_q, 64]   swizzled tile images
     float* o_part;                 // [b, n_csplit, H_q, r_pad]   un-normalised latent output, r_pad = 128 n_blk
-    float* l_part;                 // [b, n_csplit, H_q]
+    const float* l_part;           // [b, n_groups, H_q]   shares of the softmax denominator
+    bf16* o_norm;                  // [b, H_q, r_pad]      normalised latent output
+    int* done;                     // [b, n_blk]           context shares of a column block that have finished
     const int32_t* seq_lens;
     const int32_t* page_table;
     int* status;
-    int batch, H_q, n_kv, r_v, n_pad, tiles, n_blk, n_csplit, max_pos;
+    int batch, H_q, n_kv, r_v, tiles, n_blk, n_csplit, n_groups, max_pos;
     int page_size, max_pages_per_seq, n_pages;
 };
 
@@ -64,6 +177,7 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
     typedef Pv2Smem<HQ> S;
     S& sm = *reinterpret_cast<S*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
     constexpr uint32_t TM_COLS = HQ <= 32 ? 32 : 64;
+    constexpr uint32_t P_BYTES = 2 * HQ * KC * 2;
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
     const int blk = blockIdx.x, cs = blockIdx.y, s = blockIdx.z;
 
@@ -78,17 +192,12 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
     const int per = (tiles_s + p.n_csplit - 1) / p.n_csplit;
     const int tile_lo = min(tiles_s, cs * per), tile_hi = min(tiles_s, tile_lo + per);
     const int ntiles = tile_hi - tile_lo;
-    const int t_begin = tile_lo * TILE, t_end = min(len, tile_hi * TILE);
     const int rho0 = blk * 128;
 
     if (tid == 0) {
         for (int i = 0; i < P_STAGES; ++i) {
             mbar_init(&sm.full[i], 1);
             mbar_init(&sm.empty[i], 1);
-        }
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(&sm.p_full[i], P_SOFT);
-            mbar_init(&sm.p_empty[i], 1);
         }
         mbar_init(&sm.o_full, 1);
         fence_barrier_init();
@@ -108,10 +217,12 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             for (int i = 0; i < ntiles && ok; ++i) {
-                const int n0 = t_begin + i * TILE;
+                const int tile = tile_lo + i;
+                const int n0 = tile * TILE;
                 const int st = i % P_STAGES;
                 if (!mbar_wait(&sm.empty[st], ((i / P_STAGES) & 1) ^ 1)) { ok = false; break; }
-                mbar_arrive_expect_tx(&sm.full[st], 2 * TILE * KC * 2);
+                mbar_arrive_expect_tx(&sm.full[st], 2 * TILE * KC * 2 + P_BYTES);
+                bulk_load(sm.P[st][0], p.probs + ((long long)s * p.tiles + tile) * (2 * HQ * KC), P_BYTES, &sm.full[st]);
                 if (p.page_table == nullptr) {
                     tma_load_3d(sm.V[st][0], &mapCV, &sm.full[st], rho0, n0, s);
                     tma_load_3d(sm.V[st][1], &mapCV, &sm.full[st], rho0 + 64, n0, s);
@@ -142,11 +253,10 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
         if (lane == 0 && ntiles > 0) {
             const uint32_t idesc = make_idesc_bf16(128, HQ, 1, 0);
             for (int i = 0; i < ntiles && ok; ++i) {
-                const int buf = i & 1, st = i % P_STAGES;
-                if (!mbar_wait(&sm.p_full[buf], (i >> 1) & 1)) { ok = false; break; }
+                const int st = i % P_STAGES;
                 if (!mbar_wait(&sm.full[st], (i / P_STAGES) & 1)) { ok = false; break; }
                 tc_fence_after_sync();
-                const uint32_t p0 = smem_u32(sm.P[buf][0]), v0 = smem_u32(sm.V[st][0]);
+                const uint32_t p0 = smem_u32(sm.P[st][0]), v0 = smem_u32(sm.V[st][0]);
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
                     // A: C_V^T block (MN-major): 16 token rows per step, the two 64-column halves 16 KiB apart
@@ -156,117 +266,80 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
                     tc_mma_bf16(tmem, ad, bd, idesc, (i | k) != 0);
                 }
                 tc_commit(&sm.empty[st]);
-                tc_commit(&sm.p_empty[buf]);
             }
             tc_commit(&sm.o_full);
             if (!ok) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
         }
     } else {
-        // ------------------------------------------------------------------ softmax, then up-projection
-        const int t = tid - 64;                   // token inside the tile; later output column j
-        const int wq = warp - 2;
-        float l[HQ];
-#pragma unroll
-        for (int h = 0; h < HQ; ++h) l[h] = 0.f;
-        // exact maximum of every head over the WHOLE sequence, from the quarter-tile maxima the score kernel wrote
-        // ([tile][4 quarters] per head: one 16-byte load per tile, eight tiles in flight per thread)
-        for (int idx = t; idx < HQ * 4; idx += P_SOFT) {          // (head, tile phase)
-            const int h = idx >> 2, ph = idx & 3;
-            const float4* tp = reinterpret_cast<const float4*>(p.tmax + ((long long)s * p.H_q + h) * (4 * p.tiles));
-            float v = -INFINITY;
-            int i = ph;
-            for (; i + 28 < tiles_s; i += 32) {
-                float4 q[8];
-#pragma unroll
-                for (int u = 0; u < 8; ++u) q[u] = tp[i + 4 * u];
-#pragma unroll
-                for (int u = 0; u < 8; ++u) v = fmaxf(v, fmaxf(fmaxf(q[u].x, q[u].y), fmaxf(q[u].z, q[u].w)));
-            }
-            for (; i < tiles_s; i += 4) {
-                const float4 q = tp[i];
-                v = fmaxf(v, fmaxf(fmaxf(q.x, q.y), fmaxf(q.z, q.w)));
-            }
-            sm.red[ph][h] = v;
-        }
-        asm volatile("bar.sync 2, 128;" ::: "memory");
-        if (t < HQ) sm.m_s[t] = fmaxf(fmaxf(sm.red[0][t], sm.red[1][t]), fmaxf(sm.red[2][t], sm.red[3][t]));
-        asm volatile("bar.sync 2, 128;" ::: "memory");
-
-        // Scores of a tile are loaded one tile ahead, all heads at once.  The loads and the shared-memory stores are
-        // volatile asm, which keeps them in program order: loads of tile i + 1, then stores of tile i.
-        float sv[HQ];
+        // ------------------------------------------------------------------ epilogue
+        const int t = tid - 64;
+        const int quarter = warp % 4;
+        const int row = quarter * 32 + lane;              // TMEM lane = latent row of the block
+        const int r_pad = p.n_blk * 128;
+        // while the tiles stream: the reciprocal softmax denominator of every head (all shares of the sequence)
         {
-            const int n = t_begin + t;
-            const float* sp = p.scores + (long long)s * p.H_q * p.n_pad + n;
+            constexpr int PARTS = 128 / HQ;
+            const int h = t % HQ, part = t / HQ;
+            const float* lp = p.l_part + (long long)s * p.n_groups * p.H_q + h;
+            float L = 0.f;
+            for (int g = part; g < p.n_groups; g += PARTS) L += __ldg(lp + (long long)g * p.H_q);
+            sm.red[part][h] = L;
+            asm volatile("bar.sync 2, 128;" ::: "memory");
+            if (t < HQ) {
+                float Ls = 0.f;
 #pragma unroll
-            for (int h = 0; h < HQ; ++h) sv[h] = (ntiles > 0 && n < t_end) ? ldg_nc_f32(sp + (long long)h * p.n_pad) : 0.f;
-        }
-        for (int i = 0; i < ntiles; ++i) {
-            const int buf = i & 1;
-            if (!mbar_wait(&sm.p_empty[buf], ((i >> 1) & 1) ^ 1)) { ok = false; break; }
-            const bool valid = t_begin + i * TILE + t < t_end;
-            // p = 2^(s - m), rounded to bf16 (the same rounded value enters the denominator)
-            bf16 pr[HQ];
-            float ssum = 0.f;
-#pragma unroll
-            for (int h = 0; h < HQ; ++h) {
-                ssum += sv[h];
-                pr[h] = __float2bfloat16_rn(valid ? exp2f(sv[h] - sm.m_s[h]) : 0.f);
-                l[h] += __bfloat162float(pr[h]);
+                for (int i = 0; i < PARTS; ++i) Ls += sm.red[i][t];
+                sm.l_inv[t] = Ls > 0.f ? 1.f / Ls : 0.f;
+                if (!(Ls > 0.f) && blk == 0 && cs == 0) lorc_set_status(p.status, LORC_ERR_EMPTY);
             }
-            // a NaN among the scores means non-finite numbers in the cache, the factors or the query
-            if (ssum != ssum) lorc_set_status(p.status, LORC_ERR_ARG);
-            {
-                const int nn = t_begin + (i + 1) * TILE + t;
-                const float* sp = p.scores + (long long)s * p.H_q * p.n_pad + nn;
-#pragma unroll
-                for (int h = 0; h < HQ; ++h) sv[h] = (i + 1 < ntiles && nn < t_end) ? ldg_nc_f32(sp + (long long)h * p.n_pad) : 0.f;
-            }
-            const uint32_t pb = smem_u32(sm.P[buf][t >> 6]);
-            const int tc = t & 63;
-#pragma unroll
-            for (int h = 0; h < HQ; ++h) {
-                const int off = h * 128 + ((((tc >> 3) ^ (h & 7)) << 4) | ((tc & 7) << 1));
-                asm volatile("st.shared.b16 [%0], %1;" ::"r"(pb + off), "h"(__bfloat16_as_ushort(pr[h])));
-            }
-            fence_proxy_async_smem();
-            mbar_arrive(&sm.p_full[buf]);
         }
-        // softmax denominator of this context share (written once per share, by the CTA of block 0)
-#pragma unroll
-        for (int h = 0; h < HQ; ++h) {
-            float v = l[h];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-            if (lane == 0) sm.red[wq][h] = v;
-        }
-        asm volatile("bar.sync 2, 128;" ::: "memory");
-        if (blk == 0 && t < HQ)
-            p.l_part[((long long)s * p.n_csplit + cs) * p.H_q + t] =
-                (ntiles > 0 && ok) ? sm.red[0][t] + sm.red[1][t] + sm.red[2][t] + sm.red[3][t] : 0.f;
-
-        // this CTA's piece of the un-normalised latent output: TMEM lane = latent row of the block
-        if (ntiles > 0 && ok) {
+        if (ntiles > 0) {
             if (!mbar_wait(&sm.o_full, 0)) ok = false;
         }
-        {
-            const int quarter = warp % 4;
-            const int r_pad = p.n_blk * 128;
-            float* op = p.o_part + (((long long)s * p.n_csplit + cs) * p.H_q) * r_pad + rho0 + quarter * 32 + lane;
-            if (ntiles > 0 && ok) tc_fence_after_sync();
+        float acc[HQ];
+        if (ntiles > 0 && ok) {
+            tc_fence_after_sync();
 #pragma unroll
             for (int c0 = 0; c0 < HQ; c0 += 32) {
                 uint32_t r[32];
-                if (ntiles > 0 && ok) {
-                    tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + c0, r);
-                    tmem_wait_ld();
-                } else {
+                tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + c0, r);
+                tmem_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) r[i] = 0u;
-                }
-#pragma unroll
-                for (int i = 0; i < 32; ++i) op[(long long)(c0 + i) * r_pad] = __uint_as_float(r[i]);
+                for (int i = 0; i < 32; ++i) acc[c0 + i] = __uint_as_float(r[i]);
             }
+        } else {
+#pragma unroll
+            for (int h = 0; h < HQ; ++h) acc[h] = 0.f;
+        }
+        bool finish = true;
+        if (p.n_csplit > 1) {
+            // publish this share; the share that arrives last adds them all up (in share order, so the result does
+            // not depend on which one that is)
+            float* op = p.o_part + (((long long)s * p.n_csplit + cs) * p.H_q) * r_pad + rho0 + row;
+#pragma unroll
+            for (int h = 0; h < HQ; ++h) op[(long long)h * r_pad] = acc[h];
+            __threadfence();
+            asm volatile("bar.sync 2, 128;" ::: "memory");
+            if (t == 0) sm.last = atomicAdd(p.done + s * p.n_blk + blk, 1) == p.n_csplit - 1;
+            asm volatile("bar.sync 2, 128;" ::: "memory");
+            finish = sm.last != 0;
+            if (finish) {
+                __threadfence();
+                const float* ip = p.o_part + ((long long)s * p.n_csplit * p.H_q) * r_pad + rho0 + row;
+#pragma unroll
+                for (int h = 0; h < HQ; ++h) acc[h] = 0.f;
+                for (int c = 0; c < p.n_csplit; ++c) {
+#pragma unroll
+                    for (int h = 0; h < HQ; ++h) acc[h] += __ldcg(ip + ((long long)c * p.H_q + h) * r_pad);
+                }
+            }
+        } else {
+            asm volatile("bar.sync 2, 128;" ::: "memory");     // l_inv is complete
+        }
+        if (finish) {
+            bf16* on = p.o_norm + (long long)s * p.H_q * r_pad + rho0 + row;
+#pragma unroll
+            for (int h = 0; h < HQ; ++h) on[(long long)h * r_pad] = __float2bfloat16_rn(acc[h] * sm.l_inv[h]);
         }
         if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
     }
@@ -278,52 +351,6 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
 }  // namespace
 
 namespace {
-
-// ------------------------------------------------------------------------------------------------
-// normalise: o_norm[s, h, rho] = bf16( sum_shares O_lat[s, share, h, rho] / sum_shares l[s, share, h] )
-// one thread per 4 latent columns
-// ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
-lorc_normalize_kernel(const float* __restrict__ o_part, const float* __restrict__ l_part, bf16* __restrict__ o_norm,
-                      int H_q, int r_pad, int n_csplit, long long total4, int* status) {
-    const long long i4 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i4 >= total4) return;
-    const int r4n = r_pad >> 2;
-    const long long row = i4 / r4n;                   // s * H_q + h
-    const int r4 = (int)(i4 - row * r4n);
-    const int s = (int)(row / H_q), h = (int)(row - (long long)s * H_q);
-    const long long share_stride4 = (long long)H_q * r4n;
-    const float4* src = reinterpret_cast<const float4*>(o_part) + ((long long)s * n_csplit * H_q + h) * r4n + r4;
-    const float* lp = l_part + (long long)s * n_csplit * H_q + h;
-    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-    float L = 0.f;
-    int c = 0;
-    for (; c + 4 <= n_csplit; c += 4) {
-        float4 v[4];
-        float l[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            v[u] = __ldg(src + (c + u) * share_stride4);
-            l[u] = __ldg(lp + (long long)(c + u) * H_q);
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            a.x += v[u].x; a.y += v[u].y; a.z += v[u].z; a.w += v[u].w;
-            L += l[u];
-        }
-    }
-    for (; c < n_csplit; ++c) {
-        const float4 v = __ldg(src + c * share_stride4);
-        a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
-        L += __ldg(lp + (long long)c * H_q);
-    }
-    float inv = 0.f;
-    if (L > 0.f) inv = 1.f / L;
-    else if (r4 == 0) lorc_set_status(status, LORC_ERR_EMPTY);
-    __nv_bfloat162 b0 = __floats2bfloat162_rn(a.x * inv, a.y * inv), b1 = __floats2bfloat162_rn(a.z * inv, a.w * inv);
-    uint2 w = make_uint2(*reinterpret_cast<uint32_t*>(&b0), *reinterpret_cast<uint32_t*>(&b1));
-    reinterpret_cast<uint2*>(o_norm)[i4] = w;
-}
 
 // ------------------------------------------------------------------------------------------------
 // value up-projection: out[(s, h), :] = o_norm[s, h, :] . B_V[:, g(h)], a plain TMA-fed tcgen05 GEMM.
@@ -452,6 +479,30 @@ void pv_plan(const lorc_ctx* ctx, const LorcLayer& L, int batch, int max_seq_len
     *n_csplit = cs;
 }
 
+// Tiles per CTA of the probability kernel: about four CTAs per SM over the whole batch (every CTA first reduces the
+// row maxima of its sequence, so very many tiny CTAs would repeat that too often).
+void prob_plan(const lorc_ctx* ctx, int batch, int tiles, int* tiles_per_group, int* n_groups) {
+    int tpg = (int)(((long long)tiles * batch + 4LL * ctx->sm_count - 1) / (4LL * ctx->sm_count));
+    if (tpg < 1) tpg = 1;
+    *tiles_per_group = tpg;
+    *n_groups = (tiles + tpg - 1) / tpg;
+}
+
+struct PvScratch {
+    size_t part_bytes, l_bytes, on_bytes, prob_bytes, done_bytes;
+};
+
+PvScratch pv_scratch_layout(const lorc_ctx* ctx, int batch, int tiles, int n_csplit, int n_groups, size_t r_pad) {
+    PvScratch z;
+    const size_t hq = (size_t)ctx->desc.n_q_heads;
+    z.part_bytes = lorc_align_up((size_t)batch * n_csplit * hq * r_pad * sizeof(float), 256);
+    z.l_bytes = lorc_align_up((size_t)batch * n_groups * hq * sizeof(float), 256);
+    z.on_bytes = lorc_align_up((size_t)batch * hq * r_pad * sizeof(bf16), 256);
+    z.prob_bytes = lorc_align_up((size_t)batch * tiles * hq * TILE * sizeof(bf16), 256);
+    z.done_bytes = lorc_align_up((size_t)batch * (r_pad / 128) * sizeof(int), 256);
+    return z;
+}
+
 }  // namespace
 
 // ------------------------------------------------------------------------------------------------
@@ -464,10 +515,11 @@ size_t lorc_tc_pv_scratch_bytes(const lorc_ctx* ctx, int batch, int max_seq_len)
     if (cs > tiles) cs = tiles;
     if (cs > 64) cs = 64;
     if (cs < 1) cs = 1;
+    int tpg, n_groups;
+    prob_plan(ctx, batch, tiles, &tpg, &n_groups);
     const size_t r_pad = (size_t)((ctx->n + 127) / 128) * 128;
-    return lorc_align_up((size_t)batch * cs * ctx->desc.n_q_heads * r_pad * sizeof(float), 256) +
-           lorc_align_up((size_t)batch * cs * ctx->desc.n_q_heads * sizeof(float), 256) +
-           lorc_align_up((size_t)batch * ctx->desc.n_q_heads * r_pad * sizeof(bf16), 256);
+    const PvScratch z = pv_scratch_layout(ctx, batch, tiles, cs, n_groups, r_pad);
+    return z.part_bytes + z.l_bytes + z.on_bytes + z.prob_bytes + z.done_bytes;
 }
 
 cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, const CUtensorMap& mapCV,
@@ -488,44 +540,53 @@ cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView
         if (e != cudaSuccess) return e;
         attr = true;
     }
-    int n_blk, n_csplit;
+    int n_blk, n_csplit, tpg, n_groups;
     pv_plan(ctx, L, cv.batch, cv.max_seq_len, n_splits_hint, &n_blk, &n_csplit);
+    prob_plan(ctx, cv.batch, tiles, &tpg, &n_groups);
     const int r_pad = n_blk * 128;
-    size_t part_bytes, l_bytes;
-    const size_t on_bytes = lorc_align_up((size_t)cv.batch * d.n_q_heads * r_pad * sizeof(bf16), 256);
+    PvScratch z;
     for (;; --n_csplit) {
-        part_bytes = lorc_align_up((size_t)cv.batch * n_csplit * d.n_q_heads * r_pad * sizeof(float), 256);
-        l_bytes = lorc_align_up((size_t)cv.batch * n_csplit * d.n_q_heads * sizeof(float), 256);
-        if (part_bytes + l_bytes + on_bytes <= scratch_bytes) break;
+        z = pv_scratch_layout(ctx, cv.batch, tiles, n_csplit, n_groups, (size_t)r_pad);
+        if (z.part_bytes + z.l_bytes + z.on_bytes + z.prob_bytes + z.done_bytes <= scratch_bytes) break;
         if (n_csplit == 1) return cudaErrorMemoryAllocation;
     }
-    bf16* o_norm = (bf16*)((char*)scratch + part_bytes + l_bytes);
-    Pv2Params p;
-    p.scores = scores; p.tmax = tmax;
-    p.o_part = (float*)scratch;
-    p.l_part = (float*)((char*)scratch + part_bytes);
-    p.seq_lens = cv.seq_lens; p.page_table = cv.page_table; p.status = ctx->status_dev;
-    p.batch = cv.batch; p.H_q = d.n_q_heads; p.n_kv = d.n_kv_heads; p.r_v = L.r_v; p.n_pad = n_pad; p.tiles = tiles;
-    p.n_blk = n_blk; p.n_csplit = n_csplit; p.max_pos = d.max_pos;
-    p.page_size = cv.page_size; p.max_pages_per_seq = cv.max_pages_per_seq; p.n_pages = cv.n_pages;
-    dim3 grid(n_blk, n_csplit, cv.batch);
+    float* o_part = (float*)scratch;
+    float* l_part = (float*)((char*)scratch + z.part_bytes);
+    bf16* o_norm = (bf16*)((char*)scratch + z.part_bytes + z.l_bytes);
+    bf16* probs = (bf16*)((char*)scratch + z.part_bytes + z.l_bytes + z.on_bytes);
+    int* done = (int*)((char*)scratch + z.part_bytes + z.l_bytes + z.on_bytes + z.prob_bytes);
+    cudaError_t e;
     {
         LorcStageTimer timer(ctx, LORC_STAGE_PV, st);
+        ProbParams q;
+        q.scores = scores; q.tmax = tmax; q.probs = probs; q.l_part = l_part; q.done = done; q.seq_lens = cv.seq_lens;
+        q.status = ctx->status_dev; q.H_q = d.n_q_heads; q.n_pad = n_pad; q.tiles = tiles; q.tiles_per_group = tpg;
+        q.n_groups = n_groups; q.n_blk = n_blk; q.max_pos = d.max_pos;
+        dim3 pgrid(n_groups, cv.batch);
+        if (d.n_q_heads == 32)
+            lorc_prob_kernel<32><<<pgrid, 128, 0, st>>>(q);
+        else
+            lorc_prob_kernel<64><<<pgrid, 128, 0, st>>>(q);
+        *launches += 1;
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+
+        Pv2Params p;
+        p.probs = probs; p.o_part = o_part; p.l_part = l_part; p.o_norm = o_norm; p.done = done;
+        p.seq_lens = cv.seq_lens; p.page_table = cv.page_table; p.status = ctx->status_dev;
+        p.batch = cv.batch; p.H_q = d.n_q_heads; p.n_kv = d.n_kv_heads; p.r_v = L.r_v; p.tiles = tiles;
+        p.n_blk = n_blk; p.n_csplit = n_csplit; p.n_groups = n_groups; p.max_pos = d.max_pos;
+        p.page_size = cv.page_size; p.max_pages_per_seq = cv.max_pages_per_seq; p.n_pages = cv.n_pages;
+        dim3 grid(n_blk, n_csplit, cv.batch);
         if (d.n_q_heads == 32)
             lorc_pv2_kernel<32><<<grid, P_THREADS, sizeof(Pv2Smem<32>) + 1024, st>>>(mapCV, p);
         else
             lorc_pv2_kernel<64><<<grid, P_THREADS, sizeof(Pv2Smem<64>) + 1024, st>>>(mapCV, p);
+        *launches += 1;
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
     }
-    *launches += 1;
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
     LorcStageTimer timer(ctx, LORC_STAGE_COMBINE, st);
-    const long long total4 = (long long)cv.batch * d.n_q_heads * (r_pad / 4);
-    lorc_normalize_kernel<<<(unsigned)((total4 + 255) / 256), 256, 0, st>>>(p.o_part, p.l_part, o_norm, d.n_q_heads, r_pad,
-                                                                        n_csplit, total4, ctx->status_dev);
-    *launches += 1;
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
     // o_norm [b, H_q, r_pad] as (rho, head, sequence) with boxes of 64 rho x G heads x 128/G sequences
     CUtensorMap mapON;
     {
