@@ -225,6 +225,12 @@ int lorc_last_path(const lorc_ctx* ctx);
  * Without the flag it returns zeros. */
 int lorc_profile_read(lorc_ctx* ctx, float* ms, int64_t* launches);
 
+/* Switches the event bracketing of LORC_FLAG_PROFILE on (on != 0) or off for the calls that
+ * follow, on any context; while it is off the launches carry no events and may be captured
+ * into a CUDA graph.  Events still pending are kept for the next lorc_profile_read.
+ * Returns LORC_ERR_ARG for a NULL context, LORC_ERR_CUDA when the bookkeeping cannot be set up. */
+int lorc_profile_enable(lorc_ctx* ctx, int on);
+
 /* Number of kernel launches the library has enqueued on this context so far. */
 int64_t lorc_launch_count(const lorc_ctx* ctx);
 

@@ -73,6 +73,7 @@ def _signatures():
         "lorc_last_error": ([vp], C.c_char_p),
         "lorc_last_path": ([vp], i32),
         "lorc_profile_read": ([vp, C.POINTER(C.c_float), C.POINTER(i64)], i32),
+        "lorc_profile_enable": ([vp, i32], i32),
         "lorc_launch_count": ([vp], i64),
     }
 
@@ -198,6 +199,11 @@ def lorc_profile_read(ctx):
     cnt = (C.c_int64 * LORC_N_STAGES)()
     _check(ctx, _lib.lorc_profile_read(ctx, ms, cnt))
     return {name: (float(ms[i]), int(cnt[i])) for i, name in enumerate(LORC_STAGE_NAMES)}
+
+
+def lorc_profile_enable(ctx, on):
+    """Turn the per-stage event bracketing on or off for the calls that follow."""
+    _check(ctx, _lib.lorc_profile_enable(ctx, 1 if on else 0))
 
 
 def lorc_launch_count(ctx):

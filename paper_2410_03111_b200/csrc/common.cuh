@@ -60,7 +60,8 @@ struct lorc_ctx {
     int last_path = 0;
     int64_t launches = 0;
     LorcTcState* tc = nullptr;
-    LorcProfile* prof = nullptr;   // non-null iff LORC_FLAG_PROFILE
+    LorcProfile* prof = nullptr;   // event bookkeeping, created on first use
+    bool prof_on = false;          // LORC_FLAG_PROFILE or lorc_profile_enable
 };
 
 // RAII bracket: records an event pair around the launches issued in its scope (no-op unless profiling).
@@ -68,7 +69,8 @@ struct LorcStageTimer {
     LorcProfile* p;
     LorcProfile::Rec rec;
     cudaStream_t st;
-    LorcStageTimer(const lorc_ctx* ctx, int stage, cudaStream_t stream) : p(ctx->prof), st(stream) {
+    LorcStageTimer(const lorc_ctx* ctx, int stage, cudaStream_t stream)
+        : p(ctx->prof_on ? ctx->prof : nullptr), st(stream) {
         if (!p) return;
         rec.stage = stage;
         rec.e0 = p->get();

@@ -130,7 +130,10 @@ int lorc_create(const lorc_model_desc* desc, lorc_ctx** out) {
     ctx->n = desc->n_kv_heads * desc->d_head;
     ctx->group = desc->n_q_heads / desc->n_kv_heads;
     ctx->layers.resize(desc->n_layers);
-    if (desc->flags & LORC_FLAG_PROFILE) ctx->prof = new (std::nothrow) LorcProfile();
+    if (desc->flags & LORC_FLAG_PROFILE) {
+        ctx->prof = new (std::nothrow) LorcProfile();
+        ctx->prof_on = ctx->prof != nullptr;
+    }
     cudaError_t e = cudaGetDevice(&ctx->device);
     if (e == cudaSuccess)
         e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device);
@@ -399,6 +402,16 @@ int lorc_profile_read(lorc_ctx* ctx, float* ms, int64_t* launches) {
         if (ms) ms[i] = acc[i];
         if (launches) launches[i] = cnt[i];
     }
+    return LORC_OK;
+}
+
+int lorc_profile_enable(lorc_ctx* ctx, int on) {
+    if (!ctx) return LORC_ERR_ARG;
+    if (on && !ctx->prof) {
+        ctx->prof = new (std::nothrow) LorcProfile();
+        if (!ctx->prof) return fail(ctx, LORC_ERR_CUDA, "lorc_profile_enable: out of host memory");
+    }
+    ctx->prof_on = on != 0;
     return LORC_OK;
 }
 
