@@ -47,8 +47,10 @@ def parse_args():
 
 
 # DRAM traffic of one lorc_score_kernel launch, from the ncu capture summarised in
-# profiles/lorc_score_kernel_cfg2_layer0.md (None once the kernel has changed since that capture).
-SCORE_KERNEL_TRAFFIC = None
+# profiles/attention_kernels_cfg2_layers0-1.md (set to None once the kernel has changed since that capture).  The
+# capture is of the layer with rank 928; the read traffic is the latent keys, which grow with rank, batch and
+# context, the written traffic the scores, which grow with batch and context only.
+SCORE_KERNEL_TRAFFIC = {"read_bytes": 127.73e6, "write_bytes": 10.85e6, "rank": 928, "batch": 16, "context": 4100}
 
 
 def load_peaks():
