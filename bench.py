@@ -40,6 +40,8 @@ def parse_args():
     ap.add_argument("--debug-fp32", action="store_true", help="time the plain fp32 kernels")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--ref-budget", type=float, default=6.0,
+                    help="--impl reference: seconds of oracle time sampled per step")
     ap.add_argument("--no-graph", action="store_true", help="launch call by call instead of replaying a CUDA graph")
     ap.add_argument("--stages", action="store_true",
                     help="call-by-call launches with per-kernel CUDA events; adds a 'stages' object (ms per step)")
@@ -296,7 +298,7 @@ def run_reference(args, shape, n_layers):
     vals = []
     per_rank, desc, threads = None, "", 1
     for i in range(args.warmup + args.steps):
-        per_rank, desc, threads, units = oracle_sample(shape, n_layers, budget_s=6.0,
+        per_rank, desc, threads, units = oracle_sample(shape, n_layers, budget_s=args.ref_budget,
                                                        layers=[0, n_layers - 1] if n_layers > 1 else [0])
         step_s = per_rank * sum(shape.ranks[:n_layers]) * shape.batch
         if i >= args.warmup:
@@ -313,6 +315,21 @@ def run_reference(args, shape, n_layers):
         "gpu_launches": 0,
     }
     print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- ranks
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of timings over all ranks (the slowest replica sets the job's time)."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
+
+
+def whole_job_rate(batch, steps, world, seconds):
+    """Tokens per second of the whole job: every rank decodes `batch` sequences per step (weak scaling)."""
+    return batch * steps * world / seconds
 
 
 # --------------------------------------------------------------------------- main
@@ -447,15 +464,10 @@ def main():
         d2h = n_layers * oh[0].numel() * 2
         e2e = (e2e_s, h2d, d2h)
 
-    # max over ranks
-    t = torch.tensor([ms, attn_ms, e2e[0] if e2e else 0.0], dtype=torch.float64, device=device)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms, attn_ms, e2e_s = (float(v) for v in t.tolist())
+    ms, attn_ms, e2e_s = max_over_ranks([ms, attn_ms, e2e[0] if e2e else 0.0], dist, device)
 
     if rank == 0:
-        tokens = b * args.steps * world
-        value = tokens / (ms * 1e-3)
+        value = whole_job_rate(b, args.steps, world, ms * 1e-3)
         n_ctx_mid = n_ctx_start + args.steps      # context the attention-only pass sees
         flops, byts = algorithmic_counts(shape, wl.ranks, b, n_ctx_mid)
         attn_ms_step = attn_ms / args.steps
