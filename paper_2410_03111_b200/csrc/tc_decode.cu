@@ -34,14 +34,14 @@ constexpr float LOG2E = 1.4426950408889634f;
 // ------------------------------------------------------------------------------------------------
 // score kernel
 // ------------------------------------------------------------------------------------------------
-constexpr int S_STAGES = 4;
+constexpr int S_STAGES = 6;
 constexpr int S_THREADS = 320;       // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
 constexpr int S_EPI = 256;
 
 struct ScoreSmem {
     bf16 A[S_STAGES][TILE * KC];          // latent slice  [128 tokens][64]       16 KiB
     bf16 B[S_STAGES][128 * KC];           // this CTA's half of the B_K^T slice [128 features][64]   16 KiB
-    float4 trig[TILE][32];                // in-tile rotation table, see rope_tile_kernel                     64 KiB
+    float4 trig[33][32];                  // in-tile rotation table, see rope_tile_kernel                     16.5 KiB
     float qrot[2][2][1024];               // [buffer][head of pair][rotated, scaled query; see qrot_index]    16 KiB
     uint64_t full[S_STAGES], empty[S_STAGES], acc_full[2], acc_empty[2], trig_full;
     uint32_t tmem_base;
@@ -54,7 +54,7 @@ struct ScoreParams {
     const int32_t* seq_lens;
     const int32_t* page_table;     // NULL: contiguous
     const float2* rope_table;      // [max_pos][64]
-    const float4* rope_tile;       // [128][32]  in-tile rotation table in its shared-memory layout
+    const float4* rope_tile;       // [33][32]   in-tile rotation table in its shared-memory layout
     int* status;
     int batch, H_q, n_hp, r_k, n_pad, tiles_per_seq, tile_pairs, max_pos;
     int page_size, max_pages_per_seq, n_pages;
@@ -131,8 +131,7 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
         if (lane == 0) {
             // constant in-tile rotation table, fetched while the first stages fill
             mbar_arrive_expect_tx(&sm.trig_full, (uint32_t)sizeof(sm.trig));
-            for (int i = 0; i < 4; ++i)
-                bulk_load(&sm.trig[i * 32][0], p.rope_tile + i * 32 * 32, (uint32_t)sizeof(sm.trig) / 4, &sm.trig_full);
+            bulk_load(&sm.trig[0][0], p.rope_tile, (uint32_t)sizeof(sm.trig), &sm.trig_full);
             uint32_t it = 0;
             bool ok = true;
             for (int u = pair_id; u < total_units && ok; u += n_pairs) {
@@ -258,7 +257,8 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
                 for (int g = 0; g < G; ++g) acc[m][g] = 0.f;
             const uint32_t tbase = tmem + ((uint32_t)(quarter * 32) << 16) + buf * 256 + grp * 128;
             const float4* q4 = reinterpret_cast<const float4*>(sm.qrot[qb][grp]) + c;
-            const float4* tr4 = &sm.trig[quarter * 32 + r][0];
+            const float4* tr4 = &sm.trig[quarter * 8 + r][0];   // rotation of this thread's first token, quarter*32 + r
+            const float4* tw4 = &sm.trig[32][0] + c;            // rotation by 8 positions
             const int tswz = (r & 1) << 2;                      // odd rows of the table swap 64-byte halves
 #pragma unroll 1
             for (int jc = 0; jc < 2; ++jc) {
@@ -271,9 +271,11 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
                 tmem_wait_ld();
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    float4 tr[4];
-#pragma unroll
-                    for (int m = 0; m < 4; ++m) tr[m] = tr4[m * 8 * 32 + ((jc * 16 + k * 4 + c) ^ tswz)];
+                    // (cos, sin) of this thread's first token for its two rotary pairs, and of the 8-position step
+                    // that leads to its other three tokens (r + 8, r + 16, r + 24): angle addition instead of a
+                    // table row per token
+                    const float4 t0 = tr4[(jc * 16 + k * 4 + c) ^ tswz];
+                    const float4 tw = tw4[jc * 16 + k * 4];
 #pragma unroll
                     for (int e = 0; e < 2; ++e) {
                         float qa[G], qbv[G];
@@ -284,15 +286,21 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
                             qa[g4 * 4 + 0] = x.x; qa[g4 * 4 + 1] = x.y; qa[g4 * 4 + 2] = x.z; qa[g4 * 4 + 3] = x.w;
                             qbv[g4 * 4 + 0] = y.x; qbv[g4 * 4 + 1] = y.y; qbv[g4 * 4 + 2] = y.z; qbv[g4 * 4 + 3] = y.w;
                         }
+                        float cs = e ? t0.z : t0.x, sn = e ? t0.w : t0.y;
+                        const float wc = e ? tw.z : tw.x, ws = e ? tw.w : tw.y;
 #pragma unroll
                         for (int m = 0; m < 4; ++m) {
                             const float a = __uint_as_float(ra[m >> 1][4 * k + 2 * (m & 1) + e]);
                             const float b = __uint_as_float(rb[m >> 1][4 * k + 2 * (m & 1) + e]);
-                            const float cs = e ? tr[m].z : tr[m].x, sn = e ? tr[m].w : tr[m].y;
                             const float ka = a * cs - b * sn;
                             const float kb = a * sn + b * cs;
 #pragma unroll
                             for (int g = 0; g < G; ++g) acc[m][g] = fmaf(qbv[g], kb, fmaf(qa[g], ka, acc[m][g]));
+                            if (m < 3) {
+                                const float nc = cs * wc - sn * ws;
+                                sn = fmaf(cs, ws, sn * wc);
+                                cs = nc;
+                            }
                         }
                     }
                 }
@@ -348,17 +356,21 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
     if (warp == 1) tmem_dealloc_pair(tmem, 512);
 }
 
-// Constant in-tile rotation table (cos, sin)(t * theta_j), t < 128, j < 64, in the layout the score kernel keeps in
-// shared memory: row t holds 32 pieces of 16 bytes, piece (j / 2) ^ (4 (t & 1)) = (cos_j, sin_j, cos_j+1, sin_j+1) for
-// even j.  (The swap of 64-byte halves on odd rows spreads the epilogue's accesses over all banks.)
+// Constant in-tile rotation table in the layout the score kernel keeps in shared memory: 33 rows of 32 pieces of
+// 16 bytes.  Row 8 q + r (q < 4, r < 8) holds (cos, sin)(t theta_j) for the token t = 32 q + r, piece
+// (j / 2) ^ (4 (r & 1)) = (cos_j, sin_j, cos_j+1, sin_j+1) for even j (the swap of 64-byte halves on odd rows spreads
+// the epilogue's accesses over all banks); row 32 holds the same for a step of 8 positions, unswizzled.  The other
+// tokens of a tile follow by angle addition: t + 8 m.
 __global__ void rope_tile_kernel(float2* out, double theta) {
     int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= 64 * TILE) return;
-    int t = i / 64, j = i % 64;
+    if (i >= 33 * 64) return;
+    int row = i / 64, j = i % 64;
+    const int t = row < 32 ? (row >> 3) * 32 + (row & 7) : 8;
+    const int swz = row < 32 ? (row & 1) << 2 : 0;
     double inv = pow(theta, -(double)j / 64.0);
     double sn, cs;
     sincos((double)t * inv, &sn, &cs);
-    out[(t * 32 + ((j >> 1) ^ ((t & 1) << 2))) * 2 + (j & 1)] = make_float2((float)cs, (float)sn);
+    out[(row * 32 + ((j >> 1) ^ swz)) * 2 + (j & 1)] = make_float2((float)cs, (float)sn);
 }
 
 }  // namespace
@@ -467,9 +479,9 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
     LorcTcLayer& TL = T->layers[layer];
     const lorc_model_desc& d = ctx->desc;
     if (!T->rope_tile) {
-        cudaError_t e = cudaMalloc(&T->rope_tile, sizeof(float2) * 64 * TILE);
+        cudaError_t e = cudaMalloc(&T->rope_tile, sizeof(float2) * 64 * 33);
         if (e != cudaSuccess) return e;
-        rope_tile_kernel<<<(64 * TILE + 255) / 256, 256, 0, st>>>(T->rope_tile, d.rope_theta);
+        rope_tile_kernel<<<(64 * 33 + 255) / 256, 256, 0, st>>>(T->rope_tile, d.rope_theta);
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
