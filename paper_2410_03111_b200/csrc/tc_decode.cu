@@ -260,47 +260,46 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
             const float4* tr4 = &sm.trig[quarter * 8 + r][0];   // rotation of this thread's first token, quarter*32 + r
             const float4* tw4 = &sm.trig[32][0] + c;            // rotation by 8 positions
             const int tswz = (r & 1) << 2;                      // odd rows of the table swap 64-byte halves
+            // One 8-column step at a time, NOT unrolled: the loop body stays small enough for the instruction cache
+            // next to the scheduler, which the TMA and MMA warps on the same scheduler need as well.
 #pragma unroll 1
-            for (int jc = 0; jc < 2; ++jc) {
-                uint32_t ra[2][16], rb[2][16];
+            for (int kk = 0; kk < 8; ++kk) {
+                uint32_t ra[2][4], rb[2][4];
 #pragma unroll
                 for (int hf = 0; hf < 2; ++hf) {
-                    tmem_ld16x256_x4(tbase + ((uint32_t)(hf * 16) << 16) + jc * 32, ra[hf]);
-                    tmem_ld16x256_x4(tbase + ((uint32_t)(hf * 16) << 16) + 64 + jc * 32, rb[hf]);
+                    tmem_ld16x256_x1(tbase + ((uint32_t)(hf * 16) << 16) + kk * 8, ra[hf]);
+                    tmem_ld16x256_x1(tbase + ((uint32_t)(hf * 16) << 16) + 64 + kk * 8, rb[hf]);
                 }
+                // (cos, sin) of this thread's first token for its two rotary pairs, and of the 8-position step that
+                // leads to its other three tokens (r + 8, r + 16, r + 24): angle addition instead of a table row per
+                // token
+                const float4 t0 = tr4[(kk * 4 + c) ^ tswz];
+                const float4 tw = tw4[kk * 4];
                 tmem_wait_ld();
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    // (cos, sin) of this thread's first token for its two rotary pairs, and of the 8-position step
-                    // that leads to its other three tokens (r + 8, r + 16, r + 24): angle addition instead of a
-                    // table row per token
-                    const float4 t0 = tr4[(jc * 16 + k * 4 + c) ^ tswz];
-                    const float4 tw = tw4[jc * 16 + k * 4];
+                for (int e = 0; e < 2; ++e) {
+                    float qa[G], qbv[G];
 #pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        float qa[G], qbv[G];
+                    for (int g4 = 0; g4 < G / 4; ++g4) {
+                        const float4 x = q4[(((kk * 2 + e) * 2 + 0) * (G / 4) + g4) * 4];
+                        const float4 y = q4[(((kk * 2 + e) * 2 + 1) * (G / 4) + g4) * 4];
+                        qa[g4 * 4 + 0] = x.x; qa[g4 * 4 + 1] = x.y; qa[g4 * 4 + 2] = x.z; qa[g4 * 4 + 3] = x.w;
+                        qbv[g4 * 4 + 0] = y.x; qbv[g4 * 4 + 1] = y.y; qbv[g4 * 4 + 2] = y.z; qbv[g4 * 4 + 3] = y.w;
+                    }
+                    float cs = e ? t0.z : t0.x, sn = e ? t0.w : t0.y;
+                    const float wc = e ? tw.z : tw.x, ws = e ? tw.w : tw.y;
 #pragma unroll
-                        for (int g4 = 0; g4 < G / 4; ++g4) {
-                            const float4 x = q4[((((jc * 4 + k) * 2 + e) * 2 + 0) * (G / 4) + g4) * 4];
-                            const float4 y = q4[((((jc * 4 + k) * 2 + e) * 2 + 1) * (G / 4) + g4) * 4];
-                            qa[g4 * 4 + 0] = x.x; qa[g4 * 4 + 1] = x.y; qa[g4 * 4 + 2] = x.z; qa[g4 * 4 + 3] = x.w;
-                            qbv[g4 * 4 + 0] = y.x; qbv[g4 * 4 + 1] = y.y; qbv[g4 * 4 + 2] = y.z; qbv[g4 * 4 + 3] = y.w;
-                        }
-                        float cs = e ? t0.z : t0.x, sn = e ? t0.w : t0.y;
-                        const float wc = e ? tw.z : tw.x, ws = e ? tw.w : tw.y;
+                    for (int m = 0; m < 4; ++m) {
+                        const float a = __uint_as_float(ra[m >> 1][2 * (m & 1) + e]);
+                        const float b = __uint_as_float(rb[m >> 1][2 * (m & 1) + e]);
+                        const float ka = a * cs - b * sn;
+                        const float kb = a * sn + b * cs;
 #pragma unroll
-                        for (int m = 0; m < 4; ++m) {
-                            const float a = __uint_as_float(ra[m >> 1][4 * k + 2 * (m & 1) + e]);
-                            const float b = __uint_as_float(rb[m >> 1][4 * k + 2 * (m & 1) + e]);
-                            const float ka = a * cs - b * sn;
-                            const float kb = a * sn + b * cs;
-#pragma unroll
-                            for (int g = 0; g < G; ++g) acc[m][g] = fmaf(qbv[g], kb, fmaf(qa[g], ka, acc[m][g]));
-                            if (m < 3) {
-                                const float nc = cs * wc - sn * ws;
-                                sn = fmaf(cs, ws, sn * wc);
-                                cs = nc;
-                            }
+                        for (int g = 0; g < G; ++g) acc[m][g] = fmaf(qbv[g], kb, fmaf(qa[g], ka, acc[m][g]));
+                        if (m < 3) {
+                            const float nc = cs * wc - sn * ws;
+                            sn = fmaf(cs, ws, sn * wc);
+                            cs = nc;
                         }
                     }
                 }
