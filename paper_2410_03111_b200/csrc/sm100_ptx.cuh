@@ -54,6 +54,24 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
+// The same test and wait on a raw 32-bit shared-memory address (loops that step through barrier arrays).
+__device__ __forceinline__ bool mbar_try_wait_addr(uint32_t bar_addr, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar_addr), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx_addr(uint32_t bar_addr, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_addr), "r"(bytes) : "memory");
+}
+
 // Wait for the phase with the given parity to complete, for at most ~2 seconds.
 #define SM100_WAIT_LIMIT_NS 2000000000ull
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
@@ -64,6 +82,20 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 0x3ff) == 0 && global_timer_ns() - t0 > SM100_WAIT_LIMIT_NS) return false;
     }
+}
+
+static __device__ __noinline__ bool mbar_wait_slow_addr(uint32_t bar_addr, uint32_t parity) {
+    const uint64_t t0 = global_timer_ns();
+    uint32_t spins = 0;
+    while (true) {
+        if (mbar_try_wait_addr(bar_addr, parity)) return true;
+        if ((++spins & 0x3ff) == 0 && global_timer_ns() - t0 > SM100_WAIT_LIMIT_NS) return false;
+    }
+}
+// Bounded wait whose fast path is a single test (the retry loop lives out of line).
+__device__ __forceinline__ bool mbar_wait_addr(uint32_t bar_addr, uint32_t parity) {
+    if (mbar_try_wait_addr(bar_addr, parity)) return true;
+    return mbar_wait_slow_addr(bar_addr, parity);
 }
 
 // Make generic-proxy writes to shared memory visible to the async proxy (TMA, tcgen05.mma).

@@ -126,25 +126,33 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
     tc_fence_after_sync();
     const uint32_t tmem = sm.tmem_base;
 
+    // The two single-thread loops below share their schedulers with epilogue warps that keep them busy, so they are
+    // written to need few issue slots per stage: stage index and phase advance incrementally, shared-memory
+    // addresses and descriptor words are base + stage * constant.
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
         if (lane == 0) {
             // constant in-tile rotation table, fetched while the first stages fill
             mbar_arrive_expect_tx(&sm.trig_full, (uint32_t)sizeof(sm.trig));
             bulk_load(&sm.trig[0][0], p.rope_tile, (uint32_t)sizeof(sm.trig), &sm.trig_full);
-            uint32_t it = 0;
+            const uint32_t a_base = smem_u32(sm.A[0]), b_base = smem_u32(sm.B[0]);
+            const uint32_t empty0 = smem_u32(&sm.empty[0]), full0 = smem_u32(&sm.full[0]);
+            const uint32_t lead_full0 = mapa_shared(full0, 0);   // all bytes of a stage are counted on the leader's barrier
+            const bool paged = p.page_table != nullptr;
+            const int b_row = rank * 128;
+            uint32_t st = 0, par = 1;                            // stage and the parity its empty barrier is waited with
             bool ok = true;
             for (int u = pair_id; u < total_units && ok; u += n_pairs) {
                 Unit un;
                 if (!decode_unit(p, u, rank, un)) continue;
-                for (int kc = 0; kc < nkc; ++kc, ++it) {
-                    const int st = it % S_STAGES;
-                    if (!mbar_wait(&sm.empty[st], ((it / S_STAGES) & 1) ^ 1)) { ok = false; break; }
-                    // all bytes of the stage, from both CTAs, are counted on the leader's barrier
-                    const uint32_t lead_bar = mapa_shared(smem_u32(&sm.full[st]), 0);
-                    if (rank == 0) mbar_arrive_expect_tx(&sm.full[st], 2 * 2 * TILE * KC * 2);
-                    if (p.page_table == nullptr) {
-                        tma_load_3d_pair(sm.A[st], &mapCK, lead_bar, kc * KC, un.tile * TILE, un.s);
+                const int row0 = un.tile * TILE, brow = un.hp * 256 + b_row;
+                for (int x = 0; x < nkc * KC; x += KC) {
+                    if (!mbar_wait_addr(empty0 + st * 8, par)) { ok = false; break; }
+                    if (rank == 0) mbar_arrive_expect_tx_addr(full0 + st * 8, 2 * 2 * TILE * KC * 2);
+                    const uint32_t lead_bar = lead_full0 + st * 8;
+                    const uint32_t a_dst = a_base + st * (TILE * KC * 2);
+                    if (!paged) {
+                        tma_load_3d_pair_addr(a_dst, &mapCK, lead_bar, x, row0, un.s);
                     } else {
                         // one box per page; pages past the end of the sequence (or with a bad table entry) are read
                         // from page 0: those rows are masked, but every box must deliver its bytes
@@ -159,19 +167,29 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
                                     page = 0;
                                 }
                             }
-                            tma_load_3d_pair(sm.A[st] + pg * p.page_size * KC, &mapCK, lead_bar, kc * KC, 0, page);
+                            tma_load_3d_pair_addr(a_dst + pg * p.page_size * KC * 2, &mapCK, lead_bar, x, 0, page);
                         }
                     }
-                    tma_load_2d_pair(sm.B[st], &mapBKT, lead_bar, kc * KC, un.hp * 256 + rank * 128);
+                    tma_load_2d_pair_addr(b_base + st * (128 * KC * 2), &mapBKT, lead_bar, x, brow);
+                    if (++st == S_STAGES) { st = 0; par ^= 1; }
                 }
             }
             if (!ok) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader CTA only)
-        if (lane == 0 && rank == 0) {
+        // The whole warp walks the loop (so the compiler can keep addresses and descriptor words in uniform
+        // registers, which is what the MMA instruction takes); one elected lane issues.
+        if (rank == 0) {
             const uint32_t idesc = make_idesc_bf16(256, 256, 0, 0);
-            uint32_t it = 0, uc = 0;
+            // descriptor words of stage 0, k-step 0; a stage adds its byte offset >> 4 to the low word, a k-step
+            // (16 columns = 32 bytes inside the 128-byte swizzle row) adds 2
+            const uint64_t da0 = make_smem_desc_sw128(smem_u32(sm.A[0]), 0, 1024);
+            const uint64_t db0 = make_smem_desc_sw128(smem_u32(sm.B[0]), 0, 1024);
+            const uint32_t a_lo0 = (uint32_t)da0, a_hi = (uint32_t)(da0 >> 32);
+            const uint32_t b_lo0 = (uint32_t)db0, b_hi = (uint32_t)(db0 >> 32);
+            const uint32_t empty0 = smem_u32(&sm.empty[0]), full0 = smem_u32(&sm.full[0]);
+            uint32_t st = 0, par = 0, uc = 0;
             bool ok = true;
             for (int u = pair_id; u < total_units && ok; u += n_pairs) {
                 Unit un;
@@ -179,23 +197,30 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
                 const int buf = uc & 1;
                 if (!mbar_wait(&sm.acc_empty[buf], ((uc >> 1) & 1) ^ 1)) { ok = false; break; }
                 tc_fence_after_sync();
-                for (int kc = 0; kc < nkc; ++kc, ++it) {
-                    const int st = it % S_STAGES;
-                    if (!mbar_wait(&sm.full[st], (it / S_STAGES) & 1)) { ok = false; break; }
+                const uint32_t d = tmem + buf * 256;
+                for (int kc = 0; kc < nkc; ++kc) {
+                    if (!mbar_wait_addr(full0 + st * 8, par)) { ok = false; break; }
                     tc_fence_after_sync();
-                    const uint32_t a0 = smem_u32(sm.A[st]), b0 = smem_u32(sm.B[st]);
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        tc_mma_bf16_pair(tmem + buf * 256, make_smem_desc_sw128(a0 + k * 32, 0, 1024),
-                                         make_smem_desc_sw128(b0 + k * 32, 0, 1024), idesc, (kc | k) != 0);
+                    const uint32_t a_lo = a_lo0 + st * (TILE * KC * 2 / 16), b_lo = b_lo0 + st * (128 * KC * 2 / 16);
+                    if (elect_one()) {
+                        if (kc == 0)
+                            tc_mma_bf16_pair_set(d, a_lo, a_hi, b_lo, b_hi, idesc);
+                        else
+                            tc_mma_bf16_pair_acc(d, a_lo, a_hi, b_lo, b_hi, idesc);
+                        tc_mma_bf16_pair_acc(d, a_lo + 2, a_hi, b_lo + 2, b_hi, idesc);
+                        tc_mma_bf16_pair_acc(d, a_lo + 4, a_hi, b_lo + 4, b_hi, idesc);
+                        tc_mma_bf16_pair_acc(d, a_lo + 6, a_hi, b_lo + 6, b_hi, idesc);
+                        tc_commit_pair_addr(empty0 + st * 8);        // frees the stage in both CTAs
                     }
-                    tc_commit_pair(&sm.empty[st]);        // frees the stage in both CTAs
+                    __syncwarp();
+                    if (++st == S_STAGES) { st = 0; par ^= 1; }
                 }
                 if (!ok) break;
-                tc_commit_pair(&sm.acc_full[buf]);        // both CTAs' epilogues may read their accumulators
+                if (elect_one()) tc_commit_pair(&sm.acc_full[buf]);   // both CTAs' epilogues may read their accumulators
+                __syncwarp();
                 ++uc;
             }
-            if (!ok) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
+            if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
         }
     } else {
         // ------------------------------------------------------------------ epilogue: RoPE + scores
