@@ -131,10 +131,13 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
     // addresses and descriptor words are base + stage * constant.
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
+        // (whole warp in the loop, one elected lane issues: see the MMA warp below)
         if (lane == 0) {
             // constant in-tile rotation table, fetched while the first stages fill
             mbar_arrive_expect_tx(&sm.trig_full, (uint32_t)sizeof(sm.trig));
             bulk_load(&sm.trig[0][0], p.rope_tile, (uint32_t)sizeof(sm.trig), &sm.trig_full);
+        }
+        {
             const uint32_t a_base = smem_u32(sm.A[0]), b_base = smem_u32(sm.B[0]);
             const uint32_t empty0 = smem_u32(&sm.empty[0]), full0 = smem_u32(&sm.full[0]);
             const uint32_t lead_full0 = mapa_shared(full0, 0);   // all bytes of a stage are counted on the leader's barrier
@@ -148,33 +151,36 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
                 const int row0 = un.tile * TILE, brow = un.hp * 256 + b_row;
                 for (int x = 0; x < nkc * KC; x += KC) {
                     if (!mbar_wait_addr(empty0 + st * 8, par)) { ok = false; break; }
-                    if (rank == 0) mbar_arrive_expect_tx_addr(full0 + st * 8, 2 * 2 * TILE * KC * 2);
                     const uint32_t lead_bar = lead_full0 + st * 8;
                     const uint32_t a_dst = a_base + st * (TILE * KC * 2);
-                    if (!paged) {
-                        tma_load_3d_pair_addr(a_dst, &mapCK, lead_bar, x, row0, un.s);
-                    } else {
-                        // one box per page; pages past the end of the sequence (or with a bad table entry) are read
-                        // from page 0: those rows are masked, but every box must deliver its bytes
-                        const int ppt = TILE / p.page_size;
-                        for (int pg = 0; pg < ppt; ++pg) {
-                            const int lp = un.tile * ppt + pg;
-                            int page = 0;
-                            if ((long long)lp * p.page_size < un.len && lp < p.max_pages_per_seq) {
-                                page = p.page_table[(long long)un.s * p.max_pages_per_seq + lp];
-                                if (page < 0 || page >= p.n_pages) {
-                                    lorc_set_status(p.status, LORC_ERR_CAPACITY);
-                                    page = 0;
+                    if (elect_one()) {
+                        if (rank == 0) mbar_arrive_expect_tx_addr(full0 + st * 8, 2 * 2 * TILE * KC * 2);
+                        if (!paged) {
+                            tma_load_3d_pair_addr(a_dst, &mapCK, lead_bar, x, row0, un.s);
+                        } else {
+                            // one box per page; pages past the end of the sequence (or with a bad table entry) are
+                            // read from page 0: those rows are masked, but every box must deliver its bytes
+                            const int ppt = TILE / p.page_size;
+                            for (int pg = 0; pg < ppt; ++pg) {
+                                const int lp = un.tile * ppt + pg;
+                                int page = 0;
+                                if ((long long)lp * p.page_size < un.len && lp < p.max_pages_per_seq) {
+                                    page = p.page_table[(long long)un.s * p.max_pages_per_seq + lp];
+                                    if (page < 0 || page >= p.n_pages) {
+                                        lorc_set_status(p.status, LORC_ERR_CAPACITY);
+                                        page = 0;
+                                    }
                                 }
+                                tma_load_3d_pair_addr(a_dst + pg * p.page_size * KC * 2, &mapCK, lead_bar, x, 0, page);
                             }
-                            tma_load_3d_pair_addr(a_dst + pg * p.page_size * KC * 2, &mapCK, lead_bar, x, 0, page);
                         }
+                        tma_load_2d_pair_addr(b_base + st * (128 * KC * 2), &mapBKT, lead_bar, x, brow);
                     }
-                    tma_load_2d_pair_addr(b_base + st * (128 * KC * 2), &mapBKT, lead_bar, x, brow);
+                    __syncwarp();
                     if (++st == S_STAGES) { st = 0; par ^= 1; }
                 }
             }
-            if (!ok) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
+            if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader CTA only)
