@@ -215,12 +215,15 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        // The whole warp walks the loop and one elected lane issues: the asynchronous instructions take their
+        // operands from uniform registers, which the compiler only uses in warp-uniform code.
+        {
             for (int i = 0; i < ntiles && ok; ++i) {
                 const int tile = tile_lo + i;
                 const int n0 = tile * TILE;
                 const int st = i % P_STAGES;
                 if (!mbar_wait(&sm.empty[st], ((i / P_STAGES) & 1) ^ 1)) { ok = false; break; }
+                if (elect_one()) {
                 mbar_arrive_expect_tx(&sm.full[st], 2 * TILE * KC * 2 + P_BYTES);
                 bulk_load(sm.P[st][0], p.probs + ((long long)s * p.tiles + tile) * (2 * HQ * KC), P_BYTES, &sm.full[st]);
                 if (p.page_table == nullptr) {
@@ -245,30 +248,36 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
                         tma_load_3d(sm.V[st][1] + pg * p.page_size * KC, &mapCV, &sm.full[st], rho0 + 64, 0, page);
                     }
                 }
+                }
+                __syncwarp();
             }
-            if (!ok) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
+            if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0 && ntiles > 0) {
+        // ------------------------------------------------------------------ MMA issuer (warp-uniform, elected lane)
+        if (ntiles > 0) {
             const uint32_t idesc = make_idesc_bf16(128, HQ, 1, 0);
             for (int i = 0; i < ntiles && ok; ++i) {
                 const int st = i % P_STAGES;
                 if (!mbar_wait(&sm.full[st], (i / P_STAGES) & 1)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t p0 = smem_u32(sm.P[st][0]), v0 = smem_u32(sm.V[st][0]);
+                if (elect_one()) {
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    // A: C_V^T block (MN-major): 16 token rows per step, the two 64-column halves 16 KiB apart
-                    const uint64_t ad = make_smem_desc_sw128(v0 + k * 2048, TILE * KC * 2, 1024);
-                    // B: P [HQ][128 tokens] (K-major), 64-token chunks of HQ*128 bytes
-                    const uint64_t bd = make_smem_desc_sw128(p0 + (k >> 2) * (HQ * KC * 2) + (k & 3) * 32, 0, 1024);
-                    tc_mma_bf16(tmem, ad, bd, idesc, (i | k) != 0);
+                    for (int k = 0; k < 8; ++k) {
+                        // A: C_V^T block (MN-major): 16 token rows per step, the two 64-column halves 16 KiB apart
+                        const uint64_t ad = make_smem_desc_sw128(v0 + k * 2048, TILE * KC * 2, 1024);
+                        // B: P [HQ][128 tokens] (K-major), 64-token chunks of HQ*128 bytes
+                        const uint64_t bd = make_smem_desc_sw128(p0 + (k >> 2) * (HQ * KC * 2) + (k & 3) * 32, 0, 1024);
+                        tc_mma_bf16(tmem, ad, bd, idesc, (i | k) != 0);
+                    }
+                    tc_commit(&sm.empty[st]);
                 }
-                tc_commit(&sm.empty[st]);
+                __syncwarp();
             }
-            tc_commit(&sm.o_full);
-            if (!ok) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
+            if (elect_one()) tc_commit(&sm.o_full);
+            __syncwarp();
+            if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
         }
     } else {
         // ------------------------------------------------------------------ epilogue
@@ -402,34 +411,38 @@ lorc_upproj_kernel(const __grid_constant__ CUtensorMap mapON, const __grid_const
     bool ok = true;
 
     if (warp == 0) {
-        if (lane == 0) {
-            for (int kc = 0; kc < nkc; ++kc) {
-                const int st = kc % U_STAGES;
-                if (!mbar_wait(&sm.empty[st], ((kc / U_STAGES) & 1) ^ 1)) { ok = false; break; }
+        // (warp-uniform loops, one elected lane issues)
+        for (int kc = 0; kc < nkc; ++kc) {
+            const int st = kc % U_STAGES;
+            if (!mbar_wait(&sm.empty[st], ((kc / U_STAGES) & 1) ^ 1)) { ok = false; break; }
+            if (elect_one()) {
                 mbar_arrive_expect_tx(&sm.full[st], 2 * 128 * KC * 2);
                 // rows (s, i): box of G heads x 128/G sequences (sequences past the batch read as zero)
                 tma_load_3d(sm.A[st], &mapON, &sm.full[st], kc * KC, g * p.G, chunk * seqs_per_cta);
                 tma_load_2d(sm.B[st], &mapBVT, &sm.full[st], kc * KC, g * 128);
             }
-            if (!ok) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
+            __syncwarp();
         }
+        if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
     } else if (warp == 1) {
-        if (lane == 0) {
-            const uint32_t idesc = make_idesc_bf16(128, 128, 0, 0);
-            for (int kc = 0; kc < nkc; ++kc) {
-                const int st = kc % U_STAGES;
-                if (!mbar_wait(&sm.full[st], (kc / U_STAGES) & 1)) { ok = false; break; }
-                tc_fence_after_sync();
-                const uint32_t a0 = smem_u32(sm.A[st]), b0 = smem_u32(sm.B[st]);
+        const uint32_t idesc = make_idesc_bf16(128, 128, 0, 0);
+        for (int kc = 0; kc < nkc; ++kc) {
+            const int st = kc % U_STAGES;
+            if (!mbar_wait(&sm.full[st], (kc / U_STAGES) & 1)) { ok = false; break; }
+            tc_fence_after_sync();
+            const uint32_t a0 = smem_u32(sm.A[st]), b0 = smem_u32(sm.B[st]);
+            if (elect_one()) {
 #pragma unroll
                 for (int k = 0; k < 4; ++k)
                     tc_mma_bf16(tmem, make_smem_desc_sw128(a0 + k * 32, 0, 1024), make_smem_desc_sw128(b0 + k * 32, 0, 1024),
                                 idesc, (kc | k) != 0);
                 tc_commit(&sm.empty[st]);
             }
-            tc_commit(&sm.d_full);
-            if (!ok) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
+            __syncwarp();
         }
+        if (elect_one()) tc_commit(&sm.d_full);
+        __syncwarp();
+        if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
     } else {
         if (!mbar_wait(&sm.d_full, 0)) ok = false;
         if (ok) {
