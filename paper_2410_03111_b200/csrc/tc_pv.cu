@@ -57,52 +57,62 @@ __device__ __forceinline__ int prob_image_offset(int h, int tc) {
     return h * 128 + ((((tc >> 3) ^ (h & 7)) << 4) | ((tc & 7) << 1));
 }
 
+// 256 threads: thread = (token of the tile, half of the heads).
 template <int HQ>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(256)
 lorc_prob_kernel(const ProbParams p) {
+    constexpr int NH = HQ / 2;                        // heads per thread
     __shared__ float m_s[HQ];
-    __shared__ float red[4][HQ];
-    const int t = threadIdx.x, warp = t / 32, lane = t % 32;
+    __shared__ float red[8][HQ];
+    const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
+    const int t = tid & 127, hh = tid >> 7, h0 = hh * NH;
     const int grp = blockIdx.x, s = blockIdx.y;
     int len = p.seq_lens[s];
     if (len > p.max_pos || len < 0) len = 0;        // the score kernel reports the capacity error
     const int tiles_s = (len + TILE - 1) / TILE;
     const int tile_lo = min(tiles_s, grp * p.tiles_per_group), tile_hi = min(tiles_s, tile_lo + p.tiles_per_group);
-    if (grp == 0 && t < p.n_blk) p.done[s * p.n_blk + t] = 0;
-    float l[HQ];
+    if (grp == 0 && tid < p.n_blk) p.done[s * p.n_blk + tid] = 0;
+    float l[NH];
 #pragma unroll
-    for (int h = 0; h < HQ; ++h) l[h] = 0.f;
+    for (int i = 0; i < NH; ++i) l[i] = 0.f;
     if (tile_lo < tile_hi) {
         // the scores of the first tile are requested before the maxima, so the two round trips overlap
-        float sv[HQ];
-        const float* sbase = p.scores + (long long)s * p.H_q * p.n_pad + t;
+        float sv[NH];
+        const float* sbase = p.scores + ((long long)s * p.H_q + h0) * p.n_pad + t;
         {
             const int n = tile_lo * TILE + t;
 #pragma unroll
-            for (int h = 0; h < HQ; ++h) sv[h] = n < len ? ldg_nc_f32(sbase + (long long)h * p.n_pad + tile_lo * TILE) : 0.f;
+            for (int i = 0; i < NH; ++i) sv[i] = n < len ? ldg_nc_f32(sbase + (long long)i * p.n_pad + tile_lo * TILE) : 0.f;
         }
         // exact maximum of every head over the WHOLE sequence ([tile][4 quarters] per head: one 16-byte load per
-        // tile, eight tiles in flight per thread)
-        for (int idx = t; idx < HQ * 4; idx += 128) {          // (head, tile phase)
-            const int h = idx >> 2, ph = idx & 3;
+        // tile; a thread takes every eighth tile of one head, eight loads in flight)
+        for (int idx = tid; idx < HQ * 8; idx += 256) {          // (head, tile phase)
+            const int h = idx >> 3, ph = idx & 7;
             const float4* tp = reinterpret_cast<const float4*>(p.tmax + ((long long)s * p.H_q + h) * (4 * p.tiles));
             float v = -INFINITY;
             int i = ph;
-            for (; i + 28 < tiles_s; i += 32) {
+            for (; i + 56 < tiles_s; i += 64) {
                 float4 q[8];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) q[u] = tp[i + 4 * u];
+                for (int u = 0; u < 8; ++u) q[u] = tp[i + 8 * u];
 #pragma unroll
                 for (int u = 0; u < 8; ++u) v = fmaxf(v, fmaxf(fmaxf(q[u].x, q[u].y), fmaxf(q[u].z, q[u].w)));
             }
-            for (; i < tiles_s; i += 4) {
-                const float4 q = tp[i];
-                v = fmaxf(v, fmaxf(fmaxf(q.x, q.y), fmaxf(q.z, q.w)));
-            }
+            float4 q[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                q[u] = (i + 8 * u < tiles_s) ? tp[i + 8 * u] : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v = fmaxf(v, fmaxf(fmaxf(q[u].x, q[u].y), fmaxf(q[u].z, q[u].w)));
             red[ph][h] = v;
         }
         __syncthreads();
-        if (t < HQ) m_s[t] = fmaxf(fmaxf(red[0][t], red[1][t]), fmaxf(red[2][t], red[3][t]));
+        if (tid < HQ) {
+            float v = red[0][tid];
+#pragma unroll
+            for (int i = 1; i < 8; ++i) v = fmaxf(v, red[i][tid]);
+            m_s[tid] = v;
+        }
         __syncthreads();
         for (int tile = tile_lo; tile < tile_hi; ++tile) {
             const bool valid = tile * TILE + t < len;
@@ -110,37 +120,53 @@ lorc_prob_kernel(const ProbParams p) {
                            (((long long)s * p.tiles + tile) * 2 + (t >> 6)) * (HQ * KC * 2);
             const int tc = t & 63;
             float ssum = 0.f;
-            bf16 pr[HQ];
+            bf16 pr[NH];
 #pragma unroll
-            for (int h = 0; h < HQ; ++h) {
-                ssum += sv[h];
+            for (int i = 0; i < NH; ++i) {
+                ssum += sv[i];
                 // p = 2^(s - m), rounded to bf16 (the same rounded value enters the denominator)
-                pr[h] = __float2bfloat16_rn(valid ? exp2f(sv[h] - m_s[h]) : 0.f);
-                l[h] += __bfloat162float(pr[h]);
+                pr[i] = __float2bfloat16_rn(valid ? exp2f(sv[i] - m_s[h0 + i]) : 0.f);
+                l[i] += __bfloat162float(pr[i]);
             }
             // a NaN among the scores means non-finite numbers in the cache, the factors or the query
             if (ssum != ssum) lorc_set_status(p.status, LORC_ERR_ARG);
             if (tile + 1 < tile_hi) {
                 const int n = (tile + 1) * TILE + t;
 #pragma unroll
-                for (int h = 0; h < HQ; ++h)
-                    sv[h] = n < len ? ldg_nc_f32(sbase + (long long)h * p.n_pad + (tile + 1) * TILE) : 0.f;
+                for (int i = 0; i < NH; ++i)
+                    sv[i] = n < len ? ldg_nc_f32(sbase + (long long)i * p.n_pad + (tile + 1) * TILE) : 0.f;
             }
 #pragma unroll
-            for (int h = 0; h < HQ; ++h) *reinterpret_cast<bf16*>(img + prob_image_offset(h, tc)) = pr[h];
+            for (int i = 0; i < NH; ++i) *reinterpret_cast<bf16*>(img + prob_image_offset(h0 + i, tc)) = pr[i];
         }
     }
-    // this group's share of the softmax denominator (zero for a group past the end of the sequence)
+    // This group's share of the softmax denominator (zero for a group past the end of the sequence).  A warp holds
+    // 32 tokens x NH heads; each exchange step halves the heads a lane carries, so NH - 1 (+1) shuffles add them all.
     __syncthreads();
+    {
+        int n = NH;
 #pragma unroll
-    for (int h = 0; h < HQ; ++h) {
-        float v = l[h];
+        for (int step = 16; step >= 1; step >>= 1) {
+            if (n > 1) {
+                const bool upper = (lane & step) != 0;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        if (lane == 0) red[warp][h] = v;
+                for (int i = 0; i < NH / 2; ++i) {
+                    if (i < n / 2) {
+                        const float keep = upper ? l[i + n / 2] : l[i];
+                        const float send = upper ? l[i] : l[i + n / 2];
+                        l[i] = keep + __shfl_xor_sync(0xffffffffu, send, step);
+                    }
+                }
+                n >>= 1;
+            } else {
+                l[0] += __shfl_xor_sync(0xffffffffu, l[0], step);
+            }
+        }
+        // the lane now holds head (lane * NH / 32) of its half
+        if ((lane & (32 / NH - 1)) == 0) red[warp & 3][h0 + lane * NH / 32] = l[0];
     }
     __syncthreads();
-    if (t < HQ) p.l_part[((long long)s * p.n_groups + grp) * p.H_q + t] = red[0][t] + red[1][t] + red[2][t] + red[3][t];
+    if (tid < HQ) p.l_part[((long long)s * p.n_groups + grp) * p.H_q + tid] = red[0][tid] + red[1][tid] + red[2][tid] + red[3][tid];
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -577,9 +603,9 @@ cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView
         q.n_groups = n_groups; q.n_blk = n_blk; q.max_pos = d.max_pos;
         dim3 pgrid(n_groups, cv.batch);
         if (d.n_q_heads == 32)
-            lorc_prob_kernel<32><<<pgrid, 128, 0, st>>>(q);
+            lorc_prob_kernel<32><<<pgrid, 256, 0, st>>>(q);
         else
-            lorc_prob_kernel<64><<<pgrid, 128, 0, st>>>(q);
+            lorc_prob_kernel<64><<<pgrid, 256, 0, st>>>(q);
         *launches += 1;
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
