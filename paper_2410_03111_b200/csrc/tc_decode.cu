@@ -188,6 +188,7 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
         // registers, which is what the MMA instruction takes); one elected lane issues.
         if (rank == 0) {
             const uint32_t idesc = make_idesc_bf16(256, 256, 0, 0);
+            const int nk_last = (p.r_k - (nkc - 1) * KC + 15) >> 4;   // 16-column steps the last stage really holds
             // descriptor words of stage 0, k-step 0; a stage adds its byte offset >> 4 to the low word, a k-step
             // (16 columns = 32 bytes inside the 128-byte swizzle row) adds 2
             const uint64_t da0 = make_smem_desc_sw128(smem_u32(sm.A[0]), 0, 1024);
@@ -213,9 +214,10 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
                             tc_mma_bf16_pair_set(d, a_lo, a_hi, b_lo, b_hi, idesc);
                         else
                             tc_mma_bf16_pair_acc(d, a_lo, a_hi, b_lo, b_hi, idesc);
-                        tc_mma_bf16_pair_acc(d, a_lo + 2, a_hi, b_lo + 2, b_hi, idesc);
-                        tc_mma_bf16_pair_acc(d, a_lo + 4, a_hi, b_lo + 4, b_hi, idesc);
-                        tc_mma_bf16_pair_acc(d, a_lo + 6, a_hi, b_lo + 6, b_hi, idesc);
+                        const int nk = (kc + 1 < nkc) ? 4 : nk_last;
+                        if (nk > 1) tc_mma_bf16_pair_acc(d, a_lo + 2, a_hi, b_lo + 2, b_hi, idesc);
+                        if (nk > 2) tc_mma_bf16_pair_acc(d, a_lo + 4, a_hi, b_lo + 4, b_hi, idesc);
+                        if (nk > 3) tc_mma_bf16_pair_acc(d, a_lo + 6, a_hi, b_lo + 6, b_hi, idesc);
                         tc_commit_pair_addr(empty0 + st * 8);        // frees the stage in both CTAs
                     }
                     __syncwarp();
