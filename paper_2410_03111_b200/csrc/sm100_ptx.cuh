@@ -16,6 +16,15 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return (uint32_t)__cvta_generic_to_shared(p);
 }
 
+// Programmatic dependent launch.  A kernel launched with the programmatic-serialization attribute may start while
+// the kernel before it in the stream still runs.  grid_dep_wait() returns once that kernel has completed and its
+// writes are visible; grid_dep_launch() lets the kernel AFTER this one start early in the same way.  Every kernel here
+// calls grid_dep_launch() only after its own grid_dep_wait() and after it has claimed its tensor memory: a kernel
+// that has started therefore knows that everything up to the predecessor of its predecessor is complete, and can
+// never hold tensor memory that a block of an earlier kernel is still waiting for.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ uint64_t global_timer_ns() {
     uint64_t t;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -304,4 +313,21 @@ static inline bool lorc_make_tmap_bf16(CUtensorMap* map, const void* base, int r
                      es, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
+}
+
+// Launch with the programmatic-serialization attribute (see grid_dep_wait above).
+template <typename... KArgs>
+static inline cudaError_t lorc_launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                                cudaStream_t stream, KArgs... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
 }

@@ -114,7 +114,13 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
         fence_barrier_init();
         prefetch_tensormap(&mapCK);
         prefetch_tensormap(&mapBKT);
+        // constant in-tile rotation table: does not depend on earlier work in the stream
+        mbar_arrive_expect_tx(&sm.trig_full, (uint32_t)sizeof(sm.trig));
+        bulk_load(&sm.trig[0][0], p.rope_tile, (uint32_t)sizeof(sm.trig), &sm.trig_full);
     }
+    // Everything above may overlap the tail of the previous kernel in the stream; inputs are read, results written
+    // and tensor memory claimed only once that kernel has completed.
+    grid_dep_wait();
     if (warp == 1) {
         tmem_alloc_pair(&sm.tmem_base, 512);
         tmem_relinquish_pair();
@@ -124,6 +130,7 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
     cluster_arrive_release();                            // the peer's barriers are initialised before anyone signals them
     cluster_wait_acquire();
     tc_fence_after_sync();
+    grid_dep_launch();
     const uint32_t tmem = sm.tmem_base;
 
     // The two single-thread loops below share their schedulers with epilogue warps that keep them busy, so they are
@@ -132,11 +139,6 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
         // (whole warp in the loop, one elected lane issues: see the MMA warp below)
-        if (lane == 0) {
-            // constant in-tile rotation table, fetched while the first stages fill
-            mbar_arrive_expect_tx(&sm.trig_full, (uint32_t)sizeof(sm.trig));
-            bulk_load(&sm.trig[0][0], p.rope_tile, (uint32_t)sizeof(sm.trig), &sm.trig_full);
-        }
         {
             const uint32_t a_base = smem_u32(sm.A[0]), b_base = smem_u32(sm.B[0]);
             const uint32_t empty0 = smem_u32(&sm.empty[0]), full0 = smem_u32(&sm.full[0]);
@@ -558,14 +560,14 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
     const size_t smem1 = sizeof(ScoreSmem) + 1024;
     {
         LorcStageTimer timer(ctx, LORC_STAGE_SCORE, st);
+        cudaError_t e;
         if (ctx->group == 4)
-            lorc_score_kernel<4><<<grid1, S_THREADS, smem1, st>>>(TL.mapCK, TL.mapBKT, sp);
+            e = lorc_launch_dependent(lorc_score_kernel<4>, dim3(grid1), dim3(S_THREADS), smem1, st, TL.mapCK, TL.mapBKT, sp);
         else
-            lorc_score_kernel<8><<<grid1, S_THREADS, smem1, st>>>(TL.mapCK, TL.mapBKT, sp);
+            e = lorc_launch_dependent(lorc_score_kernel<8>, dim3(grid1), dim3(S_THREADS), smem1, st, TL.mapCK, TL.mapBKT, sp);
+        *launches += 1;
+        if (e != cudaSuccess) return e;
     }
-    *launches += 1;
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
     return lorc_tc_pv_launch(ctx, L, cv, TL.mapCV, TL.mapBVT, scores, tmax, n_pad, tiles, n_splits, pv_scratch, pv_bytes,
                              out, st, launches);
 }

@@ -67,6 +67,8 @@ lorc_prob_kernel(const ProbParams p) {
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
     const int t = tid & 127, hh = tid >> 7, h0 = hh * NH;
     const int grp = blockIdx.x, s = blockIdx.y;
+    grid_dep_wait();                                 // the scores come from the kernel before this one
+    grid_dep_launch();
     int len = p.seq_lens[s];
     if (len > p.max_pos || len < 0) len = 0;        // the score kernel reports the capacity error
     const int tiles_s = (len + TILE - 1) / TILE;
@@ -243,15 +245,29 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
         // ------------------------------------------------------------------ TMA producer
         // The whole warp walks the loop and one elected lane issues: the asynchronous instructions take their
         // operands from uniform registers, which the compiler only uses in warp-uniform code.
+        // The kernel before this one only writes the probabilities and denominators; the latent values were complete
+        // before IT could start.  So the first stages' C_V boxes are requested right away, and only the probability
+        // tiles wait for that kernel to finish.
         {
             for (int i = 0; i < ntiles && ok; ++i) {
                 const int tile = tile_lo + i;
                 const int n0 = tile * TILE;
                 const int st = i % P_STAGES;
+                if (i == P_STAGES) {
+                    // probability tiles of the stages whose C_V boxes went out before the wait
+                    grid_dep_wait();
+                    if (elect_one()) {
+                        for (int j = 0; j < P_STAGES; ++j)
+                            bulk_load(sm.P[j][0], p.probs + ((long long)s * p.tiles + tile_lo + j) * (2 * HQ * KC), P_BYTES,
+                                      &sm.full[j]);
+                    }
+                    __syncwarp();
+                }
                 if (!mbar_wait(&sm.empty[st], ((i / P_STAGES) & 1) ^ 1)) { ok = false; break; }
                 if (elect_one()) {
                 mbar_arrive_expect_tx(&sm.full[st], 2 * TILE * KC * 2 + P_BYTES);
-                bulk_load(sm.P[st][0], p.probs + ((long long)s * p.tiles + tile) * (2 * HQ * KC), P_BYTES, &sm.full[st]);
+                if (i >= P_STAGES)
+                    bulk_load(sm.P[st][0], p.probs + ((long long)s * p.tiles + tile) * (2 * HQ * KC), P_BYTES, &sm.full[st]);
                 if (p.page_table == nullptr) {
                     tma_load_3d(sm.V[st][0], &mapCV, &sm.full[st], rho0, n0, s);
                     tma_load_3d(sm.V[st][1], &mapCV, &sm.full[st], rho0 + 64, n0, s);
@@ -274,6 +290,15 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
                         tma_load_3d(sm.V[st][1] + pg * p.page_size * KC, &mapCV, &sm.full[st], rho0 + 64, 0, page);
                     }
                 }
+                }
+                __syncwarp();
+            }
+            if (ntiles <= P_STAGES) {
+                grid_dep_wait();
+                if (elect_one()) {
+                    for (int j = 0; j < ntiles; ++j)
+                        bulk_load(sm.P[j][0], p.probs + ((long long)s * p.tiles + tile_lo + j) * (2 * HQ * KC), P_BYTES,
+                                  &sm.full[j]);
                 }
                 __syncwarp();
             }
@@ -311,6 +336,8 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
         const int quarter = warp % 4;
         const int row = quarter * 32 + lane;              // TMEM lane = latent row of the block
         const int r_pad = p.n_blk * 128;
+        grid_dep_wait();                              // denominators come from the kernel before this one
+        grid_dep_launch();
         // while the tiles stream: the reciprocal softmax denominator of every head (all shares of the sequence)
         {
             constexpr int PARTS = 128 / HQ;
@@ -438,14 +465,28 @@ lorc_upproj_kernel(const __grid_constant__ CUtensorMap mapON, const __grid_const
 
     if (warp == 0) {
         // (warp-uniform loops, one elected lane issues)
+        // The factor slices of the first stages do not depend on the kernel before this one: they are requested
+        // before the wait, the latent rows after it.
+        const int npre = nkc < U_STAGES ? nkc : U_STAGES;
+        if (elect_one()) {
+            for (int kc = 0; kc < npre; ++kc) {
+                mbar_arrive_expect_tx(&sm.full[kc], 2 * 128 * KC * 2);
+                tma_load_2d(sm.B[kc], &mapBVT, &sm.full[kc], kc * KC, g * 128);
+            }
+        }
+        __syncwarp();
+        grid_dep_wait();                             // the normalised latent rows come from the kernel before
+        grid_dep_launch();
         for (int kc = 0; kc < nkc; ++kc) {
             const int st = kc % U_STAGES;
-            if (!mbar_wait(&sm.empty[st], ((kc / U_STAGES) & 1) ^ 1)) { ok = false; break; }
+            if (kc >= npre && !mbar_wait(&sm.empty[st], ((kc / U_STAGES) & 1) ^ 1)) { ok = false; break; }
             if (elect_one()) {
-                mbar_arrive_expect_tx(&sm.full[st], 2 * 128 * KC * 2);
+                if (kc >= npre) {
+                    mbar_arrive_expect_tx(&sm.full[st], 2 * 128 * KC * 2);
+                    tma_load_2d(sm.B[st], &mapBVT, &sm.full[st], kc * KC, g * 128);
+                }
                 // rows (s, i): box of G heads x 128/G sequences (sequences past the batch read as zero)
                 tma_load_3d(sm.A[st], &mapON, &sm.full[st], kc * KC, g * p.G, chunk * seqs_per_cta);
-                tma_load_2d(sm.B[st], &mapBVT, &sm.full[st], kc * KC, g * 128);
             }
             __syncwarp();
         }
@@ -470,6 +511,7 @@ lorc_upproj_kernel(const __grid_constant__ CUtensorMap mapON, const __grid_const
         __syncwarp();
         if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
     } else {
+        grid_dep_wait();
         if (!mbar_wait(&sm.d_full, 0)) ok = false;
         if (ok) {
             tc_fence_after_sync();
@@ -603,11 +645,10 @@ cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView
         q.n_groups = n_groups; q.n_blk = n_blk; q.max_pos = d.max_pos;
         dim3 pgrid(n_groups, cv.batch);
         if (d.n_q_heads == 32)
-            lorc_prob_kernel<32><<<pgrid, 256, 0, st>>>(q);
+            e = lorc_launch_dependent(lorc_prob_kernel<32>, pgrid, dim3(256), 0, st, q);
         else
-            lorc_prob_kernel<64><<<pgrid, 256, 0, st>>>(q);
+            e = lorc_launch_dependent(lorc_prob_kernel<64>, pgrid, dim3(256), 0, st, q);
         *launches += 1;
-        e = cudaGetLastError();
         if (e != cudaSuccess) return e;
 
         Pv2Params p;
@@ -618,11 +659,10 @@ cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView
         p.page_size = cv.page_size; p.max_pages_per_seq = cv.max_pages_per_seq; p.n_pages = cv.n_pages;
         dim3 grid(n_blk, n_csplit, cv.batch);
         if (d.n_q_heads == 32)
-            lorc_pv2_kernel<32><<<grid, P_THREADS, sizeof(Pv2Smem<32>) + 1024, st>>>(mapCV, p);
+            e = lorc_launch_dependent(lorc_pv2_kernel<32>, grid, dim3(P_THREADS), sizeof(Pv2Smem<32>) + 1024, st, mapCV, p);
         else
-            lorc_pv2_kernel<64><<<grid, P_THREADS, sizeof(Pv2Smem<64>) + 1024, st>>>(mapCV, p);
+            e = lorc_launch_dependent(lorc_pv2_kernel<64>, grid, dim3(P_THREADS), sizeof(Pv2Smem<64>) + 1024, st, mapCV, p);
         *launches += 1;
-        e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
     LorcStageTimer timer(ctx, LORC_STAGE_COMBINE, st);
@@ -638,7 +678,7 @@ cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView
     u.out = out; u.status = ctx->status_dev;
     u.batch = cv.batch; u.H_q = d.n_q_heads; u.G = ctx->group; u.r_v = L.r_v;
     dim3 ugrid(d.n_kv_heads, (cv.batch * ctx->group + 127) / 128);
-    lorc_upproj_kernel<<<ugrid, U_THREADS, sizeof(UpSmem) + 1024, st>>>(mapON, mapBVT, u);
+    e = lorc_launch_dependent(lorc_upproj_kernel, ugrid, dim3(U_THREADS), sizeof(UpSmem) + 1024, st, mapON, mapBVT, u);
     *launches += 1;
-    return cudaGetLastError();
+    return e;
 }
