@@ -81,12 +81,13 @@ __device__ __forceinline__ bool decode_unit(const ScoreParams& p, int u, int ran
 // j = 32 jc + 8k + 2c + e (k = 0..3, e = 0..1): four tokens share every query operand the thread loads, and the four
 // lanes of equal r add their partial dots at the end.
 //
-// Float index of query head g, pair j, component `half` (0: first half of the head, 1: second) in qrot[][]: the four
-// c of equal (jc, k, e, half, g / 4) are neighbouring 16-byte pieces, one conflict-free shared-memory access.
+// Float index of query head g, pair j, component `half` (0: first half of the head, 1: second) in qrot[][].  One
+// 16-byte piece holds two heads x the thread's two adjacent pairs (e = j & 1), i.e. two packed-fp32 operands; the four
+// c of equal (kk, half, g / 2) are neighbouring pieces, one conflict-free shared-memory access.
 template <int G>
 __device__ __forceinline__ int qrot_index(int j, int half, int g) {
-    const int jc = j >> 5, k = (j >> 3) & 3, c = (j >> 1) & 3, e = j & 1;
-    return ((((((jc * 4 + k) * 2 + e) * 2 + half) * (G / 4) + (g >> 2)) * 4 + c) << 2) + (g & 3);
+    const int kk = j >> 3, c = (j >> 1) & 3, e = j & 1;
+    return ((((kk * 2 + half) * (G / 2) + (g >> 1)) * 4 + c) << 2) + ((g & 1) << 1) + e;
 }
 
 template <int G>
@@ -285,18 +286,21 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
 
             if (!mbar_wait(&sm.acc_full[buf], (uc >> 1) & 1)) { ok = false; break; }
             tc_fence_after_sync();
-            float acc[4][G];
+            // Packed fp32: every operation below acts on the thread's two adjacent rotary pairs (columns 2c, 2c + 1
+            // of the 8-column step) at once, which halves the instructions the epilogue issues.  acc2[m][g] holds the
+            // partial dots of the even and the odd pairs; they are added at the end.
+            uint64_t acc2[4][G];
 #pragma unroll
             for (int m = 0; m < 4; ++m)
 #pragma unroll
-                for (int g = 0; g < G; ++g) acc[m][g] = 0.f;
+                for (int g = 0; g < G; ++g) acc2[m][g] = 0ull;
             const uint32_t tbase = tmem + ((uint32_t)(quarter * 32) << 16) + buf * 256 + grp * 128;
-            const float4* q4 = reinterpret_cast<const float4*>(sm.qrot[qb][grp]) + c;
-            const float4* tr4 = &sm.trig[quarter * 8 + r][0];   // rotation of this thread's first token, quarter*32 + r
-            const float4* tw4 = &sm.trig[32][0] + c;            // rotation by 8 positions
+            const ulonglong2* q2 = reinterpret_cast<const ulonglong2*>(sm.qrot[qb][grp]) + c;
+            const ulonglong2* tr2 = reinterpret_cast<const ulonglong2*>(&sm.trig[quarter * 8 + r][0]);  // first token
+            const ulonglong2* tw2 = reinterpret_cast<const ulonglong2*>(&sm.trig[32][0]) + c;           // 8-position step
             const int tswz = (r & 1) << 2;                      // odd rows of the table swap 64-byte halves
-            // One 8-column step at a time, NOT unrolled: the loop body stays small enough for the instruction cache
-            // next to the scheduler, which the TMA and MMA warps on the same scheduler need as well.
+            const uint64_t minus1 = f2_pack(-1.f, -1.f);
+            // One 8-column step at a time, NOT unrolled: the loop body stays small.
 #pragma unroll 1
             for (int kk = 0; kk < 8; ++kk) {
                 uint32_t ra[2][4], rb[2][4];
@@ -305,40 +309,47 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
                     tmem_ld16x256_x1(tbase + ((uint32_t)(hf * 16) << 16) + kk * 8, ra[hf]);
                     tmem_ld16x256_x1(tbase + ((uint32_t)(hf * 16) << 16) + 64 + kk * 8, rb[hf]);
                 }
-                // (cos, sin) of this thread's first token for its two rotary pairs, and of the 8-position step that
-                // leads to its other three tokens (r + 8, r + 16, r + 24): angle addition instead of a table row per
-                // token
-                const float4 t0 = tr4[(kk * 4 + c) ^ tswz];
-                const float4 tw = tw4[kk * 4];
+                // (cos, -sin) of this thread's first token for its two rotary pairs, and (cos, sin) of the 8-position
+                // step that leads to its other three tokens (r + 8, r + 16, r + 24): angle addition instead of a table
+                // row per token
+                const ulonglong2 t0 = tr2[(kk * 4 + c) ^ tswz];
+                const ulonglong2 tw = tw2[kk * 4];
+                uint64_t cs = t0.x, ns = t0.y;                 // (cos_e0, cos_e1), (-sin_e0, -sin_e1)
+                const uint64_t wc = tw.x, ws = tw.y, nws = f2_mul(tw.y, minus1);
+                uint64_t qa[G], qbv[G];
+#pragma unroll
+                for (int gp = 0; gp < G / 2; ++gp) {
+                    const ulonglong2 x = q2[((kk * 2 + 0) * (G / 2) + gp) * 4];
+                    const ulonglong2 y = q2[((kk * 2 + 1) * (G / 2) + gp) * 4];
+                    qa[2 * gp] = x.x; qa[2 * gp + 1] = x.y;
+                    qbv[2 * gp] = y.x; qbv[2 * gp + 1] = y.y;
+                }
                 tmem_wait_ld();
 #pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    float qa[G], qbv[G];
+                for (int m = 0; m < 4; ++m) {
+                    const uint64_t a = f2_pack(__uint_as_float(ra[m >> 1][2 * (m & 1)]), __uint_as_float(ra[m >> 1][2 * (m & 1) + 1]));
+                    const uint64_t b = f2_pack(__uint_as_float(rb[m >> 1][2 * (m & 1)]), __uint_as_float(rb[m >> 1][2 * (m & 1) + 1]));
+                    const uint64_t na = f2_mul(a, minus1);
+                    const uint64_t ka = f2_fma(b, ns, f2_mul(a, cs));       // a cos - b sin
+                    const uint64_t kb = f2_fma(b, cs, f2_mul(na, ns));      // a sin + b cos
 #pragma unroll
-                    for (int g4 = 0; g4 < G / 4; ++g4) {
-                        const float4 x = q4[(((kk * 2 + e) * 2 + 0) * (G / 4) + g4) * 4];
-                        const float4 y = q4[(((kk * 2 + e) * 2 + 1) * (G / 4) + g4) * 4];
-                        qa[g4 * 4 + 0] = x.x; qa[g4 * 4 + 1] = x.y; qa[g4 * 4 + 2] = x.z; qa[g4 * 4 + 3] = x.w;
-                        qbv[g4 * 4 + 0] = y.x; qbv[g4 * 4 + 1] = y.y; qbv[g4 * 4 + 2] = y.z; qbv[g4 * 4 + 3] = y.w;
-                    }
-                    float cs = e ? t0.z : t0.x, sn = e ? t0.w : t0.y;
-                    const float wc = e ? tw.z : tw.x, ws = e ? tw.w : tw.y;
-#pragma unroll
-                    for (int m = 0; m < 4; ++m) {
-                        const float a = __uint_as_float(ra[m >> 1][2 * (m & 1) + e]);
-                        const float b = __uint_as_float(rb[m >> 1][2 * (m & 1) + e]);
-                        const float ka = a * cs - b * sn;
-                        const float kb = a * sn + b * cs;
-#pragma unroll
-                        for (int g = 0; g < G; ++g) acc[m][g] = fmaf(qbv[g], kb, fmaf(qa[g], ka, acc[m][g]));
-                        if (m < 3) {
-                            const float nc = cs * wc - sn * ws;
-                            sn = fmaf(cs, ws, sn * wc);
-                            cs = nc;
-                        }
+                    for (int g = 0; g < G; ++g) acc2[m][g] = f2_fma(qbv[g], kb, f2_fma(qa[g], ka, acc2[m][g]));
+                    if (m < 3) {
+                        const uint64_t nc = f2_fma(ns, ws, f2_mul(cs, wc));   // cos cos' - sin sin'
+                        ns = f2_fma(ns, wc, f2_mul(cs, nws));                 // -(cos sin' + sin cos')
+                        cs = nc;
                     }
                 }
             }
+            float acc[4][G];
+#pragma unroll
+            for (int m = 0; m < 4; ++m)
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    float x, y;
+                    f2_unpack(acc2[m][g], x, y);
+                    acc[m][g] = x + y;
+                }
             tc_fence_before_sync();
             mbar_arrive_cluster(lead_acc_empty[buf]);
             // add the four lanes' partial dots; lane c ends with the heads g = 4i + c
@@ -392,7 +403,7 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
 
 // Constant in-tile rotation table in the layout the score kernel keeps in shared memory: 33 rows of 32 pieces of
 // 16 bytes.  Row 8 q + r (q < 4, r < 8) holds (cos, sin)(t theta_j) for the token t = 32 q + r, piece
-// (j / 2) ^ (4 (r & 1)) = (cos_j, sin_j, cos_j+1, sin_j+1) for even j (the swap of 64-byte halves on odd rows spreads
+// (j / 2) ^ (4 (r & 1)) = (cos_j, cos_j+1, -sin_j, -sin_j+1) for even j (the swap of 64-byte halves on odd rows spreads
 // the epilogue's accesses over all banks); row 32 holds the same for a step of 8 positions, unswizzled.  The other
 // tokens of a tile follow by angle addition: t + 8 m.
 __global__ void rope_tile_kernel(float2* out, double theta) {
@@ -404,7 +415,10 @@ __global__ void rope_tile_kernel(float2* out, double theta) {
     double inv = pow(theta, -(double)j / 64.0);
     double sn, cs;
     sincos((double)t * inv, &sn, &cs);
-    out[(row * 32 + ((j >> 1) ^ swz)) * 2 + (j & 1)] = make_float2((float)cs, (float)sn);
+    // piece = (cos_j, cos_j+1, -sin_j, -sin_j+1) in the token rows, (cos, cos, +sin, +sin) in the step row
+    float* piece = reinterpret_cast<float*>(out) + (row * 32 + ((j >> 1) ^ swz)) * 4;
+    piece[j & 1] = (float)cs;
+    piece[2 + (j & 1)] = row < 32 ? -(float)sn : (float)sn;
 }
 
 }  // namespace
