@@ -37,6 +37,7 @@ constexpr float LOG2E = 1.4426950408889634f;
 constexpr int S_STAGES = 6;
 constexpr int S_THREADS = 320;       // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
 constexpr int S_EPI = 256;
+constexpr int S_LENS = 96;
 
 struct ScoreSmem {
     bf16 A[S_STAGES][TILE * KC];          // latent slice  [128 tokens][64]       16 KiB
@@ -45,6 +46,7 @@ struct ScoreSmem {
     float qrot[2][2][1024];               // [buffer][head of pair][rotated, scaled query; see qrot_index]    16 KiB
     uint64_t full[S_STAGES], empty[S_STAGES], acc_full[2], acc_empty[2], trig_full;
     uint32_t tmem_base;
+    int32_t lens[S_LENS];                 // sequence lengths of the first S_LENS sequences (the rest are read from global)
 };
 
 struct ScoreParams {
@@ -66,13 +68,14 @@ struct Unit {
 
 // Unit `u` of the pair: (sequence, tile pair, KV-head pair).  Valid when the pair's first tile starts inside the
 // sequence; the second CTA's tile may lie past the end (its rows are then masked or not written at all).
-__device__ __forceinline__ bool decode_unit(const ScoreParams& p, int u, int rank, Unit& un) {
+__device__ __forceinline__ bool decode_unit(const ScoreParams& p, const int32_t* lens_sm, int u, int rank, Unit& un) {
     un.hp = u % p.n_hp;
     int r = u / p.n_hp;
     const int tp = r % p.tile_pairs;
     un.s = r / p.tile_pairs;
     un.tile = 2 * tp + rank;
-    un.len = p.seq_lens[un.s];
+    // a shared-memory copy spares every role a global round trip at each unit boundary
+    un.len = un.s < S_LENS ? lens_sm[un.s] : p.seq_lens[un.s];
     return un.len > 0 && un.len <= p.max_pos && 2 * tp * TILE < un.len;
 }
 
@@ -122,6 +125,7 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
     // Everything above may overlap the tail of the previous kernel in the stream; inputs are read, results written
     // and tensor memory claimed only once that kernel has completed.
     grid_dep_wait();
+    for (int i = tid; i < S_LENS && i < p.batch; i += S_THREADS) sm.lens[i] = p.seq_lens[i];
     if (warp == 1) {
         tmem_alloc_pair(&sm.tmem_base, 512);
         tmem_relinquish_pair();
@@ -150,7 +154,7 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
             bool ok = true;
             for (int u = pair_id; u < total_units && ok; u += n_pairs) {
                 Unit un;
-                if (!decode_unit(p, u, rank, un)) continue;
+                if (!decode_unit(p, sm.lens, u, rank, un)) continue;
                 const int row0 = un.tile * TILE, brow = un.hp * 256 + b_row;
                 for (int x = 0; x < nkc * KC; x += KC) {
                     if (!mbar_wait_addr(empty0 + st * 8, par)) { ok = false; break; }
@@ -203,7 +207,7 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
             bool ok = true;
             for (int u = pair_id; u < total_units && ok; u += n_pairs) {
                 Unit un;
-                if (!decode_unit(p, u, rank, un)) continue;
+                if (!decode_unit(p, sm.lens, u, rank, un)) continue;
                 const int buf = uc & 1;
                 if (!mbar_wait(&sm.acc_empty[buf], ((uc >> 1) & 1) ^ 1)) { ok = false; break; }
                 tc_fence_after_sync();
@@ -264,7 +268,7 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
         };
         Unit un;
         int u = pair_id;
-        while (u < total_units && !decode_unit(p, u, rank, un)) u += n_pairs;
+        while (u < total_units && !decode_unit(p, sm.lens, u, rank, un)) u += n_pairs;
         if (u < total_units) fetch_query(un);
         while (u < total_units && ok) {
             const int buf = uc & 1, qb = uc & 1;
@@ -281,7 +285,7 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
             // next unit of this pair
             Unit un_next;
             int u_next = u + n_pairs;
-            while (u_next < total_units && !decode_unit(p, u_next, rank, un_next)) u_next += n_pairs;
+            while (u_next < total_units && !decode_unit(p, sm.lens, u_next, rank, un_next)) u_next += n_pairs;
             if (u_next < total_units) fetch_query(un_next);
 
             if (!mbar_wait(&sm.acc_full[buf], (uc >> 1) & 1)) { ok = false; break; }
