@@ -249,8 +249,9 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
         bool ok = mbar_wait(&sm.trig_full, 0);
         const uint32_t lead_acc_empty[2] = {mapa_shared(smem_u32(&sm.acc_empty[0]), 0),
                                             mapa_shared(smem_u32(&sm.acc_empty[1]), 0)};
-        // The query of the NEXT unit is fetched while this unit's accumulators are processed.
-        float q_a[QL], q_b[QL];
+        // The query of the NEXT unit is fetched while this unit's accumulators are processed: the loads below are
+        // only issued here (raw bits, volatile asm), nothing touches their results before the next unit's rotation.
+        uint16_t q_a[QL], q_b[QL];
         float2 q_cs[QL];
         auto fetch_query = [&](const Unit& un) {
             // query position relative to the tile start (a tile wholly past the sequence is masked anyway)
@@ -261,9 +262,10 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
                 const int hh = idx >> 6, j = idx & 63;
                 const int h = un.hp * 2 * G + hh;
                 const bf16* qp = p.q + ((long long)un.s * p.H_q + h) * 128;
-                q_cs[i] = p.rope_table[(long long)delta * 64 + j];
-                q_a[i] = __bfloat162float(qp[j]);
-                q_b[i] = __bfloat162float(qp[j + 64]);
+                const float2* cp = p.rope_table + (long long)delta * 64 + j;
+                asm volatile("ld.global.nc.v2.f32 {%0, %1}, [%2];" : "=f"(q_cs[i].x), "=f"(q_cs[i].y) : "l"(cp));
+                asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(q_a[i]) : "l"(qp + j));
+                asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(q_b[i]) : "l"(qp + j + 64));
             }
         };
         Unit un;
@@ -278,8 +280,9 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
                 const int idx = te + i * S_EPI;
                 const int hh = idx >> 6, j = idx & 63;
                 const int hip = hh / G, g = hh - hip * G;
-                sm.qrot[qb][hip][qrot_index<G>(j, 0, g)] = (q_a[i] * q_cs[i].x - q_b[i] * q_cs[i].y) * scale;
-                sm.qrot[qb][hip][qrot_index<G>(j, 1, g)] = (q_a[i] * q_cs[i].y + q_b[i] * q_cs[i].x) * scale;
+                const float qa_ = __uint_as_float((uint32_t)q_a[i] << 16), qb_ = __uint_as_float((uint32_t)q_b[i] << 16);
+                sm.qrot[qb][hip][qrot_index<G>(j, 0, g)] = (qa_ * q_cs[i].x - qb_ * q_cs[i].y) * scale;
+                sm.qrot[qb][hip][qrot_index<G>(j, 1, g)] = (qa_ * q_cs[i].y + qb_ * q_cs[i].x) * scale;
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");
             // next unit of this pair
