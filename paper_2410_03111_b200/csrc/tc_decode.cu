@@ -284,6 +284,7 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
                 sm.qrot[qb][hip][qrot_index<G>(j, 0, g)] = (qa_ * q_cs[i].x - qb_ * q_cs[i].y) * scale;
                 sm.qrot[qb][hip][qrot_index<G>(j, 1, g)] = (qa_ * q_cs[i].y + qb_ * q_cs[i].x) * scale;
             }
+            __syncwarp();   // a named barrier counts a warp once only if the warp arrives converged
             asm volatile("bar.sync 1, 256;" ::: "memory");
             // next unit of this pair
             Unit un_next;

@@ -346,6 +346,7 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
             float L = 0.f;
             for (int g = part; g < p.n_groups; g += PARTS) L += __ldg(lp + (long long)g * p.H_q);
             sm.red[part][h] = L;
+            __syncwarp();   // a named barrier counts a warp once only if the warp arrives converged
             asm volatile("bar.sync 2, 128;" ::: "memory");
             if (t < HQ) {
                 float Ls = 0.f;
@@ -381,8 +382,10 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
 #pragma unroll
             for (int h = 0; h < HQ; ++h) op[(long long)h * r_pad] = acc[h];
             __threadfence();
+            __syncwarp();   // a named barrier counts a warp once only if the warp arrives converged
             asm volatile("bar.sync 2, 128;" ::: "memory");
             if (t == 0) sm.last = atomicAdd(p.done + s * p.n_blk + blk, 1) == p.n_csplit - 1;
+            __syncwarp();   // a named barrier counts a warp once only if the warp arrives converged
             asm volatile("bar.sync 2, 128;" ::: "memory");
             finish = sm.last != 0;
             if (finish) {
@@ -396,6 +399,7 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
                 }
             }
         } else {
+            __syncwarp();   // a named barrier counts a warp once only if the warp arrives converged
             asm volatile("bar.sync 2, 128;" ::: "memory");     // l_inv is complete
         }
         if (finish) {
