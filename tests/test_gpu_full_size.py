@@ -90,3 +90,48 @@ def test_sampled_outputs_at_full_size(name, n_layers, samples):
         assert O.rel_l2_rows(got, want) <= TOL, (name, l, s, O.rel_l2_rows(got, want))
     del wl
     torch.cuda.empty_cache()
+
+
+RAGGED = ["cfg5_ragged_r384", "cfg5_ragged_r1024"]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("name", RAGGED)
+def test_ragged_paged_batch_at_full_size(name):
+    """64 sequences of 512 ... 16384 tokens in 64-token pages scattered over the pool: the shortest, the longest and
+    two more sequences against the oracle, which reads the same seeded cache rows through the same page table."""
+    import torch
+    from workloads import device as wdev
+    L = helpers.lib()
+    shape = synth.CONFIGS[name]
+    device = torch.device("cuda", 0)
+    r = shape.ranks[0]
+    prob = helpers.Problem(shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.d_head, r, r, theta=shape.rope_theta,
+                           p=shape.sigma_p)
+    lens = synth.ragged_lengths(shape.batch, shape.ragged[0], shape.ragged[1])
+    sess = helpers.Session(prob, int(lens.max()) + 64, shape.batch)
+    cache, k, v, sl, ptd, pt = helpers.paged_cache(sess, shape.batch, lens, shape.page_size, order_seed=11)
+    k.copy_(wdev.latents(tuple(k.shape), shape.sigma_p, 0, "k", device))
+    v.copy_(wdev.latents(tuple(v.shape), shape.sigma_p, 0, "v", device))
+    q = wdev.queries((shape.batch, shape.n_q_heads, shape.d_head), 0, 0, device, 8.0)
+    out = torch.zeros(shape.batch, shape.n_q_heads, shape.d_head, dtype=torch.bfloat16, device=device)
+    L.lorc_decode_attn(sess.ctx, 0, cache, q, out)
+    torch.cuda.synchronize()
+    assert L.lorc_sync_status(sess.ctx) == 0, L.lorc_last_error(sess.ctx)
+    assert L.lorc_last_path(sess.ctx) == 2
+    got_all = _f64(out)
+    assert np.all(np.isfinite(got_all))
+    order = np.argsort(lens)
+    picks = [int(order[0]), int(order[-1]), int(order[len(order) // 3]), int(order[2 * len(order) // 3])]
+    ps = shape.page_size
+    for s in picks:
+        n = int(lens[s])
+        pages = torch.tensor(pt[s, :(n + ps - 1) // ps].astype(np.int64), device=device)
+        ck = _f64(k[pages].reshape(-1, r)[:n])
+        cv = _f64(v[pages].reshape(-1, r)[:n])
+        want = O.decode_attn_latent(ck, cv, prob.B_k, prob.B_v, _f64(q[s]), shape.n_kv_heads, shape.rope_theta)
+        err = O.rel_l2_rows(got_all[s], want)
+        assert err <= TOL, (name, s, n, err)
+    sess.close()
+    del k, v
+    torch.cuda.empty_cache()

@@ -12,7 +12,7 @@ import torch
 
 from .synth import BASE_SEED
 
-_TAGS = {"U": 1, "V": 2, "X": 3, "Q": 4}
+_TAGS = {"U": 1, "V": 2, "X": 3, "Q": 4, "C": 5}
 
 
 def _gen(device, *key):
@@ -52,3 +52,13 @@ def queries(shape, layer, step, device, scale=1.0):
     """q ~ scale * N(0,1) in bf16; shape [batch, H_q, d_h]."""
     g = _gen(device, layer, step, _TAGS["Q"])
     return (scale * torch.randn(*shape, generator=g, device=device, dtype=torch.float32)).to(torch.bfloat16)
+
+
+def latents(shape, p, layer, which, device):
+    """Synthetic cache rows for tests that start from a filled cache: coordinate i ~ N(0, i^-2p) in bf16, the
+    distribution the rows have when the hidden states are N(0, I) and the spectrum is i^-p; `shape` ends with r."""
+    w = {"k": 0, "v": 1}[which]
+    g = _gen(device, layer, w, _TAGS["C"])
+    r = shape[-1]
+    sigma = torch.arange(1, r + 1, device=device, dtype=torch.float32) ** (-float(p))
+    return (torch.randn(*shape, generator=g, device=device, dtype=torch.float32) * sigma).to(torch.bfloat16)
