@@ -43,22 +43,11 @@ __device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
 
-// D (+)= A . B over the pair: M = 256 (128 rows in each CTA's TMEM), each CTA supplies its A rows and half of
-// the N rows of B at the same shared-memory offsets.  Issued by one thread of the leader CTA (rank 0).
-__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                                 uint32_t accumulate) {
-    asm volatile(
-        "{\n\t"
-        ".reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t"
-        "}\n" ::"r"(d_tmem),
-        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
 
-// The same MMA with the descriptors given as (low word, high word): the low word holds the start address (>> 4), so a
-// caller that walks through stages and k-steps only adds small constants to it.  Accumulating form.
+// D[256 x N] (+)= A[256 x 16] . B[N x 16]^T on a CTA pair (cta_group::2), issued by one thread of the leader CTA; each
+// CTA holds its 128 rows of A and its half of B in its own shared memory at the same offsets.  The descriptors are
+// given as (low word, high word): the low word holds the start address (>> 4), so a caller that walks through stages
+// and k-steps only adds small constants to it.  Accumulating form.
 __device__ __forceinline__ void tc_mma_bf16_pair_acc(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
                                                      uint32_t b_hi, uint32_t idesc) {
     asm volatile(
@@ -108,25 +97,11 @@ __device__ __forceinline__ void tc_commit_pair_addr(uint32_t bar_addr) {
 
 // TMA tiled loads into this CTA's shared memory, completion bytes counted on the mbarrier `bar_cluster_addr`
 // (a shared::cluster address, normally the leader's barrier).
-__device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int x,
-                                                 int y) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(smem_u32(smem_dst)), "l"(map), "r"(bar_cluster_addr), "r"(x), "r"(y)
-        : "memory");
-}
 __device__ __forceinline__ void tma_load_2d_pair_addr(uint32_t smem_dst, const CUtensorMap* map, uint32_t bar_cluster_addr,
                                                       int x, int y) {
     asm volatile(
         "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(smem_dst), "l"(map), "r"(bar_cluster_addr), "r"(x), "r"(y)
-        : "memory");
-}
-__device__ __forceinline__ void tma_load_3d_pair(void* smem_dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int x,
-                                                 int y, int z) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(smem_u32(smem_dst)), "l"(map), "r"(bar_cluster_addr), "r"(x), "r"(y), "r"(z)
         : "memory");
 }
 __device__ __forceinline__ void tma_load_3d_pair_addr(uint32_t smem_dst, const CUtensorMap* map, uint32_t bar_cluster_addr,

@@ -235,19 +235,10 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         : "memory");
 }
 
-// 16 lanes x 256 bits, four repeats along the columns: thread i of the warp receives, for repeat k = 0..3,
-//   r[4k + 0], r[4k + 1] = lane (i / 4),     columns 8k + 2 (i % 4) and + 1
-//   r[4k + 2], r[4k + 3] = lane (i / 4) + 8, the same two columns
-// (the accumulator fragment of an m16n8 MMA, repeated); the lane field of taddr names the first of the 16 lanes.
-__device__ __forceinline__ void tmem_ld16x256_x4(uint32_t taddr, uint32_t (&r)[16]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.16x256b.x4.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr)
-        : "memory");
-}
-
+// 16 lanes x 256 bits: thread i of the warp receives the accumulator fragment of an m16n8 MMA,
+//   r[0], r[1] = lane (i / 4),     columns 2 (i % 4) and + 1
+//   r[2], r[3] = lane (i / 4) + 8, the same two columns;
+// the lane field of taddr names the first of the 16 lanes.
 // Packed fp32 pairs (two independent fp32 operations per instruction; the results are ordinary IEEE fp32).
 __device__ __forceinline__ uint64_t f2_pack(float x, float y) {
     uint64_t r;
@@ -268,7 +259,6 @@ __device__ __forceinline__ uint64_t f2_mul(uint64_t a, uint64_t b) {
     return d;
 }
 
-// One repeat of the same shape: r[0], r[1] = lane (i / 4), columns 2 (i % 4) and + 1; r[2], r[3] = lane (i / 4) + 8.
 __device__ __forceinline__ void tmem_ld16x256_x1(uint32_t taddr, uint32_t (&r)[4]) {
     asm volatile("tcgen05.ld.sync.aligned.16x256b.x1.b32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
