@@ -44,13 +44,30 @@ append_mma_kernel(const bf16* __restrict__ x, const bf16* __restrict__ A_tiled, 
         const uint4* xb = reinterpret_cast<const uint4*>(x + (m0 + g + 8) * D + k_begin) + t;
         const uint4* wb = reinterpret_cast<const uint4*>(A_tiled) + ((long long)blockIdx.x * (D / 32) + k_begin / 32) * 32 + lane;
         const uint4 zero = make_uint4(0, 0, 0, 0);
-#pragma unroll 8
-        for (int kb = 0; kb < kspan / 32; ++kb) {
-            const uint4 w = __ldg(wb + kb * 32);
-            const uint4 lo = row_lo ? __ldg(xa + kb * 4) : zero;
-            const uint4 hi = row_hi ? __ldg(xb + kb * 4) : zero;
-            mma_bf16_16816(c, lo.x, hi.x, lo.y, hi.y, w.x, w.y);
-            mma_bf16_16816(c, lo.z, hi.z, lo.w, hi.w, w.z, w.w);
+        // The factor comes from HBM and nothing else in the kernel takes long: up to 16 steps' worth of it (8 KiB per
+        // warp) is requested before the first MMA (volatile asm keeps the loads together, ahead of their uses).
+        const int steps = kspan / 32;
+        for (int kb0 = 0; kb0 < steps; kb0 += 16) {
+            uint4 w[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                w[i] = zero;
+                if (kb0 + i < steps) {
+                    const uint4* src = wb + (kb0 + i) * 32;
+                    asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(w[i].x), "=r"(w[i].y), "=r"(w[i].z), "=r"(w[i].w)
+                                 : "l"(src));
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                if (kb0 + i < steps) {
+                    const uint4 lo = row_lo ? __ldg(xa + (kb0 + i) * 4) : zero;
+                    const uint4 hi = row_hi ? __ldg(xb + (kb0 + i) * 4) : zero;
+                    mma_bf16_16816(c, lo.x, hi.x, lo.y, hi.y, w[i].x, w[i].y);
+                    mma_bf16_16816(c, lo.z, hi.z, lo.w, hi.w, w[i].z, w[i].w);
+                }
+            }
         }
     }
     red[warp][lane][0] = c[0];
