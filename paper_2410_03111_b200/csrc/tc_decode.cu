@@ -436,7 +436,7 @@ __global__ void rope_tile_kernel(float2* out, double theta) {
 // ------------------------------------------------------------------------------------------------
 struct LorcTcLayer {
     bool has_bkt = false;
-    CUtensorMap mapBKT, mapBVT;         // B_K^T in 64 x 128 swizzled boxes; B_V^T in 64 x 128 swizzled boxes
+    CUtensorMap mapBKT, mapBVT;         // B_K^T in 64 x 128 swizzled boxes; B_V^T in 64 x 32 swizzled boxes
     // cache maps are rebuilt only when the cache geometry or pointers change
     const void* k_ptr = nullptr;
     const void* v_ptr = nullptr;
@@ -553,7 +553,7 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
         uint32_t box[2] = {KC, 128};
         if (!lorc_make_tmap_bf16(&TL.mapBKT, L.B_kT, 2, dims, str, box)) return cudaErrorInvalidValue;
         uint64_t d2[2] = {(uint64_t)L.r_v, (uint64_t)ctx->n}, s2[1] = {(uint64_t)L.r_v * 2};
-        uint32_t b2[2] = {KC, 128};
+        uint32_t b2[2] = {KC, 32};          // the up-projection takes a quarter of a head's columns per CTA
         if (!lorc_make_tmap_bf16(&TL.mapBVT, L.B_vT, 2, d2, s2, b2)) return cudaErrorInvalidValue;
         TL.has_bkt = true;
     }

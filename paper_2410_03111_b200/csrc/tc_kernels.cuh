@@ -21,7 +21,7 @@ cudaError_t lorc_tc_append(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
 // Softmax + P.C_V and value up-projection (tc_pv.cu).  scores [b, H_q, n_pad] (log2 units) and
 // tmax [b, H_q, tiles, 4] (maxima of each 32-token quarter tile) come from the score kernel.
 // mapCV: C_V cache in 64-column x 128-row (or page-sized) swizzled boxes; mapBVT: B_V^T [n, r_v] in swizzled
-// boxes of 64 latent columns x 128 rows.  Launches the PV kernel and the up-projection kernel that writes `out`.
+// boxes of 64 latent columns x 32 rows.  Launches the PV kernel and the up-projection kernel that writes `out`.
 size_t lorc_tc_pv_scratch_bytes(const lorc_ctx* ctx, int batch, int max_seq_len);
 cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, const CUtensorMap& mapCV,
                               const CUtensorMap& mapBVT, const float* scores, const float* tmax, int n_pad, int tiles,

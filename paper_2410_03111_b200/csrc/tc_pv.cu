@@ -420,14 +420,16 @@ namespace {
 
 // ------------------------------------------------------------------------------------------------
 // value up-projection: out[(s, h), :] = o_norm[s, h, :] . B_V[:, g(h)], a plain TMA-fed tcgen05 GEMM.
-// grid (n_kv_heads, ceil(batch * G / 128)): 128 output rows (s, i) x 128 columns, K = r_v in slices of 64.
+// grid (n_kv_heads, ceil(batch * G / 128), 4): 128 output rows (s, i) x 32 of the head's 128 columns, K = r_v in
+// slices of 64.  (Splitting the columns gives four times the CTAs and small stages, so a whole rank is in flight.)
 // ------------------------------------------------------------------------------------------------
-constexpr int U_STAGES = 6;
+constexpr int U_STAGES = 10;         // 10 x 20 KiB: most ranks fit in one round of loads
 constexpr int U_THREADS = 192;
+constexpr int U_NCOL = 32;           // output columns per CTA (a quarter of a head)
 
 struct UpSmem {
     bf16 A[U_STAGES][128 * KC];           // o_norm rows [128 rows (s, i)][64 rho]
-    bf16 B[U_STAGES][128 * KC];           // B_V^T slice [128 columns j][64 rho]
+    bf16 B[U_STAGES][U_NCOL * KC];        // B_V^T slice [32 columns j][64 rho]
     uint64_t full[U_STAGES], empty[U_STAGES], d_full;
     uint32_t tmem_base;
 };
@@ -444,9 +446,10 @@ lorc_upproj_kernel(const __grid_constant__ CUtensorMap mapON, const __grid_const
     extern __shared__ uint8_t raw[];
     UpSmem& sm = *reinterpret_cast<UpSmem*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
-    const int g = blockIdx.x, chunk = blockIdx.y;
+    const int g = blockIdx.x, chunk = blockIdx.y, cq = blockIdx.z;     // KV head, block of 128 rows, column quarter
     const int nkc = (p.r_v + KC - 1) / KC;
     const int seqs_per_cta = 128 / p.G;
+    constexpr uint32_t STAGE_BYTES = (128 + U_NCOL) * KC * 2;
     if (tid == 0) {
         for (int i = 0; i < U_STAGES; ++i) {
             mbar_init(&sm.full[i], 1);
@@ -458,7 +461,7 @@ lorc_upproj_kernel(const __grid_constant__ CUtensorMap mapON, const __grid_const
         prefetch_tensormap(&mapBVT);
     }
     if (warp == 1) {
-        tmem_alloc(&sm.tmem_base, 128);
+        tmem_alloc(&sm.tmem_base, 32);
         tmem_relinquish();
     }
     tc_fence_before_sync();
@@ -474,8 +477,8 @@ lorc_upproj_kernel(const __grid_constant__ CUtensorMap mapON, const __grid_const
         const int npre = nkc < U_STAGES ? nkc : U_STAGES;
         if (elect_one()) {
             for (int kc = 0; kc < npre; ++kc) {
-                mbar_arrive_expect_tx(&sm.full[kc], 2 * 128 * KC * 2);
-                tma_load_2d(sm.B[kc], &mapBVT, &sm.full[kc], kc * KC, g * 128);
+                mbar_arrive_expect_tx(&sm.full[kc], STAGE_BYTES);
+                tma_load_2d(sm.B[kc], &mapBVT, &sm.full[kc], kc * KC, g * 128 + cq * U_NCOL);
             }
         }
         __syncwarp();
@@ -486,8 +489,8 @@ lorc_upproj_kernel(const __grid_constant__ CUtensorMap mapON, const __grid_const
             if (kc >= npre && !mbar_wait(&sm.empty[st], ((kc / U_STAGES) & 1) ^ 1)) { ok = false; break; }
             if (elect_one()) {
                 if (kc >= npre) {
-                    mbar_arrive_expect_tx(&sm.full[st], 2 * 128 * KC * 2);
-                    tma_load_2d(sm.B[st], &mapBVT, &sm.full[st], kc * KC, g * 128);
+                    mbar_arrive_expect_tx(&sm.full[st], STAGE_BYTES);
+                    tma_load_2d(sm.B[st], &mapBVT, &sm.full[st], kc * KC, g * 128 + cq * U_NCOL);
                 }
                 // rows (s, i): box of G heads x 128/G sequences (sequences past the batch read as zero)
                 tma_load_3d(sm.A[st], &mapON, &sm.full[st], kc * KC, g * p.G, chunk * seqs_per_cta);
@@ -496,7 +499,7 @@ lorc_upproj_kernel(const __grid_constant__ CUtensorMap mapON, const __grid_const
         }
         if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
     } else if (warp == 1) {
-        const uint32_t idesc = make_idesc_bf16(128, 128, 0, 0);
+        const uint32_t idesc = make_idesc_bf16(128, U_NCOL, 0, 0);
         for (int kc = 0; kc < nkc; ++kc) {
             const int st = kc % U_STAGES;
             if (!mbar_wait(&sm.full[st], (kc / U_STAGES) & 1)) { ok = false; break; }
@@ -523,13 +526,12 @@ lorc_upproj_kernel(const __grid_constant__ CUtensorMap mapON, const __grid_const
             const int quarter = warp % 4;
             const int row = quarter * 32 + lane;
             const int s = chunk * seqs_per_cta + row / p.G, h = g * p.G + row % p.G;
-#pragma unroll
-            for (int c0 = 0; c0 < 128; c0 += 32) {
+            {
                 uint32_t r[32];
-                tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + c0, r);
+                tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16), r);
                 tmem_wait_ld();
                 if (s < p.batch) {
-                    uint4* dst = reinterpret_cast<uint4*>(p.out + ((long long)s * p.H_q + h) * 128 + c0);
+                    uint4* dst = reinterpret_cast<uint4*>(p.out + ((long long)s * p.H_q + h) * 128 + cq * U_NCOL);
 #pragma unroll
                     for (int q4 = 0; q4 < 4; ++q4) {
                         uint32_t w[4];
@@ -548,7 +550,7 @@ lorc_upproj_kernel(const __grid_constant__ CUtensorMap mapON, const __grid_const
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem, 128);
+    if (warp == 1) tmem_dealloc(tmem, 32);
 }
 
 // Column blocks and context shares of one PV launch: two CTAs fit on an SM, so aim at filling those slots once.
@@ -681,7 +683,7 @@ cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView
     UpParams u;
     u.out = out; u.status = ctx->status_dev;
     u.batch = cv.batch; u.H_q = d.n_q_heads; u.G = ctx->group; u.r_v = L.r_v;
-    dim3 ugrid(d.n_kv_heads, (cv.batch * ctx->group + 127) / 128);
+    dim3 ugrid(d.n_kv_heads, (cv.batch * ctx->group + 127) / 128, 128 / U_NCOL);
     e = lorc_launch_dependent(lorc_upproj_kernel, ugrid, dim3(U_THREADS), sizeof(UpSmem) + 1024, st, mapON, mapBVT, u);
     *launches += 1;
     return e;
