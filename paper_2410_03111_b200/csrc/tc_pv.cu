@@ -27,7 +27,7 @@ namespace {
 
 constexpr int TILE = 128;
 constexpr int KC = 64;
-constexpr int P_STAGES = 2;          // 2 x 40 KiB: two CTAs fit on an SM
+constexpr int P_STAGES = 4;          // 4 x 40 KiB (48 KiB with 64 query heads): one CTA per SM, 160 KiB in flight
 constexpr int P_THREADS = 192;       // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
 
 // read-only global load that the compiler keeps in program order with the other volatile asm of this file
@@ -199,7 +199,7 @@ struct Pv2Params {
 };
 
 template <int HQ>
-__global__ void __launch_bounds__(P_THREADS, 2)
+__global__ void __launch_bounds__(P_THREADS, 1)
 lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
     extern __shared__ uint8_t raw[];
     typedef Pv2Smem<HQ> S;
@@ -553,12 +553,14 @@ lorc_upproj_kernel(const __grid_constant__ CUtensorMap mapON, const __grid_const
     if (warp == 1) tmem_dealloc(tmem, 32);
 }
 
-// Column blocks and context shares of one PV launch: two CTAs fit on an SM, so aim at filling those slots once.
+// Column blocks and context shares of one PV launch: one CTA per SM, and as few context shares as fill the SMs once
+// (a CTA with four stages in flight pulls its share of the HBM bandwidth alone; fewer shares mean longer streams per
+// CTA and, at one share, no share reduction at all).
 void pv_plan(const lorc_ctx* ctx, const LorcLayer& L, int batch, int max_seq_len, int n_splits_hint, int* n_blk,
              int* n_csplit) {
     const int tiles = (max_seq_len + TILE - 1) / TILE;
     *n_blk = (L.r_v + 127) / 128;
-    const int slots = 2 * ctx->sm_count;
+    const int slots = ctx->sm_count;
     int cs = n_splits_hint > 0 ? n_splits_hint : slots / (batch * *n_blk);
     if (cs > tiles) cs = tiles;
     if (cs > 64) cs = 64;
