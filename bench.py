@@ -42,6 +42,8 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--ref-budget", type=float, default=6.0,
                     help="--impl reference: seconds of oracle time sampled per step")
+    ap.add_argument("--full-rank", action="store_true",
+                    help="time the uncompressed reference mode (ordinary KV cache, no latents) instead of the latent path")
     ap.add_argument("--no-graph", action="store_true", help="launch call by call instead of replaying a CUDA graph")
     ap.add_argument("--stages", action="store_true",
                     help="call-by-call launches with per-kernel CUDA events; adds a 'stages' object (ms per step)")
@@ -134,7 +136,7 @@ def algorithmic_counts(shape, ranks, batch, n_ctx):
 class Workload:
     """Factors, prefilled latent caches and per-step inputs of one configuration on one GPU."""
 
-    def __init__(self, L, shape, n_layers, total_steps, device, flags):
+    def __init__(self, L, shape, n_layers, total_steps, device, flags, full_rank=False):
         import torch
         from paper_2410_03111_b200 import host
         from workloads import device as wdev
@@ -153,9 +155,16 @@ class Workload:
             r = self.ranks[l]
             Uk, sk, Vk = wdev.weight_generators(shape.d_model, shape.n, shape.sigma_p, l, "k", device)
             Uv, sv, Vv = wdev.weight_generators(shape.d_model, shape.n, shape.sigma_p, l, "v", device)
-            Ak, Bk = host.factors_from_svd(Uk, sk, Vk, r)
-            Av, Bv = host.factors_from_svd(Uv, sv, Vv, r)
-            L.lorc_load_factors(self.ctx, l, L.LORC_MODE_LATENT, r, r, Ak, Bk, Av, Bv)
+            if full_rank:
+                # the uncompressed mode takes the dense weights; its cache rows are whole keys and values
+                Ak, Av = host.dense_weight(Uk, sk, Vk), host.dense_weight(Uv, sv, Vv)
+                Bk = Bv = None
+                L.lorc_load_factors(self.ctx, l, L.LORC_MODE_FULL, 0, 0, Ak, None, Av, None)
+                r = shape.n
+            else:
+                Ak, Bk = host.factors_from_svd(Uk, sk, Vk, r)
+                Av, Bv = host.factors_from_svd(Uv, sv, Vv, r)
+                L.lorc_load_factors(self.ctx, l, L.LORC_MODE_LATENT, r, r, Ak, Bk, Av, Bv)
             k = torch.zeros(b, self.n_max, r, dtype=torch.bfloat16, device=device)
             v = torch.zeros(b, self.n_max, r, dtype=torch.bfloat16, device=device)
             self.keep.append((k, v))
@@ -367,7 +376,7 @@ def main():
         args.no_graph = True
     e2e_steps = 0 if args.no_e2e else max(2, min(args.steps, 8))
     total_steps = args.warmup + args.steps + e2e_steps + 4
-    wl = Workload(L, shape, n_layers, total_steps, device, flags)
+    wl = Workload(L, shape, n_layers, total_steps, device, flags, full_rank=args.full_rank)
     b = shape.batch
 
     def barrier():
@@ -426,7 +435,7 @@ def main():
     # the dominant kernel alone: the same attention calls again, launched one by one with a CUDA event before and
     # after every kernel on the launching stream (the library's own stage bracketing)
     score_prof = None
-    if not args.debug_fp32:
+    if not args.debug_fp32 and not args.full_rank:
         L.lorc_profile_read(wl.ctx)
         L.lorc_profile_enable(wl.ctx, True)
         prof_reps = max(3, min(args.steps, 8))
@@ -470,6 +479,11 @@ def main():
         value = whole_job_rate(b, args.steps, world, ms * 1e-3)
         n_ctx_mid = n_ctx_start + args.steps      # context the attention-only pass sees
         flops, byts = algorithmic_counts(shape, wl.ranks, b, n_ctx_mid)
+        if args.full_rank:
+            # uncompressed mode: scores and PV over whole keys and values, 2 n bf16 numbers read per token
+            n, Hq, dh = shape.n, shape.n_q_heads, shape.d_head
+            flops = len(wl.ranks) * b * n_ctx_mid * 4.0 * Hq * dh
+            byts = len(wl.ranks) * (b * n_ctx_mid * 2.0 * 2.0 * n + 4.0 * b * Hq * dh)
         attn_ms_step = attn_ms / args.steps
         t_tc = flops / (peaks["bf16_tflops_sustained"] * 1e12)
         t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
@@ -482,7 +496,8 @@ def main():
                        "ranks_mean": sum(wl.ranks) / len(wl.ranks), "l2": "inputs larger than L2 (latent cache %.1f GB)" %
                        (sum(2 * 2 * r for r in wl.ranks) * b * n_ctx_mid / 1e9),
                        "kernel_path": {1: "plain fp32 CUDA-core", 2: "tcgen05"}.get(path, str(path)),
-                       "replicas": world, "launch": "cuda graph per step" if use_graph else "call by call"},
+                       "replicas": world, "launch": "cuda graph per step" if use_graph else "call by call",
+                       "mode": "full-rank reference (uncompressed KV cache)" if args.full_rank else "latent"},
             "decode_attn": {"ms_per_step": attn_ms_step, "tokens_per_s": b * world / (attn_ms_step * 1e-3),
                             "roofline_ms": max(t_tc, t_hbm) * 1e3, "frac_of_roofline": max(t_tc, t_hbm) * 1e3 / attn_ms_step,
                             "hbm_gbs": byts / (attn_ms_step * 1e-3) / 1e9},
@@ -510,8 +525,12 @@ def main():
                                 "timing": "CUDA events around every launch, call-by-call pass after the timed steps",
                                 "stage_ms_per_step": score_prof[2]}
         else:
-            line["roofline"] = {"bound": "alu", "achieved": achieved, "peak": None, "unit": "TFLOP/s", "frac": None,
-                                "traffic": None, "kernel": "plain fp32 CUDA-core kernels (debug path)"}
+            gbs = byts / (attn_ms_step * 1e-3) / 1e9
+            line["roofline"] = {"bound": "hbm" if args.full_rank else "alu", "achieved": gbs if args.full_rank else achieved,
+                                "peak": peaks["hbm_gbs"] if args.full_rank else None,
+                                "unit": "GB/s" if args.full_rank else "TFLOP/s",
+                                "frac": gbs / peaks["hbm_gbs"] if args.full_rank else None, "traffic": None,
+                                "kernel": "plain fp32 CUDA-core kernels (reference mode / debug path), whole lorc_decode_attn"}
         if stages:
             line["stages"] = stages
         if e2e:
