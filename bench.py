@@ -40,8 +40,9 @@ def parse_args():
     ap.add_argument("--debug-fp32", action="store_true", help="time the plain fp32 kernels")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--ref-budget", type=float, default=6.0,
-                    help="--impl reference: seconds of oracle time sampled per step")
+    ap.add_argument("--ref-budget", type=float, default=None,
+                    help="--impl reference: seconds of oracle time sampled per step "
+                         "(default: 100 s shared by all steps, at most 6 s each)")
     ap.add_argument("--full-rank", action="store_true",
                     help="time the uncompressed reference mode (ordinary KV cache, no latents) instead of the latent path")
     ap.add_argument("--no-graph", action="store_true", help="launch call by call instead of replaying a CUDA graph")
@@ -362,8 +363,9 @@ def run_reference(args, shape, n_layers):
     """The oracle as the reference arm: each step times a bounded sample and scales it."""
     vals = []
     per_rank, desc, threads = None, "", 1
+    budget = args.ref_budget if args.ref_budget else min(6.0, 100.0 / max(1, args.warmup + args.steps))
     for i in range(args.warmup + args.steps):
-        per_rank, desc, threads, units = oracle_sample(shape, n_layers, budget_s=args.ref_budget,
+        per_rank, desc, threads, units = oracle_sample(shape, n_layers, budget_s=budget,
                                                        layers=[0, n_layers - 1] if n_layers > 1 else [0])
         step_s = per_rank * sum(shape.ranks[:n_layers]) * shape.batch
         if i >= args.warmup:
