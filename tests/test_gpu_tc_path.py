@@ -61,6 +61,23 @@ def test_tc_decode_contiguous(r_k, r_v, lens):
     sess.close()
 
 
+def test_tc_decode_large_batch_of_short_sequences():
+    """More sequences than the score kernel caches lengths for, several 128-row blocks of output rows in the value
+    up-projection, and contexts of one to three tiles."""
+    prob = _prob(96, 72)
+    b = 104
+    lens = [int(v) for v in synth.ragged_lengths(b, 1, 300, base_seed=77)]
+    n_max = max(lens) + 3
+    sess = H.Session(prob, max_pos=n_max, batch=b)
+    ck, cv = _latents(prob, lens, 20)
+    cache, k, v, sl = H.contiguous_cache(sess, b, n_max, lens, ck, cv)
+    q = synth.queries(b, GEOM["H_q"], GEOM["d_h"], 20, 3, 8.0).astype(np.float64)
+    got = H.host_f64(_run(sess, cache, q))
+    want = H.oracle_decode(prob, ck, cv, q)
+    assert O.rel_l2_rows(got, want) <= TOL
+    sess.close()
+
+
 def test_tc_decode_matches_plain_kernels_and_split_counts():
     import torch
     prob = _prob(160, 224, layer=21)
