@@ -60,12 +60,29 @@ append_mma_kernel(const bf16* __restrict__ x, const bf16* __restrict__ A_tiled, 
                 }
             }
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                if (kb0 + i < steps) {
-                    const uint4 lo = row_lo ? __ldg(xa + (kb0 + i) * 4) : zero;
-                    const uint4 hi = row_hi ? __ldg(xb + (kb0 + i) * 4) : zero;
-                    mma_bf16_16816(c, lo.x, hi.x, lo.y, hi.y, w[i].x, w[i].y);
-                    mma_bf16_16816(c, lo.z, hi.z, lo.w, hi.w, w[i].z, w[i].w);
+            for (int i0 = 0; i0 < 16; i0 += 8) {
+                uint4 lo[8], hi[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    lo[i] = zero;
+                    hi[i] = zero;
+                    if (kb0 + i0 + i < steps) {
+                        if (row_lo)
+                            asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];"
+                                         : "=r"(lo[i].x), "=r"(lo[i].y), "=r"(lo[i].z), "=r"(lo[i].w)
+                                         : "l"(xa + (kb0 + i0 + i) * 4));
+                        if (row_hi)
+                            asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];"
+                                         : "=r"(hi[i].x), "=r"(hi[i].y), "=r"(hi[i].z), "=r"(hi[i].w)
+                                         : "l"(xb + (kb0 + i0 + i) * 4));
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (kb0 + i0 + i < steps) {
+                        mma_bf16_16816(c, lo[i].x, hi[i].x, lo[i].y, hi[i].y, w[i0 + i].x, w[i0 + i].y);
+                        mma_bf16_16816(c, lo[i].z, hi[i].z, lo[i].w, hi[i].w, w[i0 + i].z, w[i0 + i].w);
+                    }
                 }
             }
         }
