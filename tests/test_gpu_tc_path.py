@@ -78,6 +78,27 @@ def test_tc_decode_large_batch_of_short_sequences():
     sess.close()
 
 
+def test_tc_decode_repeated_calls_are_bit_identical():
+    """Back-to-back calls overlap their kernels' heads and tails (dependent launches), and the context shares of a
+    column block are added by whichever share finishes last: neither may show in the result."""
+    import torch
+    prob = _prob(256, 256)
+    lens = [1500, 700, 129]
+    b, n_max = len(lens), max(lens) + 3
+    sess = H.Session(prob, max_pos=n_max, batch=b)
+    ck, cv = _latents(prob, lens, 20)
+    cache, k, v, sl = H.contiguous_cache(sess, b, n_max, lens, ck, cv)
+    q = H.dev_bf16(synth.queries(b, GEOM["H_q"], GEOM["d_h"], 20, 5, 8.0).astype(np.float64))
+    outs = [torch.zeros(b, GEOM["H_q"], GEOM["d_h"], dtype=torch.bfloat16, device="cuda") for _ in range(24)]
+    for o in outs:                              # no synchronisation in between
+        sess.L.lorc_decode_attn(sess.ctx, 0, cache, q, o)
+    torch.cuda.synchronize()
+    assert sess.L.lorc_sync_status(sess.ctx) == 0, sess.L.lorc_last_error(sess.ctx)
+    for o in outs[1:]:
+        assert torch.equal(o, outs[0])
+    sess.close()
+
+
 def test_tc_decode_matches_plain_kernels_and_split_counts():
     import torch
     prob = _prob(160, 224, layer=21)
