@@ -59,7 +59,7 @@ __device__ __forceinline__ int prob_image_offset(int h, int tc) {
 
 // 256 threads: thread = (token of the tile, half of the heads).
 template <int HQ>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 3)
 lorc_prob_kernel(const ProbParams p) {
     constexpr int NH = HQ / 2;                        // heads per thread
     __shared__ float m_s[HQ];
