@@ -553,7 +553,7 @@ def main():
             "config": {"workload": shape.name, "layers": n_layers, "batch": b, "context": shape.context,
                        "ranks_mean": sum(wl.ranks) / len(wl.ranks), "l2": "inputs larger than L2 (latent cache %.1f GB)" %
                        (sum(2 * 2 * r for r in wl.ranks) * b * n_ctx_mid / 1e9),
-                       "kernel_path": {1: "plain fp32 CUDA-core", 2: "tcgen05"}.get(path, str(path)),
+                       "kernel_path": {1: "plain fp32 CUDA-core", 2: "tcgen05", 3: "mma.sync streaming kernel (uncompressed mode)"}.get(path, str(path)),
                        "replicas": world, "launch": "cuda graph per step" if use_graph else "call by call",
                        "mode": "full-rank reference (uncompressed KV cache)" if args.full_rank else "latent"},
             "decode_attn": {"ms_per_step": attn_ms_step, "tokens_per_s": b * world / (attn_ms_step * 1e-3),
@@ -588,7 +588,7 @@ def main():
                                 "peak": peaks["hbm_gbs"] if args.full_rank else None,
                                 "unit": "GB/s" if args.full_rank else "TFLOP/s",
                                 "frac": gbs / peaks["hbm_gbs"] if args.full_rank else None, "traffic": None,
-                                "kernel": "plain fp32 CUDA-core kernels (reference mode / debug path), whole lorc_decode_attn"}
+                                "kernel": "whole lorc_decode_attn (" + {1: "plain fp32 CUDA-core kernels", 3: "mma.sync streaming kernel + merge"}.get(path, str(path)) + ")"}
         if stages:
             line["stages"] = stages
         if e2e:

@@ -215,7 +215,8 @@ const char* lorc_last_error(const lorc_ctx* ctx);
 
 /* Which kernel family the last lorc_decode_attn / lorc_append call on this
  * context used: 0 = none yet, 1 = plain fp32 CUDA-core kernels, 2 = tensor-core
- * (tcgen05) kernels.  For tests and benchmarks. */
+ * (tcgen05) kernels of the latent mode, 3 = warp-level tensor-core (mma.sync) kernel of
+ * the uncompressed mode.  For tests and benchmarks. */
 int lorc_last_path(const lorc_ctx* ctx);
 
 /* Contexts created with LORC_FLAG_PROFILE record a CUDA event before and after every

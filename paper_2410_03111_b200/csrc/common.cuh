@@ -119,6 +119,11 @@ cudaError_t lorc_generic_build_rope_table(float2* table, int max_pos, int d_head
 cudaError_t lorc_generic_transpose(const bf16* in, bf16* out, int rows, int cols, cudaStream_t st);
 cudaError_t lorc_generic_append(const lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv,
                                 const bf16* x, int T, cudaStream_t st, int* launches);
+// Uncompressed mode, 128-wide heads, bf16 path: streaming decode kernel on mma.sync (full_decode.cu).  Leaves the same
+// per-split partial results as the plain kernel, for lorc_generic_combine.
+bool lorc_full_decode_supported(const lorc_ctx* ctx, const LorcLayer& L);
+cudaError_t lorc_full_decode(const lorc_ctx* ctx, const CacheView& cv, const bf16* q, int n_splits, float* part_ml,
+                             float* part_o, cudaStream_t st, int* launches);
 cudaError_t lorc_generic_decode(const lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv,
                                 const bf16* q, bf16* out, int n_splits, float* part_ml,
                                 float* part_o, cudaStream_t st, int* launches);

@@ -449,6 +449,15 @@ cudaError_t lorc_generic_decode(const lorc_ctx* ctx, const LorcLayer& L, const C
     const int G = ctx->group;
     const bool latent = (L.mode == LORC_MODE_LATENT);
     dim3 grid(n_splits, d.n_kv_heads, cv.batch);
+    if (lorc_full_decode_supported(ctx, L)) {
+        // uncompressed mode with 128-wide heads: the streaming kernel on the warp-level tensor cores
+        {
+            LorcStageTimer timer(ctx, LORC_STAGE_SCORE, st);
+            cudaError_t e = lorc_full_decode(ctx, cv, q, n_splits, part_ml, part_o, st, launches);
+            if (e != cudaSuccess) return e;
+        }
+        return lorc_generic_combine(ctx, L, cv.batch, n_splits, part_ml, part_o, out, st, launches);
+    }
     {
     LorcStageTimer timer(ctx, LORC_STAGE_SCORE, st);
 #define LAUNCH_DEC(DHV, LAT)                                                                      \

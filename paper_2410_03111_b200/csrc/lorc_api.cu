@@ -313,7 +313,7 @@ int lorc_decode_attn(lorc_ctx* ctx, int layer, const lorc_cache* cache, const vo
     float* part_o = (float*)((char*)ctx->ws + w.off_o);
     e = lorc_generic_decode(ctx, *L, cv, (const bf16*)q, (bf16*)out, S, part_ml, part_o, st, &launches);
     ctx->launches += launches;
-    ctx->last_path = 1;
+    ctx->last_path = lorc_full_decode_supported(ctx, *L) ? 3 : 1;
     if (e != cudaSuccess) return fail_cuda(ctx, e, "lorc_decode_attn");
     return LORC_OK;
 }

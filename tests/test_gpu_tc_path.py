@@ -197,3 +197,39 @@ def test_tc_append_then_decode_chain_and_host_entry():
     want = H.oracle_decode(prob, ck, cv, q.astype(np.float64))
     assert O.rel_l2_rows(H.host_f64(oh), want) <= TOL
     sess.close()
+
+
+# ------------------------------------------------------------------- uncompressed reference mode, 128-wide heads
+@pytest.mark.parametrize("H_q,lens,paged", [
+    (32, [700, 64, 1, 129], False),          # G = 4
+    (64, [300, 517], False),                 # G = 8
+    (32, [450, 33, 200], True),              # 64-token pages in a random physical order
+])
+def test_full_rank_mode_streaming_kernel(H_q, lens, paged):
+    """Ordinary KV cache (keys stored rotated): the streaming decode kernel against textbook attention over the
+    uncompressed weights, with several context-split counts."""
+    import torch
+    D, H_kv, d_h = 1024, 8, 128
+    prob = H.Problem(D, H_q, H_kv, d_h, 64, 64, theta=500000.0, layer=31)
+    b, n_max = len(lens), max(lens) + 5
+    sess = H.Session(prob, max_pos=n_max, batch=b, mode=1)
+    xs = [synth.hidden_states(n_max, D, 31, chunk=300 + s).astype(np.float64) for s in range(b)]
+    if paged:
+        cache, k, v, sl, ptd, pt = H.paged_cache(sess, b, [n_max] * b, 64, order_seed=5)
+    else:
+        cache, k, v, sl = H.contiguous_cache(sess, b, n_max, [n_max] * b)
+    sess.L.lorc_append(sess.ctx, 0, cache, H.dev_bf16(np.stack(xs)), T=n_max)
+    sl[:] = torch.tensor(lens, dtype=torch.int32)
+    q = synth.queries(b, H_q, d_h, 31, 1, 8.0).astype(np.float64)
+    want = [O.decode_attn_full(xs[s][:lens[s]], prob.W_k, prob.W_v, q[s], H_kv, prob.theta) for s in range(b)]
+    outs = []
+    for n_splits in (0, 1, 3):
+        out = torch.zeros(b, H_q, d_h, dtype=torch.bfloat16, device="cuda")
+        sess.L.lorc_decode_attn(sess.ctx, 0, cache, H.dev_bf16(q), out, n_splits=n_splits)
+        assert sess.L.lorc_sync_status(sess.ctx) == 0, sess.L.lorc_last_error(sess.ctx)
+        assert sess.L.lorc_last_path(sess.ctx) == 3, "the streaming kernel of the uncompressed mode was not taken"
+        got = H.host_f64(out)
+        for s in range(b):
+            assert O.rel_l2_rows(got[s], want[s]) <= TOL, (n_splits, s, O.rel_l2_rows(got[s], want[s]))
+        outs.append(got)
+    sess.close()
