@@ -7,7 +7,9 @@
 //   S[16 x 16 tok]  = Q^[16 x 128] . K[16 tok x 128]^T     q^ = RoPE(q, N-1)/sqrt(d_h) split into bf16 hi + lo parts,
 //                                                           so the scores keep fp32-level accuracy
 //   p = exp(S - m) rounded to bf16 (the same rounded value enters the denominator)
-//   O[16 x 128]    += P[16 x 16 tok] . V[16 tok x 128]      V staged in the warp's own shared-memory slice
+//   O[16 x 128]    += P[16 x 16 tok] . V[16 tok x 128]
+// Keys and values of a warp's 16 tokens are staged in its own double-buffered shared-memory slice by asynchronous
+// copies (the next tile is in flight while the current one is worked on) and read with ldmatrix.
 //
 // Each CTA leaves (m, l, un-normalised O) per query head for the merge kernel of the plain family.
 #include <math.h>
@@ -20,12 +22,16 @@ constexpr int FD_DH = 128;
 constexpr int FD_TILE = 64;          // tokens per CTA iteration (16 per warp)
 constexpr int FD_VPAD = 8;           // bf16 elements of padding per staged value row (keeps ldmatrix conflict-free)
 
-__device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                          uint32_t b1) {
+// m16n8k16 bf16 MMA whose A rows 8..15 are zero (operands a1, a3 = 0): c0, c1 belong to row lane / 4; the
+// padding row's results are discarded.
+__device__ __forceinline__ void mma_16816_lo(float& c0, float& c1, uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
     asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+        "{\n\t"
+        ".reg .f32 d2, d3;\n\t"          // results of the padding rows: zero, never read
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,d2,d3}, {%2,%3,%4,%3}, {%5,%6}, {%0,%1,%7,%7};\n\t"
+        "}\n"
+        : "+f"(c0), "+f"(c1)
+        : "r"(a0), "r"(0u), "r"(a2), "r"(b0), "r"(b1), "f"(0.f));
 }
 
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* smem_row) {
@@ -40,20 +46,41 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void* smem_row) {
+    const uint32_t addr = (uint32_t)__cvta_generic_to_shared(smem_row);
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+
+// 16-byte asynchronous copy global -> shared (bypassing L1), grouped with commit / wait
+__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gsrc) {
+    const uint32_t addr = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(addr), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+constexpr int FD_ROW = FD_DH + FD_VPAD;              // staged row length in bf16 elements (272 bytes)
+
 struct FdSmem {
     float qs[8][FD_DH];                              // rotated, scaled queries of the G heads (rows G..7 zero)
+    float m[4][8], l[4][8];
     union {
-        bf16 v[4][16][FD_DH + FD_VPAD];              // per warp: its 16 value rows
+        bf16 kv[4][2][2][16][FD_ROW];                // [warp][buffer][keys | values][token][dimension]
         float o[4][8][FD_DH];                        // after the loop: every warp's un-normalised output
     } u;
-    float m[4][8], l[4][8];
 };
 
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(128, 3)
 full_decode_mma_kernel(const bf16* __restrict__ q, CacheView cv, int G, int n_splits, int rope_style,
                        const float2* __restrict__ rope_table, int max_pos, float* __restrict__ part_ml,
                        float* __restrict__ part_o, int* status) {
-    __shared__ __align__(16) FdSmem sm;
+    extern __shared__ __align__(16) uint8_t fd_raw[];
+    FdSmem& sm = *reinterpret_cast<FdSmem*>(fd_raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, t = lane & 3;            // fragment row / column group of this lane
     const int split = blockIdx.x, kvh = blockIdx.y, s = blockIdx.z;
@@ -68,6 +95,39 @@ full_decode_mma_kernel(const bf16* __restrict__ q, CacheView cv, int G, int n_sp
     const int tiles = (len + FD_TILE - 1) / FD_TILE;
     const int tps = (tiles + n_splits - 1) / n_splits;
     const int t_begin = min(len, split * tps * FD_TILE), t_end = min(len, (split + 1) * tps * FD_TILE);
+    const int col0 = kvh * FD_DH;
+
+    // Stage the 16 key rows and 16 value rows of the warp's tile that starts at token t0 into buffer `buf`
+    // (asynchronous 16-byte copies, two rows per step; rows that do not exist are zero).  Returns, in lanes 0..15,
+    // the cache row of token t0 + lane (-1: none).
+    auto stage = [&](int t0, int buf) -> long long {
+        long long my_row = -1;
+        if (lane < 16 && t0 + lane < t_end) {
+            my_row = lorc_row_index(cv, s, t0 + lane);
+            if (my_row < 0) lorc_set_status(status, LORC_ERR_CAPACITY);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int r = 2 * i + (lane >> 4);
+            const long long row = __shfl_sync(0xffffffffu, my_row, r);
+            bf16* kd = &sm.u.kv[warp][buf][0][r][(lane & 15) * 8];
+            bf16* vd = &sm.u.kv[warp][buf][1][r][(lane & 15) * 8];
+            if (row >= 0) {
+                cp_async_16(kd, reinterpret_cast<const uint4*>(cv.k + row * cv.w_k + col0) + (lane & 15));
+                cp_async_16(vd, reinterpret_cast<const uint4*>(cv.v + row * cv.w_v + col0) + (lane & 15));
+            } else {
+                *reinterpret_cast<uint4*>(kd) = make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint4*>(vd) = make_uint4(0, 0, 0, 0);
+            }
+        }
+        cp_async_commit();
+        return my_row;
+    };
+
+    // the first tile is on its way while the query is prepared
+    const int t_first = t_begin + warp * 16;
+    long long row_cur = -1;
+    if (t_first < t_end) row_cur = stage(t_first, 0);
 
     // q^ = RoPE(q, N - 1) / sqrt(d_h) for the G heads of this KV head
     for (int i = tid; i < 8 * (FD_DH / 2); i += 128) {
@@ -88,75 +148,51 @@ full_decode_mma_kernel(const bf16* __restrict__ q, CacheView cv, int G, int n_sp
     }
     __syncthreads();
 
-    // Query fragments.  The contraction index of an MMA may be numbered freely as long as both operands agree: k-step
-    // 2j / 2j+1 of lane (g, t) covers the dimensions 32 j + 8 t + {0..3} / {4..7}, so a lane's key operand for two
-    // k-steps is one 16-byte load of 8 consecutive dimensions.  Rows 8..15 of the tile are padding (zero operands).
+    // Query fragments of row g (rows 8..15 of the tile are padding): k-step ks covers the dimensions 16 ks .. + 15,
+    // split into bf16 hi + lo parts.
     uint32_t qhi[8][2], qlo[8][2];
 #pragma unroll
     for (int ks = 0; ks < 8; ++ks) {
-        const int d0 = 32 * (ks >> 1) + 8 * t + 4 * (ks & 1);
-        float v[4], hi[4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            v[e] = g < 8 ? sm.qs[g][d0 + e] : 0.f;
-            hi[e] = __bfloat162float(__float2bfloat16_rn(v[e]));
+        for (int half = 0; half < 2; ++half) {
+            const int d0 = 16 * ks + 8 * half + 2 * t;
+            const float v0 = sm.qs[g][d0], v1 = sm.qs[g][d0 + 1];
+            const float h0 = __bfloat162float(__float2bfloat16_rn(v0)), h1 = __bfloat162float(__float2bfloat16_rn(v1));
+            qhi[ks][half] = pack_bf16(h0, h1);
+            qlo[ks][half] = pack_bf16(v0 - h0, v1 - h1);
         }
-        qhi[ks][0] = pack_bf16(hi[0], hi[1]);
-        qhi[ks][1] = pack_bf16(hi[2], hi[3]);
-        qlo[ks][0] = pack_bf16(v[0] - hi[0], v[1] - hi[1]);
-        qlo[ks][1] = pack_bf16(v[2] - hi[2], v[3] - hi[3]);
     }
 
-    float o[16][4];                                   // O[rows g, g + 8][dims 8 dt + 2 t, + 1]
+    float o[16][2];                                   // O[row g][dims 8 dt + 2 t, + 1]
 #pragma unroll
-    for (int dt = 0; dt < 16; ++dt)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) o[dt][e] = 0.f;
+    for (int dt = 0; dt < 16; ++dt) o[dt][0] = o[dt][1] = 0.f;
     float m_run = -INFINITY, l_run = 0.f;             // running maximum and (per-lane partial) denominator of row g
 
-    const int col0 = kvh * FD_DH;
-    for (int t0 = t_begin + warp * 16; t0 < t_end; t0 += FD_TILE) {
-        // rows of this warp's 16 tokens (lane i < 16 looks token i up; -1: past the end or no such row)
-        long long my_row = -1;
-        if (lane < 16 && t0 + lane < t_end) {
-            my_row = lorc_row_index(cv, s, t0 + lane);
-            if (my_row < 0) lorc_set_status(status, LORC_ERR_CAPACITY);
-        }
-        // keys: tokens g and g + 8, four 16-byte pieces each
-        uint4 kf[2][4];
-#pragma unroll
-        for (int nt = 0; nt < 2; ++nt) {
-            const long long row = __shfl_sync(0xffffffffu, my_row, nt * 8 + g);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                kf[nt][j] = make_uint4(0, 0, 0, 0);
-                if (row >= 0) kf[nt][j] = __ldg(reinterpret_cast<const uint4*>(cv.k + row * cv.w_k + col0 + 32 * j + 8 * t));
-            }
-        }
-        // values: two rows per step, staged in this warp's slice (rows that do not exist are zero)
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int r = 2 * i + (lane >> 4);
-            const long long row = __shfl_sync(0xffffffffu, my_row, r);
-            uint4 val = make_uint4(0, 0, 0, 0);
-            if (row >= 0) val = __ldg(reinterpret_cast<const uint4*>(cv.v + row * cv.w_v + col0) + (lane & 15));
-            *reinterpret_cast<uint4*>(&sm.u.v[warp][r][(lane & 15) * 8]) = val;
+    const int mi = lane >> 3;                         // which 8 x 8 matrix of an ldmatrix.x4 this lane addresses
+    int it = 0;
+    for (int t0 = t_first; t0 < t_end; t0 += FD_TILE, ++it) {
+        const int buf = it & 1;
+        // next tile into the other buffer, then wait for this one
+        long long row_next = -1;
+        const bool has_next = t0 + FD_TILE < t_end;
+        if (has_next) {
+            row_next = stage(t0 + FD_TILE, buf ^ 1);
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
         }
         __syncwarp();
 
-        // scores of rows g (and padding rows g + 8) against tokens nt * 8 + 2 t, + 1
-        float sc[2][4];
+        // scores of row g against tokens nt * 8 + 2 t, + 1
+        float sc[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
 #pragma unroll
-        for (int nt = 0; nt < 2; ++nt) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) sc[nt][e] = 0.f;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                mma_16816(sc[nt], qhi[2 * j][0], 0u, qhi[2 * j][1], 0u, kf[nt][j].x, kf[nt][j].y);
-                mma_16816(sc[nt], qhi[2 * j + 1][0], 0u, qhi[2 * j + 1][1], 0u, kf[nt][j].z, kf[nt][j].w);
-                mma_16816(sc[nt], qlo[2 * j][0], 0u, qlo[2 * j][1], 0u, kf[nt][j].x, kf[nt][j].y);
-                mma_16816(sc[nt], qlo[2 * j + 1][0], 0u, qlo[2 * j + 1][1], 0u, kf[nt][j].z, kf[nt][j].w);
-            }
+        for (int ks = 0; ks < 8; ++ks) {
+            uint32_t kb[4];       // (tokens 0..7, dims 16 ks..+7), (0..7, +8..15), (tokens 8..15, ...), (8..15, ...)
+            ldmatrix_x4(kb, &sm.u.kv[warp][buf][0][(mi >> 1) * 8 + (lane & 7)][16 * ks + 8 * (mi & 1)]);
+            mma_16816_lo(sc[0][0], sc[0][1], qhi[ks][0], qhi[ks][1], kb[0], kb[1]);
+            mma_16816_lo(sc[1][0], sc[1][1], qhi[ks][0], qhi[ks][1], kb[2], kb[3]);
+            mma_16816_lo(sc[0][0], sc[0][1], qlo[ks][0], qlo[ks][1], kb[0], kb[1]);
+            mma_16816_lo(sc[1][0], sc[1][1], qlo[ks][0], qlo[ks][1], kb[2], kb[3]);
         }
         // running softmax of row g over this warp's tokens
         float mx = -INFINITY;
@@ -164,8 +200,7 @@ full_decode_mma_kernel(const bf16* __restrict__ q, CacheView cv, int G, int n_sp
         for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
-                const int tok = nt * 8 + 2 * t + e;
-                const long long row = __shfl_sync(0xffffffffu, my_row, tok);
+                const long long row = __shfl_sync(0xffffffffu, row_cur, nt * 8 + 2 * t + e);
                 if (row < 0) sc[nt][e] = -INFINITY;
                 mx = fmaxf(mx, sc[nt][e]);
             }
@@ -187,37 +222,35 @@ full_decode_mma_kernel(const bf16* __restrict__ q, CacheView cv, int G, int n_sp
             pa[1] = pack_bf16(p[1][0], p[1][1]);
         }
         m_run = m_new;
-        // O = alpha O + P V   (alpha of a lane's row; the padding rows carry zeros)
+        // O = alpha O + P V
 #pragma unroll
         for (int dp = 0; dp < 8; ++dp) {
-            uint32_t vb[4];
-            const int mi = lane >> 3;                 // which 8 x 8 matrix this lane addresses
-            ldmatrix_x4_trans(vb, &sm.u.v[warp][(mi & 1) * 8 + (lane & 7)][8 * (2 * dp + (mi >> 1))]);
+            uint32_t vb[4];       // (tokens 0..7 | 8..15) x (dims 16 dp..+7 | +8..15), transposed on the way in
+            ldmatrix_x4_trans(vb, &sm.u.kv[warp][buf][1][(mi & 1) * 8 + (lane & 7)][8 * (2 * dp + (mi >> 1))]);
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
-                float (&acc)[4] = o[2 * dp + half];
+                float (&acc)[2] = o[2 * dp + half];
                 acc[0] *= alpha;
                 acc[1] *= alpha;
-                mma_16816(acc, pa[0], 0u, pa[1], 0u, vb[2 * half], vb[2 * half + 1]);
+                mma_16816_lo(acc[0], acc[1], pa[0], pa[1], vb[2 * half], vb[2 * half + 1]);
             }
         }
-        __syncwarp();                                 // the slice is rewritten in the next iteration
+        __syncwarp();                                 // this buffer is refilled two tiles from now
+        row_cur = row_next;
     }
 
     // merge the four warps of the CTA
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-    __syncthreads();                                  // every warp is done with its value slice (the union is reused)
-    if (g < 8) {
-        if (t == 0) {
-            sm.m[warp][g] = m_run;
-            sm.l[warp][g] = l_run;
-        }
+    __syncthreads();                                  // every warp is done with its staging buffers (the union is reused)
+    if (t == 0) {
+        sm.m[warp][g] = m_run;
+        sm.l[warp][g] = l_run;
+    }
 #pragma unroll
-        for (int dt = 0; dt < 16; ++dt) {
-            sm.u.o[warp][g][8 * dt + 2 * t] = o[dt][0];
-            sm.u.o[warp][g][8 * dt + 2 * t + 1] = o[dt][1];
-        }
+    for (int dt = 0; dt < 16; ++dt) {
+        sm.u.o[warp][g][8 * dt + 2 * t] = o[dt][0];
+        sm.u.o[warp][g][8 * dt + 2 * t + 1] = o[dt][1];
     }
     __syncthreads();
     for (int h = 0; h < G; ++h) {
@@ -252,7 +285,14 @@ cudaError_t lorc_full_decode(const lorc_ctx* ctx, const CacheView& cv, const bf1
                              float* part_o, cudaStream_t st, int* launches) {
     const lorc_model_desc& d = ctx->desc;
     dim3 grid(n_splits, d.n_kv_heads, cv.batch);
-    full_decode_mma_kernel<<<grid, 128, 0, st>>>(q, cv, ctx->group, n_splits, d.rope_style, ctx->rope_table, d.max_pos,
+    static bool attr = false;
+    if (!attr) {
+        cudaError_t e = cudaFuncSetAttribute(full_decode_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)sizeof(FdSmem));
+        if (e != cudaSuccess) return e;
+        attr = true;
+    }
+    full_decode_mma_kernel<<<grid, 128, sizeof(FdSmem), st>>>(q, cv, ctx->group, n_splits, d.rope_style, ctx->rope_table, d.max_pos,
                                                  part_ml, part_o, ctx->status_dev);
     *launches += 1;
     return cudaGetLastError();
