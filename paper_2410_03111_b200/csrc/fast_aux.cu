@@ -24,9 +24,14 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// FULL (uncompressed mode): the factor is [W_K | W_V] and keys are cached rotated.  The key columns of the tiled
+// factor are permuted (see retile_factor_kernel) so that the two accumulator columns a thread ends up with are the two
+// members of one rotary pair: the rotation needs no exchange between threads.
+template <bool FULL>
 __global__ void __launch_bounds__(256)
 append_mma_kernel(const bf16* __restrict__ x, const bf16* __restrict__ A_tiled, CacheView cv, int D, int r_k,
-                  int r_v, int T, int max_pos, int* status) {
+                  int r_v, int T, int max_pos, int* status, int d_head, int rope_style,
+                  const float2* __restrict__ rope_table) {
     __shared__ float red[8][32][4];
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
     const int g = lane >> 2, t = lane & 3;
@@ -111,33 +116,54 @@ append_mma_kernel(const bf16* __restrict__ x, const bf16* __restrict__ A_tiled, 
             continue;
         }
         __nv_bfloat162 v = __floats2bfloat162_rn(c[half * 2], c[half * 2 + 1]);
-        if (col < r_k)
+        if (FULL && col < r_k) {
+            const int hd = d_head / 2, head = col / d_head, j = (col - head * d_head) >> 1;
+            const float2 cs = rope_table[(long long)pos * hd + j];
+            const float a = c[half * 2], b = c[half * 2 + 1];
+            const float ka = a * cs.x - b * cs.y, kb = a * cs.y + b * cs.x;
+            bf16* krow = cv.k + row * cv.w_k;
+            if (rope_style == LORC_ROPE_HALF_SPLIT) {
+                krow[head * d_head + j] = __float2bfloat16_rn(ka);
+                krow[head * d_head + j + hd] = __float2bfloat16_rn(kb);
+            } else {
+                *reinterpret_cast<__nv_bfloat162*>(krow + col) = __floats2bfloat162_rn(ka, kb);
+            }
+        } else if (col < r_k)
             *reinterpret_cast<__nv_bfloat162*>(cv.k + row * cv.w_k + col) = v;
         else
             *reinterpret_cast<__nv_bfloat162*>(cv.v + row * cv.w_v + (col - r_k)) = v;
     }
 }
 
-__global__ void retile_factor_kernel(const bf16* __restrict__ A_cat, bf16* __restrict__ A_tiled, int D, int R) {
+// The first `pair_cols` columns (0: none) are taken in rotary-pair order: tiled column head * d_head + 2 j + e is the
+// factor's column head * d_head + j + e * d_head / 2, so that a pair (j, j + d_head / 2) sits in adjacent columns.
+__global__ void retile_factor_kernel(const bf16* __restrict__ A_cat, bf16* __restrict__ A_tiled, int D, int R,
+                                     int pair_cols, int d_head) {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= (long long)D * R) return;
     const int e = (int)(i & 7), lane = (int)((i >> 3) & 31);
     const long long blk = i >> 8;                       // (column tile, k block)
     const int kb = (int)(blk % (D / 32)), nt = (int)(blk / (D / 32));
-    const int col = nt * 8 + (lane >> 2), k = kb * 32 + (lane & 3) * 8 + e;
+    int col = nt * 8 + (lane >> 2);
+    const int k = kb * 32 + (lane & 3) * 8 + e;
+    if (col < pair_cols) {
+        const int head = col / d_head, w = col - head * d_head;
+        col = head * d_head + (w >> 1) + (w & 1) * (d_head / 2);
+    }
     A_tiled[i] = A_cat[(long long)k * R + col];
 }
 
 }  // namespace
 
-cudaError_t lorc_fast_retile_factor(const bf16* A_cat, bf16* A_tiled, int D, int R, cudaStream_t st) {
+cudaError_t lorc_fast_retile_factor(const bf16* A_cat, bf16* A_tiled, int D, int R, int pair_cols, int d_head,
+                                    cudaStream_t st) {
     const long long total = (long long)D * R;
-    retile_factor_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(A_cat, A_tiled, D, R);
+    retile_factor_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(A_cat, A_tiled, D, R, pair_cols, d_head);
     return cudaGetLastError();
 }
 
 bool lorc_tc_append_supported(const lorc_ctx* ctx, const LorcLayer& L, const CacheView&, int) {
-    return L.mode == LORC_MODE_LATENT && ctx->desc.d_model % 256 == 0 && L.A_tiled != nullptr;
+    return ctx->desc.d_model % 256 == 0 && L.A_tiled != nullptr;
 }
 
 cudaError_t lorc_tc_append(lorc_ctx* ctx, int, const LorcLayer& L, const CacheView& cv, const bf16* x, int T,
@@ -145,8 +171,14 @@ cudaError_t lorc_tc_append(lorc_ctx* ctx, int, const LorcLayer& L, const CacheVi
     const int R = L.r_k + L.r_v;
     const long long n_tok = (long long)cv.batch * T;
     dim3 grid((R + 7) / 8, (unsigned)((n_tok + 15) / 16));
-    append_mma_kernel<<<grid, 256, 0, st>>>(x, L.A_tiled, cv, ctx->desc.d_model, L.r_k, L.r_v, T, ctx->desc.max_pos,
-                                            ctx->status_dev);
+    if (L.mode == LORC_MODE_FULL)
+        append_mma_kernel<true><<<grid, 256, 0, st>>>(x, L.A_tiled, cv, ctx->desc.d_model, L.r_k, L.r_v, T,
+                                                      ctx->desc.max_pos, ctx->status_dev, ctx->desc.d_head,
+                                                      ctx->desc.rope_style, ctx->rope_table);
+    else
+        append_mma_kernel<false><<<grid, 256, 0, st>>>(x, L.A_tiled, cv, ctx->desc.d_model, L.r_k, L.r_v, T,
+                                                       ctx->desc.max_pos, ctx->status_dev, ctx->desc.d_head,
+                                                       ctx->desc.rope_style, ctx->rope_table);
     *launches += 1;
     return cudaGetLastError();
 }

@@ -207,7 +207,10 @@ int lorc_load_factors(lorc_ctx* ctx, int layer, int mode, int r_k, int r_v, cons
     if (e == cudaSuccess)
         e = cudaMemcpy2DAsync(L.A_cat + r_k, (size_t)R * sizeof(bf16), A_v, (size_t)r_v * sizeof(bf16),
                               (size_t)r_v * sizeof(bf16), D, cudaMemcpyDeviceToDevice, st);
-    if (e == cudaSuccess && L.A_tiled) e = lorc_fast_retile_factor(L.A_cat, L.A_tiled, D, R, st);
+    if (e == cudaSuccess && L.A_tiled) {
+        const bool pairs = mode == LORC_MODE_FULL && ctx->desc.rope_style == LORC_ROPE_HALF_SPLIT;
+        e = lorc_fast_retile_factor(L.A_cat, L.A_tiled, D, R, pairs ? r_k : 0, ctx->desc.d_head, st);
+    }
     if (e == cudaSuccess && mode == LORC_MODE_LATENT) {
         e = cudaMemcpyAsync(L.B_k, B_k, (size_t)r_k * n * sizeof(bf16), cudaMemcpyDeviceToDevice, st);
         if (e == cudaSuccess)

@@ -28,8 +28,11 @@ cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView
                               int n_splits_hint, void* scratch, size_t scratch_bytes, bf16* out, cudaStream_t st,
                               int* launches);
 
-// A_cat [D, R] (row-major) -> fragment order [R/8][D/32][32 lanes][8] used by the fast append kernel.
-cudaError_t lorc_fast_retile_factor(const bf16* A_cat, bf16* A_tiled, int D, int R, cudaStream_t st);
+// A_cat [D, R] (row-major) -> fragment order [R/8][D/32][32 lanes][8] used by the fast append kernel.  The first
+// pair_cols columns (uncompressed mode with half-split rotary pairs: the key columns; otherwise 0) are laid out with the
+// two members of each rotary pair side by side.
+cudaError_t lorc_fast_retile_factor(const bf16* A_cat, bf16* A_tiled, int D, int R, int pair_cols, int d_head,
+                                    cudaStream_t st);
 
 // Drop cached per-layer state (tensor maps) when factors are reloaded / the context dies.
 void lorc_tc_invalidate_layer(lorc_ctx* ctx, int layer);

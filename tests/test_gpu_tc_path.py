@@ -219,6 +219,13 @@ def test_full_rank_mode_streaming_kernel(H_q, lens, paged):
     else:
         cache, k, v, sl = H.contiguous_cache(sess, b, n_max, [n_max] * b)
     sess.L.lorc_append(sess.ctx, 0, cache, H.dev_bf16(np.stack(xs)), T=n_max)
+    assert sess.L.lorc_last_path(sess.ctx) == 2, "the mma cache-write kernel was not taken"
+    if not paged:
+        # the cache holds the rotated key projections and the value projections, each rounded once
+        Kr = O.rope((xs[0] @ prob.W_k).reshape(-1, H_kv, d_h), np.arange(n_max)[:, None], prob.theta).reshape(-1, prob.n)
+        assert np.all(np.abs(H.host_f64(k[0]) - Kr) <= H.bf16_ulp(Kr) + 1e-6)
+        Vp = xs[0] @ prob.W_v
+        assert np.all(np.abs(H.host_f64(v[0]) - Vp) <= H.bf16_ulp(Vp) + 1e-6)
     sl[:] = torch.tensor(lens, dtype=torch.int32)
     q = synth.queries(b, H_q, d_h, 31, 1, 8.0).astype(np.float64)
     want = [O.decode_attn_full(xs[s][:lens[s]], prob.W_k, prob.W_v, q[s], H_kv, prob.theta) for s in range(b)]
