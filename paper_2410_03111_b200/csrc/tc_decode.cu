@@ -12,8 +12,9 @@
 //                 with the G rotated queries of its KV head; the scores (log2 units) go to scratch.
 //                 RoPE is split as R(n0 + t) = R(n0) R(t): R(t), t < 128, is a constant table in shared
 //                 memory and R(n0) is folded into the query once per unit (q' = R(m - n0) q).
-//                 It also leaves the maximum of every 32-token quarter tile, so that the next kernel knows
-//                 the exact row maximum of the softmax without a pass over the scores.
+//                 It also folds the maximum of every 32-token quarter tile into one word per (sequence, head)
+//                 with an atomic maximum, so that the next kernel knows the exact row maximum of the softmax
+//                 without a pass over the scores.
 //  PV kernel      softmax + P.C_V + value up-projection, split by latent columns (tc_pv.cu).
 //
 // Keys and values never exist in memory; only the 4*H_q bytes of scores per token are written.
@@ -52,7 +53,7 @@ struct ScoreSmem {
 struct ScoreParams {
     const bf16* q;                 // [b, H_q, 128]
     float* scores;                 // [b, H_q, n_pad]
-    float* tmax;                   // [b, H_q, tiles_per_seq, 4]  maxima per 32-token quarter tile
+    unsigned* rowmax;              // [b, H_q]  running row maximum as an order-preserving key (0: none yet)
     const int32_t* seq_lens;
     const int32_t* page_table;     // NULL: contiguous
     const float2* rope_table;      // [max_pos][64]
@@ -112,7 +113,7 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&sm.acc_full[i], 1);
-            mbar_init(&sm.acc_empty[i], 2 * S_EPI);      // the epilogue threads of both CTAs
+            mbar_init(&sm.acc_empty[i], 2 * S_EPI / 32); // one arrival per epilogue warp, both CTAs
         }
         mbar_init(&sm.trig_full, 1);
         fence_barrier_init();
@@ -358,8 +359,11 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
                     f2_unpack(acc2[m][g], x, y);
                     acc[m][g] = x + y;
                 }
+            // one arrival per warp (512 arrivals per unit on one barrier, half of them remote, cost about 2 % at low
+            // ranks): every lane has its accumulator values in registers (tmem_wait_ld above)
             tc_fence_before_sync();
-            mbar_arrive_cluster(lead_acc_empty[buf]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(lead_acc_empty[buf]);
             // add the four lanes' partial dots; lane c ends with the heads g = 4i + c
             float tot[4][G / 4];
 #pragma unroll
@@ -392,8 +396,7 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
                 }
 #pragma unroll
                 for (int o = 4; o < 32; o <<= 1) mxv = fmaxf(mxv, __shfl_xor_sync(0xffffffffu, mxv, o));
-                if (r == 0 && un.tile < p.tiles_per_seq)
-                    p.tmax[(((long long)un.s * p.H_q + h) * p.tiles_per_seq + un.tile) * 4 + quarter] = mxv;
+                if (r == 0 && mxv > -INFINITY) atomicMax(p.rowmax + (long long)un.s * p.H_q + h, lorc_float_key(mxv));
             }
             ++uc;
             u = u_next;
@@ -446,6 +449,9 @@ struct LorcTcLayer {
 
 struct LorcTcState {
     float2* rope_tile = nullptr;
+    unsigned* rowmax = nullptr;         // [rowmax_cap] row maxima of the softmax, see lorc_tc_decode
+    size_t rowmax_cap = 0;
+    bool rowmax_dirty = true;
     std::vector<LorcTcLayer> layers;
     bool attrs_set = false;
 };
@@ -461,6 +467,7 @@ static LorcTcState* tc_state(lorc_ctx* ctx) {
 void lorc_tc_release(lorc_ctx* ctx) {
     if (ctx->tc) {
         cudaFree(ctx->tc->rope_tile);
+        cudaFree(ctx->tc->rowmax);
         delete ctx->tc;
         ctx->tc = nullptr;
     }
@@ -491,15 +498,9 @@ static size_t tc_scores_bytes(const lorc_ctx* ctx, int batch, int max_seq_len) {
     return lorc_align_up((size_t)batch * ctx->desc.n_q_heads * n_pad * sizeof(float), 256);
 }
 
-static size_t tc_tmax_bytes(const lorc_ctx* ctx, int batch, int max_seq_len) {
-    size_t tiles = (size_t)((max_seq_len + TILE - 1) / TILE);
-    return lorc_align_up((size_t)batch * ctx->desc.n_q_heads * tiles * 4 * sizeof(float), 256);
-}
-
 size_t lorc_tc_workspace_bytes(const lorc_ctx* ctx, int batch, int max_seq_len) {
     if (!tc_shape_ok(ctx)) return 0;
-    return tc_scores_bytes(ctx, batch, max_seq_len) + tc_tmax_bytes(ctx, batch, max_seq_len) +
-           lorc_tc_pv_scratch_bytes(ctx, batch, max_seq_len);
+    return tc_scores_bytes(ctx, batch, max_seq_len) + lorc_tc_pv_scratch_bytes(ctx, batch, max_seq_len);
 }
 
 static bool build_cache_maps(LorcTcLayer& T, const LorcLayer& L, const CacheView& cv) {
@@ -562,15 +563,31 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
     const int tiles = (cv.max_seq_len + TILE - 1) / TILE;
     const int n_pad = tiles * TILE;
     const size_t sc_bytes = tc_scores_bytes(ctx, cv.batch, cv.max_seq_len);
-    const size_t tm_bytes = tc_tmax_bytes(ctx, cv.batch, cv.max_seq_len);
-    if (sc_bytes + tm_bytes >= ws_bytes) return cudaErrorMemoryAllocation;
+    if (sc_bytes >= ws_bytes) return cudaErrorMemoryAllocation;
     float* scores = (float*)ws;
-    float* tmax = (float*)((char*)ws + sc_bytes);
-    void* pv_scratch = (char*)ws + sc_bytes + tm_bytes;
-    const size_t pv_bytes = ws_bytes - sc_bytes - tm_bytes;
+    void* pv_scratch = (char*)ws + sc_bytes;
+    const size_t pv_bytes = ws_bytes - sc_bytes;
+    // Row maxima [batch, H_q]: all zero between calls (the PV kernel clears what the score kernel raised).  Owned by
+    // the library because that invariant must hold from the first call on; grown when a larger batch shows up, and
+    // cleared again after a call that did not get as far as launching the PV kernel.
+    const size_t rm_need = (size_t)cv.batch * d.n_q_heads;
+    if (rm_need > T->rowmax_cap) {
+        cudaError_t e = cudaFree(T->rowmax);
+        T->rowmax = nullptr;
+        T->rowmax_cap = 0;
+        if (e == cudaSuccess) e = cudaMalloc(&T->rowmax, rm_need * sizeof(unsigned));
+        if (e != cudaSuccess) return e;
+        T->rowmax_cap = rm_need;
+        T->rowmax_dirty = true;
+    }
+    if (T->rowmax_dirty) {
+        cudaError_t e = cudaMemsetAsync(T->rowmax, 0, T->rowmax_cap * sizeof(unsigned), st);
+        if (e != cudaSuccess) return e;
+    }
+    T->rowmax_dirty = true;
 
     ScoreParams sp;
-    sp.q = q; sp.scores = scores; sp.tmax = tmax; sp.seq_lens = cv.seq_lens; sp.page_table = cv.page_table;
+    sp.q = q; sp.scores = scores; sp.rowmax = T->rowmax; sp.seq_lens = cv.seq_lens; sp.page_table = cv.page_table;
     sp.rope_table = ctx->rope_table; sp.rope_tile = reinterpret_cast<const float4*>(T->rope_tile); sp.status = ctx->status_dev;
     sp.batch = cv.batch; sp.H_q = d.n_q_heads; sp.n_hp = d.n_kv_heads / 2; sp.r_k = L.r_k; sp.n_pad = n_pad;
     sp.tiles_per_seq = tiles; sp.tile_pairs = (tiles + 1) / 2; sp.max_pos = d.max_pos;
@@ -590,6 +607,8 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
         *launches += 1;
         if (e != cudaSuccess) return e;
     }
-    return lorc_tc_pv_launch(ctx, L, cv, TL.mapCV, TL.mapBVT, scores, tmax, n_pad, tiles, n_splits, pv_scratch, pv_bytes,
-                             out, st, launches);
+    const cudaError_t e2 = lorc_tc_pv_launch(ctx, L, cv, TL.mapCV, TL.mapBVT, scores, T->rowmax, n_pad, tiles, n_splits,
+                                             pv_scratch, pv_bytes, out, st, launches);
+    if (e2 == cudaSuccess) T->rowmax_dirty = false;
+    return e2;
 }

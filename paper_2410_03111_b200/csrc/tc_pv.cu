@@ -1,7 +1,7 @@
 // Softmax, P.C_V split by LATENT COLUMNS, and the value up-projection; the two contractions run on the tensor cores.
 //
-// Probability kernel.  One CTA per (sequence, group of 128-token tiles): finds the exact row maximum of every head
-// over the whole sequence (from the quarter-tile maxima the score kernel leaves behind), turns the scores of its
+// Probability kernel.  One CTA per (sequence, group of 128-token tiles): reads the exact row maximum of every head
+// over the whole sequence (one word per head, raised by the score kernel with atomic maxima), turns the scores of its
 // tiles into p = 2^(s - m) rounded to bf16 -- stored tile by tile as the 128-byte-swizzled K-major image the PV
 // kernel's MMA reads, so that kernel fetches a tile with one bulk copy -- and writes its share of the softmax
 // denominator.  The probabilities are computed once, not once per column block.
@@ -42,7 +42,7 @@ __device__ __forceinline__ float ldg_nc_f32(const float* p) {
 // ------------------------------------------------------------------------------------------------
 struct ProbParams {
     const float* scores;           // [b, H_q, n_pad]      log2 units
-    const float* tmax;             // [b, H_q, tiles, 4]   maxima of every 32-token quarter tile
+    const unsigned* rowmax;        // [b, H_q]   exact row maxima as order-preserving keys (0: no token seen)
     bf16* probs;                   // [b, tiles, 2 chunks of 64 tokens, H_q, 64]   swizzled tile images
     float* l_part;                 // [b, n_groups, H_q]
     int* done;                     // [b, n_blk]  arrival counters of the PV kernel's context shares, zeroed here
@@ -86,34 +86,10 @@ lorc_prob_kernel(const ProbParams p) {
 #pragma unroll
             for (int i = 0; i < NH; ++i) sv[i] = n < len ? ldg_nc_f32(sbase + (long long)i * p.n_pad + tile_lo * TILE) : 0.f;
         }
-        // exact maximum of every head over the WHOLE sequence ([tile][4 quarters] per head: one 16-byte load per
-        // tile; a thread takes every eighth tile of one head, eight loads in flight)
-        for (int idx = tid; idx < HQ * 8; idx += 256) {          // (head, tile phase)
-            const int h = idx >> 3, ph = idx & 7;
-            const float4* tp = reinterpret_cast<const float4*>(p.tmax + ((long long)s * p.H_q + h) * (4 * p.tiles));
-            float v = -INFINITY;
-            int i = ph;
-            for (; i + 56 < tiles_s; i += 64) {
-                float4 q[8];
-#pragma unroll
-                for (int u = 0; u < 8; ++u) q[u] = tp[i + 8 * u];
-#pragma unroll
-                for (int u = 0; u < 8; ++u) v = fmaxf(v, fmaxf(fmaxf(q[u].x, q[u].y), fmaxf(q[u].z, q[u].w)));
-            }
-            float4 q[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u)
-                q[u] = (i + 8 * u < tiles_s) ? tp[i + 8 * u] : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-#pragma unroll
-            for (int u = 0; u < 8; ++u) v = fmaxf(v, fmaxf(fmaxf(q[u].x, q[u].y), fmaxf(q[u].z, q[u].w)));
-            red[ph][h] = v;
-        }
-        __syncthreads();
+        // exact maximum of every head over the WHOLE sequence
         if (tid < HQ) {
-            float v = red[0][tid];
-#pragma unroll
-            for (int i = 1; i < 8; ++i) v = fmaxf(v, red[i][tid]);
-            m_s[tid] = v;
+            const unsigned key = p.rowmax[(long long)s * p.H_q + tid];
+            m_s[tid] = key ? lorc_key_float(key) : 0.f;
         }
         __syncthreads();
         for (int tile = tile_lo; tile < tile_hi; ++tile) {
@@ -189,6 +165,7 @@ struct Pv2Params {
     const bf16* probs;             // [b, tiles, 2, H_q, 64]   swizzled tile images
     float* o_part;                 // [b, n_csplit, H_q, r_pad]   un-normalised latent output, r_pad = 128 n_blk
     const float* l_part;           // [b, n_groups, H_q]   shares of the softmax denominator
+    unsigned* rowmax;              // [b, H_q]   row maxima of the softmax: zeroed here for the next call
     bf16* o_norm;                  // [b, H_q, r_pad]      normalised latent output
     int* done;                     // [b, n_blk]           context shares of a column block that have finished
     const int32_t* seq_lens;
@@ -338,6 +315,8 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
         const int r_pad = p.n_blk * 128;
         grid_dep_wait();                              // denominators come from the kernel before this one
         grid_dep_launch();
+        // the probability kernel has read the row maxima: leave them empty for the next call's score kernel
+        if (blk == 0 && cs == 0 && t < HQ) p.rowmax[(long long)s * p.H_q + t] = 0u;
         // while the tiles stream: the reciprocal softmax denominator of every head (all shares of the sequence)
         {
             constexpr int PARTS = 128 / HQ;
@@ -612,7 +591,7 @@ size_t lorc_tc_pv_scratch_bytes(const lorc_ctx* ctx, int batch, int max_seq_len)
 }
 
 cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, const CUtensorMap& mapCV,
-                              const CUtensorMap& mapBVT, const float* scores, const float* tmax, int n_pad, int tiles,
+                              const CUtensorMap& mapBVT, const float* scores, unsigned* rowmax, int n_pad, int tiles,
                               int n_splits_hint, void* scratch, size_t scratch_bytes, bf16* out, cudaStream_t st,
                               int* launches) {
     const lorc_model_desc& d = ctx->desc;
@@ -648,7 +627,7 @@ cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView
     {
         LorcStageTimer timer(ctx, LORC_STAGE_PV, st);
         ProbParams q;
-        q.scores = scores; q.tmax = tmax; q.probs = probs; q.l_part = l_part; q.done = done; q.seq_lens = cv.seq_lens;
+        q.scores = scores; q.rowmax = rowmax; q.probs = probs; q.l_part = l_part; q.done = done; q.seq_lens = cv.seq_lens;
         q.status = ctx->status_dev; q.H_q = d.n_q_heads; q.n_pad = n_pad; q.tiles = tiles; q.tiles_per_group = tpg;
         q.n_groups = n_groups; q.n_blk = n_blk; q.max_pos = d.max_pos;
         dim3 pgrid(n_groups, cv.batch);
@@ -660,7 +639,7 @@ cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView
         if (e != cudaSuccess) return e;
 
         Pv2Params p;
-        p.probs = probs; p.o_part = o_part; p.l_part = l_part; p.o_norm = o_norm; p.done = done;
+        p.probs = probs; p.o_part = o_part; p.l_part = l_part; p.rowmax = rowmax; p.o_norm = o_norm; p.done = done;
         p.seq_lens = cv.seq_lens; p.page_table = cv.page_table; p.status = ctx->status_dev;
         p.batch = cv.batch; p.H_q = d.n_q_heads; p.n_kv = d.n_kv_heads; p.r_v = L.r_v; p.tiles = tiles;
         p.n_blk = n_blk; p.n_csplit = n_csplit; p.n_groups = n_groups; p.max_pos = d.max_pos;
