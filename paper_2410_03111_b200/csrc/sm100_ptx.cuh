@@ -108,6 +108,10 @@ __device__ __forceinline__ bool mbar_wait_addr(uint32_t bar_addr, uint32_t parit
 }
 
 // Make generic-proxy writes to shared memory visible to the async proxy (TMA, tcgen05.mma).
+// orders this thread's earlier (acquired) view of memory, global included, before its later asynchronous-proxy copies
+__device__ __forceinline__ void fence_proxy_async_all() {
+    asm volatile("fence.proxy.async;" ::: "memory");
+}
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }

@@ -156,14 +156,14 @@ struct Pv2Smem {
     bf16 P[P_STAGES][2][HQ * KC];         // probabilities [HQ][128 tokens] as two 64-token chunks, 128-byte swizzle
     float red[128 / HQ][HQ];
     float l_inv[HQ];
-    uint64_t full[P_STAGES], empty[P_STAGES], o_full;
+    uint64_t full[P_STAGES], empty[P_STAGES], o_full, red_full;
     uint32_t tmem_base;
     int last;
 };
 
 struct Pv2Params {
     const bf16* probs;             // [b, tiles, 2, H_q, 64]   swizzled tile images
-    float* o_part;                 // [b, n_csplit, H_q, r_pad]   un-normalised latent output, r_pad = 128 n_blk
+    float* o_part;                 // [b, n_blk, n_csplit, H_q, 128]   un-normalised latent output of every context share
     const float* l_part;           // [b, n_groups, H_q]   shares of the softmax denominator
     unsigned* rowmax;              // [b, H_q]   row maxima of the softmax: zeroed here for the next call
     bf16* o_norm;                  // [b, H_q, r_pad]      normalised latent output
@@ -205,6 +205,7 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
             mbar_init(&sm.empty[i], 1);
         }
         mbar_init(&sm.o_full, 1);
+        mbar_init(&sm.red_full, 1);
         fence_barrier_init();
         prefetch_tensormap(&mapCV);
     }
@@ -355,11 +356,13 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
         }
         bool finish = true;
         if (p.n_csplit > 1) {
-            // publish this share; the share that arrives last adds them all up (in share order, so the result does
-            // not depend on which one that is)
-            float* op = p.o_part + (((long long)s * p.n_csplit + cs) * p.H_q) * r_pad + rho0 + row;
+            // publish this share (a contiguous [H_q][128] block); the share that arrives last adds them all up (in
+            // share order, so the result does not depend on which one that is)
+            constexpr int SHARE_FLOATS = HQ * 128;
+            float* blk_base = p.o_part + ((long long)s * p.n_blk + blk) * p.n_csplit * SHARE_FLOATS;
+            float* op = blk_base + (long long)cs * SHARE_FLOATS + row;
 #pragma unroll
-            for (int h = 0; h < HQ; ++h) op[(long long)h * r_pad] = acc[h];
+            for (int h = 0; h < HQ; ++h) op[h * 128] = acc[h];
             __threadfence();
             __syncwarp();   // a named barrier counts a warp once only if the warp arrives converged
             asm volatile("bar.sync 2, 128;" ::: "memory");
@@ -369,12 +372,32 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
             finish = sm.last != 0;
             if (finish) {
                 __threadfence();
-                const float* ip = p.o_part + ((long long)s * p.n_csplit * p.H_q) * r_pad + rho0 + row;
+                // The shares come in by bulk copy, a batch at a time, into the C_V stages (every MMA that read them has
+                // completed: o_full): one round trip per batch instead of one per share.
+                constexpr int PER = (P_STAGES * 2 * TILE * KC * 2) / (SHARE_FLOATS * 4);
+                float* stage = reinterpret_cast<float*>(&sm.V[0][0][0]);
 #pragma unroll
                 for (int h = 0; h < HQ; ++h) acc[h] = 0.f;
-                for (int c = 0; c < p.n_csplit; ++c) {
+                uint32_t par = 0;
+                for (int c0 = 0; c0 < p.n_csplit && ok; c0 += PER) {
+                    const int nb = min(PER, p.n_csplit - c0);
+                    if (c0 > 0) {
+                        __syncwarp();
+                        asm volatile("bar.sync 2, 128;" ::: "memory");   // everyone has added the previous batch
+                    }
+                    if (t == 0) {
+                        fence_proxy_async_all();     // the other shares' stores (seen through the counter) before the copies
+                        mbar_arrive_expect_tx(&sm.red_full, (uint32_t)(nb * SHARE_FLOATS * 4));
+                        for (int j = 0; j < nb; ++j)
+                            bulk_load(stage + j * SHARE_FLOATS, blk_base + (long long)(c0 + j) * SHARE_FLOATS,
+                                      SHARE_FLOATS * 4, &sm.red_full);
+                    }
+                    if (!mbar_wait(&sm.red_full, par)) { ok = false; break; }
+                    par ^= 1;
+                    for (int j = 0; j < nb; ++j) {
 #pragma unroll
-                    for (int h = 0; h < HQ; ++h) acc[h] += __ldcg(ip + ((long long)c * p.H_q + h) * r_pad);
+                        for (int h = 0; h < HQ; ++h) acc[h] += stage[(j * HQ + h) * 128 + row];
+                    }
                 }
             }
         } else {
@@ -563,7 +586,7 @@ struct PvScratch {
 PvScratch pv_scratch_layout(const lorc_ctx* ctx, int batch, int tiles, int n_csplit, int n_groups, size_t r_pad) {
     PvScratch z;
     const size_t hq = (size_t)ctx->desc.n_q_heads;
-    z.part_bytes = lorc_align_up((size_t)batch * n_csplit * hq * r_pad * sizeof(float), 256);
+    z.part_bytes = lorc_align_up((size_t)batch * n_csplit * hq * r_pad * sizeof(float), 256);   // [b][n_blk][n_csplit][H_q][128]
     z.l_bytes = lorc_align_up((size_t)batch * n_groups * hq * sizeof(float), 256);
     z.on_bytes = lorc_align_up((size_t)batch * hq * r_pad * sizeof(bf16), 256);
     z.prob_bytes = lorc_align_up((size_t)batch * tiles * hq * TILE * sizeof(bf16), 256);
