@@ -27,7 +27,9 @@ namespace {
 
 constexpr int TILE = 128;
 constexpr int KC = 64;
-constexpr int P_STAGES = 4;          // 4 x 40 KiB (48 KiB with 64 query heads): one CTA per SM, 160 KiB in flight
+// one CTA per SM; 5 stages x 40 KiB with 32 query heads (200 KiB in flight), 4 x 48 KiB with 64
+template <int HQ>
+struct PvStages { static constexpr int value = HQ <= 32 ? 5 : 4; };
 constexpr int P_THREADS = 192;       // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
 
 // read-only global load that the compiler keeps in program order with the other volatile asm of this file
@@ -152,6 +154,7 @@ lorc_prob_kernel(const ProbParams p) {
 // ------------------------------------------------------------------------------------------------
 template <int HQ>
 struct Pv2Smem {
+    static constexpr int P_STAGES = PvStages<HQ>::value;
     bf16 V[P_STAGES][2][TILE * KC];       // C_V block: two 64-column halves of [128 tokens][64]; 32 KiB / stage
     bf16 P[P_STAGES][2][HQ * KC];         // probabilities [HQ][128 tokens] as two 64-token chunks, 128-byte swizzle
     float red[128 / HQ][HQ];
@@ -180,6 +183,7 @@ __global__ void __launch_bounds__(P_THREADS, 1)
 lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
     extern __shared__ uint8_t raw[];
     typedef Pv2Smem<HQ> S;
+    constexpr int P_STAGES = PvStages<HQ>::value;
     S& sm = *reinterpret_cast<S*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
     constexpr uint32_t TM_COLS = HQ <= 32 ? 32 : 64;
     constexpr uint32_t P_BYTES = 2 * HQ * KC * 2;
