@@ -28,7 +28,7 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
 // factor are permuted (see retile_factor_kernel) so that the two accumulator columns a thread ends up with are the two
 // members of one rotary pair: the rotation needs no exchange between threads.
 template <bool FULL>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 2)
 append_mma_kernel(const bf16* __restrict__ x, const bf16* __restrict__ A_tiled, CacheView cv, int D, int r_k,
                   int r_v, int T, int max_pos, int* status, int d_head, int rope_style,
                   const float2* __restrict__ rope_table) {

@@ -199,6 +199,27 @@ def test_tc_append_then_decode_chain_and_host_entry():
     sess.close()
 
 
+def test_tc_decode_one_context_serves_batches_of_different_sizes():
+    """The library keeps one word per (sequence, head) for the softmax row maxima between calls, cleared by each call
+    for the next and grown when a larger batch arrives: a small batch, a larger one and the small one again, on one
+    context and one workspace, each against the oracle; queries of very different magnitudes in turn, so that a
+    maximum left over from an earlier call would show."""
+    import torch
+    prob = _prob(256, 256)
+    lens_small, lens_big = [300, 129], [64, 700, 1, 257, 513]
+    n_max = 720
+    sess = H.Session(prob, max_pos=n_max, batch=len(lens_big))
+    for it, (lens, q_scale) in enumerate([(lens_small, 64.0), (lens_big, 1.0), (lens_small, 0.25), (lens_big, 64.0)]):
+        b = len(lens)
+        ck, cv = _latents(prob, lens, 20)
+        cache, k, v, sl = H.contiguous_cache(sess, b, n_max, lens, ck, cv)
+        q = synth.queries(b, GEOM["H_q"], GEOM["d_h"], 20, 30 + it, q_scale).astype(np.float64)
+        got = H.host_f64(_run(sess, cache, q))
+        want = H.oracle_decode(prob, ck, cv, q)
+        assert O.rel_l2_rows(got, want) <= TOL, (it, O.rel_l2_rows(got, want))
+    sess.close()
+
+
 # ------------------------------------------------------------------- uncompressed reference mode, 128-wide heads
 @pytest.mark.parametrize("H_q,lens,paged", [
     (32, [700, 64, 1, 129], False),          # G = 4
