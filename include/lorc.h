@@ -168,6 +168,11 @@ int lorc_append(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* x
  * n_splits = 0 lets the library choose the split of the context; a positive value
  * forces it (clamped to what the workspace holds).  Uses the workspace.
  * A sequence with seq_lens[s] <= 0 gets a row of zeros and sets status EMPTY.
+ * The first call on a context, and the first call with a larger batch than any
+ * before, sets up small library-owned tables (an in-tile rotation table, one word
+ * per sequence and head for the softmax row maxima) with cudaMalloc: make those
+ * calls outside any stream capture.  Calls on one context must not overlap on the
+ * GPU (they share the workspace and those tables).
  * Errors: ARG, LAYER, WORKSPACE, UNSUPPORTED. */
 int lorc_decode_attn(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* q, void* out,
                      int n_splits, void* stream);
