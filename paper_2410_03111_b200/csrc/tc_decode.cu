@@ -341,8 +341,8 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
             // One 8-column step at a time.  Unrolled, so that the loads and the dependent fp32 chains of several steps
             // overlap (a scheduler has only two epilogue warps to switch between): measured per unit at rank 256,
             // 4.1 k clk not unrolled, 3.1 k by two, 2.8 k fully.  With eight query heads per KV head the registers
-            // only allow two steps.
-#pragma unroll(G == 4 ? 8 : 2)
+            // allow four steps.
+#pragma unroll(G == 4 ? 8 : 4)
             for (int kk = 0; kk < 8; ++kk) {
                 uint32_t ra[2][4], rb[2][4];
 #pragma unroll
