@@ -126,6 +126,27 @@ def test_tc_decode_matches_plain_kernels_and_split_counts():
     dbg.close()
 
 
+def test_tc_decode_many_context_shares_with_64_query_heads():
+    """Eight query heads per KV head, one sequence, one column block: the context is dealt over as many shares as it
+    has tiles, more than one bulk-copy batch of the share reduction holds (four shares of 32 KiB), so the last share
+    adds them up over several batches; forced share counts around the batch size as well."""
+    import torch
+    prob = H.Problem(GEOM["D"], 64, GEOM["H_kv"], GEOM["d_h"], 128, 128, theta=500000.0, layer=22)
+    lens = [1500]
+    ck, cv = _latents(prob, lens, 22)
+    q = synth.queries(1, 64, GEOM["d_h"], 22, 0, 16.0).astype(np.float64)
+    want = H.oracle_decode(prob, ck, cv, q)
+    sess = H.Session(prob, max_pos=1536, batch=1)
+    cache, k, v, sl = H.contiguous_cache(sess, 1, 1536, lens, ck, cv)
+    for S in (0, 1, 4, 5, 9, 12):
+        out = torch.zeros(1, 64, GEOM["d_h"], dtype=torch.bfloat16, device="cuda")
+        sess.L.lorc_decode_attn(sess.ctx, 0, cache, H.dev_bf16(q), out, n_splits=S)
+        assert sess.L.lorc_sync_status(sess.ctx) == 0, sess.L.lorc_last_error(sess.ctx)
+        assert sess.L.lorc_last_path(sess.ctx) == 2, "the tensor-core path was not taken"
+        assert O.rel_l2_rows(H.host_f64(out), want) <= TOL, S
+    sess.close()
+
+
 @pytest.mark.parametrize("page_size", [64, 16, 128])
 def test_tc_decode_paged_and_page_permutation(page_size):
     import torch
