@@ -340,9 +340,9 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
             const uint64_t minus1 = f2_pack(-1.f, -1.f);
             // One 8-column step at a time.  Unrolled, so that the loads and the dependent fp32 chains of several steps
             // overlap (a scheduler has only two epilogue warps to switch between): measured per unit at rank 256,
-            // 4.1 k clk not unrolled, 3.1 k by two, 2.8 k fully.  With eight query heads per KV head the registers
-            // allow four steps.
-#pragma unroll(G == 4 ? 8 : 4)
+            // 4.1 k clk not unrolled, 3.1 k by two, 2.8 k fully (165 registers, no spills, with four or eight query
+            // heads per KV head).
+#pragma unroll
             for (int kk = 0; kk < 8; ++kk) {
                 uint32_t ra[2][4], rb[2][4];
 #pragma unroll
