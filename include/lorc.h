@@ -60,9 +60,10 @@ extern "C" {
 
 /* stages reported by lorc_profile_read */
 #define LORC_STAGE_APPEND 0     /* cache write */
-#define LORC_STAGE_SCORE 1      /* key reconstruction + RoPE + scores (tensor-core path) or the whole plain kernel */
-#define LORC_STAGE_PV 2         /* softmax + P.C_V */
-#define LORC_STAGE_COMBINE 3    /* split merge + value up-projection */
+#define LORC_STAGE_SCORE 1      /* tensor-core path: key reconstruction + RoPE + scores + softmax numerators;
+                                   plain kernels: the whole split-context attention kernel */
+#define LORC_STAGE_PV 2         /* tensor-core path: change of softmax reference + P.C_V */
+#define LORC_STAGE_COMBINE 3    /* value up-projection (plain kernels: split merge + up-projection) */
 #define LORC_N_STAGES 4
 
 typedef struct lorc_ctx lorc_ctx;
@@ -97,10 +98,13 @@ typedef struct lorc_model_desc {
  *
  * seq_lens[batch] (device int32, caller-owned, never written by the library) is
  * the number of cached tokens of each sequence.  max_seq_len is a host-side upper
- * bound on seq_lens used to size launches; it must not exceed the capacity
- * (seq_stride, or max_pages_per_seq*page_size).  Rows at positions >= seq_lens[s]
- * may be read by tile loads; they must hold finite numbers (zero the cache once
- * when allocating it). */
+ * bound on seq_lens used to size launches and scratch; it must not exceed the
+ * capacity (seq_stride, or max_pages_per_seq*page_size).  The kernels enforce
+ * seq_lens[s] <= max_seq_len (rounded up to a multiple of 128 on the tensor-core
+ * path) and seq_lens[s] <= max_pos: a longer sequence is treated as empty and the
+ * status word is set to LORC_ERR_CAPACITY; nothing is read or written out of
+ * bounds.  Rows at positions >= seq_lens[s] may be read by tile loads; they must
+ * hold finite numbers (zero the cache once when allocating it). */
 typedef struct lorc_cache {
     void* k;                      /* device */
     void* v;                      /* device */
@@ -165,14 +169,18 @@ int lorc_append(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* x
  *   k_n = B_K[:, g]^T C_K[n], rotated at n;  q^ = RoPE(q, seq_lens[s]-1);
  *   p = softmax_n(q^ . k_n / sqrt(d_head)),  out = (sum_n p_n C_V[n]) B_V[:, g]
  * over n in [0, seq_lens[s]).  Keys and values are never written to memory.
- * n_splits = 0 lets the library choose the split of the context; a positive value
- * forces it (clamped to what the workspace holds).  Uses the workspace.
+ * n_splits = 0 lets the library choose how many CTAs share one sequence's context;
+ * a positive value asks for that many shares (context splits of the plain kernels
+ * and of the uncompressed mode; context shares per latent column block of the
+ * tensor-core path), clamped to what the workspace holds.  Uses the workspace.
  * A sequence with seq_lens[s] <= 0 gets a row of zeros and sets status EMPTY.
  * The first call on a context, and the first call with a larger batch than any
  * before, sets up small library-owned tables (an in-tile rotation table, one word
  * per sequence and head for the softmax row maxima) with cudaMalloc: make those
- * calls outside any stream capture.  Calls on one context must not overlap on the
- * GPU (they share the workspace and those tables).
+ * calls outside any stream capture.  A table handed to earlier calls is kept until
+ * lorc_destroy, so CUDA graphs captured before a larger batch showed up stay valid.
+ * Calls on one context must not overlap on the GPU (they share the workspace and
+ * those tables).
  * Errors: ARG, LAYER, WORKSPACE, UNSUPPORTED. */
 int lorc_decode_attn(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* q, void* out,
                      int n_splits, void* stream);
@@ -182,7 +190,9 @@ int lorc_decode_attn(lorc_ctx* ctx, int layer, const lorc_cache* cache, const vo
  * Meant for hosts that cannot allocate device memory when they call in: a server
  * that gave the whole GPU to its own memory pool at start-up, or a plug-in that
  * receives tensors but no allocator.  Same arguments, meaning and result as
- * lorc_decode_attn, computed by the plain CUDA-core kernels, but the per-split
+ * lorc_decode_attn, computed by the split-context kernels (the plain CUDA-core
+ * ones; for an uncompressed layer with 128-wide heads the mma.sync streaming
+ * kernel, as lorc_last_path reports), but the per-split
  * partial results live in a fixed array of LORC_STATIC_SCRATCH_BYTES inside the
  * library (each GPU that loads the library holds that much until the process
  * ends).  The call performs no cudaMalloc/cudaFree and ignores the workspace.

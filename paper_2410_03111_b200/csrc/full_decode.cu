@@ -285,12 +285,15 @@ cudaError_t lorc_full_decode(const lorc_ctx* ctx, const CacheView& cv, const bf1
                              float* part_o, cudaStream_t st, int* launches) {
     const lorc_model_desc& d = ctx->desc;
     dim3 grid(n_splits, d.n_kv_heads, cv.batch);
-    static bool attr = false;
-    if (!attr) {
+    // the attribute belongs to a device's copy of the kernel: one flag per device (devices beyond the table set it
+    // on every call, which is only slower)
+    static bool attr[64] = {false};
+    const bool known = ctx->device >= 0 && ctx->device < 64;
+    if (!known || !attr[ctx->device]) {
         cudaError_t e = cudaFuncSetAttribute(full_decode_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)sizeof(FdSmem));
         if (e != cudaSuccess) return e;
-        attr = true;
+        if (known) attr[ctx->device] = true;
     }
     full_decode_mma_kernel<<<grid, 128, sizeof(FdSmem), st>>>(q, cv, ctx->group, n_splits, d.rope_style, ctx->rope_table, d.max_pos,
                                                  part_ml, part_o, ctx->status_dev);

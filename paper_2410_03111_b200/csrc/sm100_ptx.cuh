@@ -271,7 +271,6 @@ __device__ __forceinline__ void tmem_ld16x256_x1(uint32_t taddr, uint32_t (&r)[4
 }
 
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ bool elect_one() {
     uint32_t pred;

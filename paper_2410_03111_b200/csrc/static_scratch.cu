@@ -113,7 +113,7 @@ extern "C" int lorc_decode_attn_static(lorc_ctx* ctx, int layer, const lorc_cach
     e = lorc_generic_decode(ctx, L, cv, (const bf16*)q, (bf16*)out, S, part_ml, part_o, (cudaStream_t)stream,
                             &launches);
     ctx->launches += launches;
-    ctx->last_path = 1;
+    ctx->last_path = lorc_full_decode_supported(ctx, L) ? 3 : 1;
     if (e != cudaSuccess) {
         ctx->err = std::string("decode_attn_static: ") + cudaGetErrorString(e);
         return LORC_ERR_CUDA;

@@ -18,16 +18,37 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
 cudaError_t lorc_tc_append(lorc_ctx* ctx, int layer, const LorcLayer& L, const CacheView& cv,
                            const bf16* x, int T, cudaStream_t st, int* launches);
 
-// Softmax + P.C_V and value up-projection (tc_pv.cu).  scores [b, H_q, n_pad] (log2 units) and
-// rowmax [b, H_q] (exact row maxima as order-preserving keys, see lorc_float_key; the PV kernel zeroes them again)
-// come from the score kernel.
-// mapCV: C_V cache in 64-column x 128-row (or page-sized) swizzled boxes; mapBVT: B_V^T [n, r_v] in swizzled
-// boxes of 64 latent columns x 32 rows.  Launches the PV kernel and the up-projection kernel that writes `out`.
+// Bytes of one probability tile image (128 tokens of one sequence, all query heads): the bf16 numerators as the PV
+// kernel's swizzled MMA operand, then float m[4][H_q] and float l[4][H_q] (reference and sum per 32-token quarter).
+__host__ __device__ inline int lorc_tc_image_bytes(int n_q_heads) { return 2 * n_q_heads * 64 * 2 + 8 * n_q_heads * 4; }
+
+// Score kernel (tc_score.cu): key reconstruction, rotation, q.k and the softmax numerators; writes one tile image per
+// 128 tokens into pimg [b, tiles, image] and raises the row maxima (integers, as order-preserving keys).  rope_tile:
+// the in-tile rotation table (33 x 32 float4, lorc_tc_rope_tile_fill).  Its first block clears zero[0 .. n_zero).
+#define LORC_SCORE_MAX_BATCH 128     // sequences per launch (larger batches take several launches)
+cudaError_t lorc_tc_score_set_attrs();
+cudaError_t lorc_tc_rope_tile_fill(float2* table, double theta, cudaStream_t st);
+cudaError_t lorc_tc_score_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, const CUtensorMap& mapCK,
+                                 const CUtensorMap& mapBKT, const bf16* q, uint8_t* pimg, unsigned* rowmax,
+                                 const float4* rope_tile, int tiles, int* zero, int n_zero, cudaStream_t st,
+                                 int* launches);
+
+// P.C_V and value up-projection (tc_pv.cu).  mapCV: C_V cache in 64-column x 128-row (or page-sized) swizzled boxes;
+// mapBVT: B_V^T [n, r_v] in swizzled boxes of 64 latent columns x 32 rows.  The plan says how a launch splits the
+// work and where its pieces of scratch lie; the `done` words (plan.n_blk * batch ints at off_done) must be zero when
+// the PV kernel starts.  The up-projection kernel writes `out` and leaves the row maxima empty again.
+struct LorcPvPlan {
+    int n_blk, n_csplit;
+    bool fits;
+    size_t off_on, off_done;
+};
 size_t lorc_tc_pv_scratch_bytes(const lorc_ctx* ctx, int batch, int max_seq_len);
+cudaError_t lorc_tc_pv_set_attrs();
+void lorc_tc_pv_plan(const lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, int n_splits_hint, size_t scratch_bytes,
+                     LorcPvPlan* plan);
 cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, const CUtensorMap& mapCV,
-                              const CUtensorMap& mapBVT, const float* scores, unsigned* rowmax, int n_pad, int tiles,
-                              int n_splits_hint, void* scratch, size_t scratch_bytes, bf16* out, cudaStream_t st,
-                              int* launches);
+                              const CUtensorMap& mapBVT, const uint8_t* pimg, unsigned* rowmax, int tiles,
+                              const LorcPvPlan& plan, void* scratch, bf16* out, cudaStream_t st, int* launches);
 
 // A_cat [D, R] (row-major) -> fragment order [R/8][D/32][32 lanes][8] used by the fast append kernel.  The first
 // pair_cols columns (uncompressed mode with half-split rotary pairs: the key columns; otherwise 0) are laid out with the
