@@ -48,14 +48,17 @@ def parse_args():
     ap.add_argument("--no-graph", action="store_true", help="launch call by call instead of replaying a CUDA graph")
     ap.add_argument("--stages", action="store_true",
                     help="call-by-call launches with per-kernel CUDA events; adds a 'stages' object (ms per step)")
+    ap.add_argument("--no-full-rank-leg", action="store_true",
+                    help="skip the 'full_rank' object (the uncompressed mode timed on the same shape in the same run)")
+    ap.add_argument("--no-other-configs", action="store_true",
+                    help="skip the 'other_configs' object (attention time of the other configurations, a few steps each)")
     return ap.parse_args()
 
 
-# DRAM traffic of one lorc_score_kernel launch, from the ncu capture summarised in
-# profiles/attention_kernels_cfg2_layers0-1.md (set to None once the kernel has changed since that capture).  The
-# capture is of the layer with rank 928; the read traffic is the latent keys, which grow with rank, batch and
-# context, the written traffic the scores, which grow with batch and context only.
-SCORE_KERNEL_TRAFFIC = {"read_bytes": 127.69e6, "write_bytes": 8.53e6, "rank": 928, "batch": 16, "context": 4100}
+# DRAM traffic of one lorc_score_kernel launch from an ncu capture of the CURRENT kernel (rank, batch and context of the
+# captured launch; the read traffic is the latent keys, which grow with rank, batch and context, the written traffic
+# the probability images, which grow with batch and context only).  None: no capture of the current kernel yet.
+SCORE_KERNEL_TRAFFIC = None
 
 
 def load_peaks():
@@ -63,8 +66,21 @@ def load_peaks():
     if os.path.exists(p):
         d = json.load(open(p))
         return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
-                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
-    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]),
+                "sustained_sm_mhz": (d.get("clocks_under_load") or {}).get("sm_mhz_median"), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "sustained_sm_mhz": 1300.0,
+            "source": "fallback"}
+
+
+def pick_tensor_peak(peaks, timed_region_s, clocks):
+    """Which bf16 peak a tensor-bound fraction is quoted against.  The burst figure unless the evidence says the run
+    sat in the regime the sustained figure was measured in: a timed region of at least a second AND a sampled SM
+    clock under load within 10 % of the clock the sustained peak was measured at."""
+    sm = (clocks or {}).get("sm_mhz")
+    ref = peaks.get("sustained_sm_mhz")
+    if timed_region_s >= 1.0 and sm and ref and sm <= 1.1 * ref:
+        return "sustained", peaks["bf16_tflops_sustained"]
+    return "burst", peaks["bf16_tflops"]
 
 
 # --------------------------------------------------------------------------- clocks
@@ -177,41 +193,77 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------ workload set-up
-def algorithmic_counts(shape, ranks, batch, n_ctx):
+def algorithmic_counts(shape, ranks, batch, tokens):
     """Per decode step over all layers: tensor-eligible FLOPs and latent+factor bytes of
-    lorc_decode_attn with every sequence holding n_ctx tokens."""
+    lorc_decode_attn with `tokens` cached tokens in total over the `batch` sequences."""
     n, Hq, dh = shape.n, shape.n_q_heads, shape.d_head
     flops = 0.0
     byts = 0.0
     for r in ranks:
         per_tok = 2.0 * r * n + 2.0 * Hq * dh + 2.0 * Hq * r
-        flops += batch * n_ctx * per_tok + batch * 2.0 * Hq * r * dh
-        byts += batch * n_ctx * 2.0 * (r + r) + 2.0 * (r + r) * n + 4.0 * batch * Hq * dh
+        flops += tokens * per_tok + batch * 2.0 * Hq * r * dh
+        byts += tokens * 2.0 * (r + r) + 2.0 * (r + r) * n + 4.0 * batch * Hq * dh
     return flops, byts
 
 
-class Workload:
-    """Factors, prefilled latent caches and per-step inputs of one configuration on one GPU."""
+def full_rank_counts(shape, n_layers, batch, tokens):
+    """The same for the uncompressed mode: scores and PV over whole keys and values, 2 n bf16 numbers read per token."""
+    n, Hq, dh = shape.n, shape.n_q_heads, shape.d_head
+    return n_layers * tokens * 4.0 * Hq * dh, n_layers * (tokens * 2.0 * 2.0 * n + 4.0 * batch * Hq * dh)
 
-    def __init__(self, L, shape, n_layers, total_steps, device, flags, full_rank=False):
+
+class Workload:
+    """Factors, filled latent caches and per-step inputs of one configuration on one GPU."""
+
+    def __init__(self, L, shape, n_layers, total_steps, device, flags, full_rank=False, seeded_cache=False,
+                 keep_layers=(), layer_ids=None):
+        """seeded_cache: fill the caches with seeded synthetic rows instead of running the prompt through
+        lorc_append (ragged paged configurations, and the short legs that only time attention).
+        keep_layers: layers whose bf16 factors are also kept on the host (for the oracle leg).
+        layer_ids: which layers of the configuration to build (default: the first n_layers); layer i of the context
+        is layer layer_ids[i] of the configuration (its rank, its seeded weights and inputs)."""
         import torch
         from paper_2410_03111_b200 import host
         from workloads import device as wdev
+        from workloads import synth
         self.L, self.shape, self.torch = L, shape, torch
+        self.layer_ids = list(layer_ids) if layer_ids is not None else list(range(n_layers))
+        n_layers = len(self.layer_ids)
         self.n_layers = n_layers
-        self.ranks = shape.ranks[:n_layers]
+        self.ranks = [shape.ranks[i] for i in self.layer_ids]
+        self.full_rank = full_rank
         b, N = shape.batch, shape.context
         self.batch = b
-        self.n_max = ((N + total_steps + 127) // 128) * 128
+        lo, hi = shape.ragged
+        if hi > 0:
+            self.lens0 = [int(x) for x in synth.ragged_lengths(b, lo, hi)]
+        else:
+            self.lens0 = [N] * b
+        self.tokens0 = sum(self.lens0)
+        self.n_max = ((max(self.lens0) + total_steps + 127) // 128) * 128
         self.ctx = L.lorc_create(n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.d_head,
                                  shape.rope_theta, max_pos=self.n_max, flags=flags)
-        self.caches, self.keep = [], []
+        self.caches, self.keep, self.host_factors = [], [], {}
         self.seq_lens = torch.zeros(b, dtype=torch.int32, device=device)
+        self.page_table = None
+        if shape.paged:
+            ps = shape.page_size
+            self.max_pages = self.n_max // ps
+            pages = [(l + total_steps + ps - 1) // ps for l in self.lens0]
+            self.n_pages = sum(pages)
+            order = synth.page_order(self.n_pages)
+            pt = torch.zeros(b, self.max_pages, dtype=torch.int32)
+            k0 = 0
+            for s_, np_ in enumerate(pages):
+                pt[s_, :np_] = torch.from_numpy(order[k0:k0 + np_].astype("int32"))
+                k0 += np_
+            self.page_table = pt.to(device)
         chunk = 512
         for l in range(n_layers):
             r = self.ranks[l]
-            Uk, sk, Vk = wdev.weight_generators(shape.d_model, shape.n, shape.sigma_p, l, "k", device)
-            Uv, sv, Vv = wdev.weight_generators(shape.d_model, shape.n, shape.sigma_p, l, "v", device)
+            lid = self.layer_ids[l]
+            Uk, sk, Vk = wdev.weight_generators(shape.d_model, shape.n, shape.sigma_p, lid, "k", device)
+            Uv, sv, Vv = wdev.weight_generators(shape.d_model, shape.n, shape.sigma_p, lid, "v", device)
             if full_rank:
                 # the uncompressed mode takes the dense weights; its cache rows are whole keys and values
                 Ak, Av = host.dense_weight(Uk, sk, Vk), host.dense_weight(Uv, sv, Vv)
@@ -222,33 +274,62 @@ class Workload:
                 Ak, Bk = host.factors_from_svd(Uk, sk, Vk, r)
                 Av, Bv = host.factors_from_svd(Uv, sv, Vv, r)
                 L.lorc_load_factors(self.ctx, l, L.LORC_MODE_LATENT, r, r, Ak, Bk, Av, Bv)
-            k = torch.zeros(b, self.n_max, r, dtype=torch.bfloat16, device=device)
-            v = torch.zeros(b, self.n_max, r, dtype=torch.bfloat16, device=device)
+                if l in keep_layers:
+                    self.host_factors[l] = tuple(t.float().cpu().numpy().astype("float64") for t in (Ak, Av, Bk, Bv))
+            if shape.paged:
+                shp = (self.n_pages, shape.page_size, r)
+            else:
+                shp = (b, self.n_max, r)
+            if seeded_cache:
+                k = wdev.latents(shp, shape.sigma_p, lid, "k", device)
+                v = wdev.latents(shp, shape.sigma_p, lid, "v", device)
+            else:
+                k = torch.zeros(*shp, dtype=torch.bfloat16, device=device)
+                v = torch.zeros(*shp, dtype=torch.bfloat16, device=device)
             self.keep.append((k, v))
-            self.caches.append(L.make_cache(k, v, self.seq_lens, b, self.n_max, seq_stride=self.n_max))
+            if shape.paged:
+                self.caches.append(L.make_cache(k, v, self.seq_lens, b, self.n_max, page_table=self.page_table,
+                                                page_size=shape.page_size, max_pages_per_seq=self.max_pages,
+                                                n_pages=self.n_pages))
+            else:
+                self.caches.append(L.make_cache(k, v, self.seq_lens, b, self.n_max, seq_stride=self.n_max))
             del Uk, Vk, Uv, Vv, Ak, Bk, Av, Bv
-        # prefill through the library's own cache write, in chunks
-        done = 0
-        while done < N:
-            T = min(chunk, N - done)
-            self.seq_lens.fill_(done + T)
-            for l in range(n_layers):
-                x = wdev.hidden_states((b, T, shape.d_model), l, done // chunk, device)
-                L.lorc_append(self.ctx, l, self.caches[l], x, T=T)
-            done += T
+        if seeded_cache:
+            self.seq_lens.copy_(torch.tensor(self.lens0, dtype=torch.int32))
+        else:
+            # prefill through the library's own cache write, in chunks
+            done = 0
+            while done < N:
+                T = min(chunk, N - done)
+                self.seq_lens.fill_(done + T)
+                for l in range(n_layers):
+                    x = wdev.hidden_states((b, T, shape.d_model), self.layer_ids[l], done // chunk, device)
+                    L.lorc_append(self.ctx, l, self.caches[l], x, T=T)
+                done += T
         torch.cuda.synchronize()
         rc = L.lorc_sync_status(self.ctx)
         if rc:
             raise RuntimeError(f"prefill failed: {L.lorc_last_error(self.ctx)}")
         # per-step inputs: a fresh token and a fresh query per layer and step
-        self.x = [wdev.hidden_states((total_steps, b, shape.d_model), l, 10 ** 6, device) for l in range(n_layers)]
-        self.q = [wdev.queries((total_steps, b, shape.n_q_heads, shape.d_head), l, 0, device, 8.0)
-                  for l in range(n_layers)]
+        self.x = [wdev.hidden_states((total_steps, b, shape.d_model), lid, 10 ** 6, device) for lid in self.layer_ids]
+        self.q = [wdev.queries((total_steps, b, shape.n_q_heads, shape.d_head), lid, 0, device, 8.0)
+                  for lid in self.layer_ids]
         self.out = torch.zeros(n_layers, b, shape.n_q_heads, shape.d_head, dtype=torch.bfloat16, device=device)
         ws_bytes = L.lorc_workspace_bytes(self.ctx, b, self.n_max)
         self.ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=device)
         L.lorc_set_workspace(self.ctx, self.ws)
         self.step_index = 0
+
+    def close(self):
+        """Release the context and every device buffer of this workload."""
+        torch = self.torch
+        torch.cuda.synchronize()
+        self.L.lorc_destroy(self.ctx)
+        for name in ("caches", "keep", "x", "q", "out", "ws", "x_cur", "q_cur", "x_all", "q_all", "g_attn", "g_step",
+                     "seq_lens", "page_table"):
+            if hasattr(self, name):
+                setattr(self, name, None)
+        torch.cuda.empty_cache()
 
     def _layers(self, xs, qs, append=True, attn=True):
         L = self.L
@@ -307,9 +388,74 @@ class Workload:
 
 
 # ------------------------------------------------------------------- CPU baseline
+def oracle_leg(wl, shape, layers, budget_s=15.0):
+    """The cpu_baseline leg: the fp64 oracle, as it stands, redoes whole (layer, sequence) units of the workload the
+    GPU just ran: the append of the last token and decode attention over the sequence's cache rows, read back from
+    the device.  It is timed, and because it works on the real inputs its result is also compared with the GPU's
+    output for the same unit (the 'parity' object).  Returns (seconds per unit-rank, description, threads, parity)."""
+    import numpy as np
+    from oracle import lorc_oracle as O
+    torch = wl.torch
+    L = wl.L
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    # one more attention call per sampled layer, so that `out` is known to belong to the query and cache used below
+    step = wl.step_index - 1
+    for l in layers:
+        L.lorc_decode_attn(wl.ctx, l, wl.caches[l], wl.q[l][step], wl.out[l])
+    torch.cuda.synchronize()
+    lens = [int(v) for v in wl.seq_lens.cpu().tolist()]
+    t_total, r_total, units, worst, worst_at = 0.0, 0, 0, 0.0, None
+    seq = 0
+    while t_total < budget_s and seq < wl.batch:
+        for l in layers:
+            r = wl.ranks[l]
+            Ak, Av, Bk, Bv = wl.host_factors[l]
+            n = lens[seq]
+            k, v = wl.keep[l]
+            if wl.page_table is not None:
+                pages = wl.page_table[seq, :(n + shape.page_size - 1) // shape.page_size].long()
+                k, v = k[pages].reshape(-1, r)[None], v[pages].reshape(-1, r)[None]
+                ck = k[0, :n].float().cpu().numpy().astype(np.float64)
+                cv = v[0, :n].float().cpu().numpy().astype(np.float64)
+            else:
+                ck = k[seq, :n].float().cpu().numpy().astype(np.float64)
+                cv = v[seq, :n].float().cpu().numpy().astype(np.float64)
+            x = wl.x[l][step][seq:seq + 1].float().cpu().numpy().astype(np.float64)
+            q = wl.q[l][step][seq].float().cpu().numpy().astype(np.float64)
+            got = wl.out[l][seq].float().cpu().numpy().astype(np.float64)
+            t0 = time.perf_counter()
+            row_k = O.append_latent_bf16(x, Ak)[0]
+            row_v = O.append_latent_bf16(x, Av)[0]
+            want = O.decode_attn_latent(ck, cv, Bk, Bv, q, shape.n_kv_heads, shape.rope_theta)
+            t_total += time.perf_counter() - t0
+            # the cache row the GPU wrote for this token against the oracle's (exactly rounded) one, in bf16 ulps
+            ulp = float(np.max(np.abs(np.concatenate([row_k - ck[n - 1], row_v - cv[n - 1]])) /
+                               np.maximum(np.abs(np.concatenate([row_k, row_v])) * 2.0 ** -8, 1e-30)))
+            err = float(O.rel_l2_rows(got, want))
+            if err > worst:
+                worst, worst_at = err, (l, seq)
+            r_total += r
+            units += 1
+            if t_total > budget_s:
+                break
+        seq += 1
+    desc = (f"{units} (layer, sequence) units of {shape.name} ({t_total:.1f} s of oracle time): layers {sorted(set(layers))}, "
+            f"their real cache rows read back from the device, append of the last token + decode attention; scaled "
+            f"to the step by rank (time per unit proportional to r_l) and by the batch")
+    parity = {"max_rel_l2_row_error": worst, "tolerance": 1e-2, "units": units, "worst_unit_layer_seq": worst_at,
+              "append_last_row_max_err_bf16_ulp": ulp,
+              "what": "GPU output vs the fp64 oracle on the sampled units, max over (sequence, head) rows of "
+                      "||gpu - oracle||_2 / ||oracle||_2; taken outside the timed region"}
+    return t_total / r_total, desc, threads, parity
+
+
 def oracle_sample(shape, n_layers, budget_s=15.0, layers=None, n_ctx=None):
-    """Time the fp64 oracle on a bounded sample of the workload: whole (layer, sequence)
-    units (one new token appended, then decode attention over the full context).
+    """The reference arm's sample: time the fp64 oracle on whole (layer, sequence) units with the workload's shapes
+    (one new token appended, then decode attention over the full context), on synthetic inputs drawn on the host.
     Returns (seconds per unit-rank, description, threads used, units timed)."""
     import numpy as np
     from oracle import lorc_oracle as O
@@ -353,7 +499,8 @@ def oracle_sample(shape, n_layers, budget_s=15.0, layers=None, n_ctx=None):
                 break
         seq += 1
     layers = sorted(set(used))
-    desc = (f"{units} (layer, sequence) units of {shape.name} ({t_total:.1f} s of oracle time): layers {layers}, "
+    desc = (f"{units} (layer, sequence) units of {shape.name} ({t_total:.1f} s of oracle time; the time per unit varies "
+            f"by a few tens of percent from sample to sample): layers {layers}, "
             f"context {N}+1, append of 1 token + decode attention; scaled to the step by rank "
             f"(time per unit proportional to r_l) and by the batch")
     return t_total / r_total, desc, threads, units
@@ -400,6 +547,77 @@ def whole_job_rate(batch, steps, world, seconds):
 
 
 # --------------------------------------------------------------------------- main
+def time_attention(wl, reps, use_graph):
+    """Device milliseconds of the attention calls of all layers (one decode step's worth), averaged over reps."""
+    torch = wl.torch
+
+    def attn_only():
+        if use_graph:
+            wl.g_attn.replay()
+        else:
+            wl._layers(None, [q[0] for q in wl.q], append=False)
+    attn_only()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        attn_only()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def attention_leg(L, shape, device, peaks, full_rank=False, steps=4, warmup=3, n_layers=None):
+    """A short, separate run of another configuration (or of the uncompressed mode): builds the workload with
+    seeded cache rows, replays `steps` whole decode steps and the attention calls alone, and reports times and
+    roofline fractions.  Everything of it is released before it returns."""
+    import torch
+    n_layers = n_layers or shape.n_layers
+    wl = Workload(L, shape, n_layers, warmup + steps + 3, device, 0, full_rank=full_rank, seeded_cache=True)
+    try:
+        wl.step()
+        torch.cuda.synchronize()
+        wl.capture()
+        for _ in range(warmup):
+            wl.step_graph()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            wl.step_graph()
+        e1.record()
+        torch.cuda.synchronize()
+        step_ms = e0.elapsed_time(e1) / steps
+        attn_ms = time_attention(wl, max(3, steps), True)
+        path = L.lorc_last_path(wl.ctx)
+        rc = L.lorc_sync_status(wl.ctx)
+        if rc:
+            raise RuntimeError(f"device status {rc}: {L.lorc_last_error(wl.ctx)}")
+        tokens = wl.tokens0 + wl.batch * (1 + warmup + steps)
+        if full_rank:
+            flops, byts = full_rank_counts(shape, n_layers, wl.batch, tokens)
+        else:
+            flops, byts = algorithmic_counts(shape, wl.ranks, wl.batch, tokens)
+        t_hbm = byts / (peaks["hbm_gbs"] * 1e9) * 1e3
+        t_burst = flops / (peaks["bf16_tflops"] * 1e12) * 1e3
+        t_sust = flops / (peaks["bf16_tflops_sustained"] * 1e12) * 1e3
+        return {
+            "workload": shape.name, "layers": n_layers, "batch": wl.batch, "cached_tokens": tokens,
+            "mode": "full-rank reference (uncompressed KV cache)" if full_rank else "latent",
+            "kernel_path": {1: "plain fp32 CUDA-core", 2: "tcgen05", 3: "mma.sync streaming kernel"}.get(path, str(path)),
+            "step_ms": step_ms, "tokens_per_s": wl.batch / (step_ms * 1e-3),
+            "attn_ms_per_step": attn_ms, "attn_tokens_per_s": wl.batch / (attn_ms * 1e-3),
+            "bytes_per_step": byts, "flops_per_step": flops, "hbm_gbs": byts / (attn_ms * 1e-3) / 1e9,
+            "achieved_tflops": flops / (attn_ms * 1e-3) / 1e12,
+            "bound": "hbm" if t_hbm >= t_burst else "tensor",
+            "frac_of_roofline_burst": max(t_hbm, t_burst) / attn_ms,
+            "frac_of_roofline_sustained": max(t_hbm, t_sust) / attn_ms,
+            "steps": steps, "cache": "seeded rows",
+        }
+    finally:
+        wl.close()
+
+
 def main():
     args = parse_args()
     from workloads import synth
@@ -434,7 +652,10 @@ def main():
         args.no_graph = True
     e2e_steps = 0 if args.no_e2e else max(2, min(args.steps, 8))
     total_steps = args.warmup + args.steps + e2e_steps + 4
-    wl = Workload(L, shape, n_layers, total_steps, device, flags, full_rank=args.full_rank)
+    do_oracle = (not args.no_cpu_baseline) and rank == 0 and world == 1 and not args.full_rank
+    oracle_layers = sorted(set([0, n_layers // 2, n_layers - 1])) if do_oracle else []
+    wl = Workload(L, shape, n_layers, total_steps, device, flags, full_rank=args.full_rank,
+                  seeded_cache=bool(shape.paged or shape.ragged[1] > 0), keep_layers=oracle_layers)
     b = shape.batch
 
     def barrier():
@@ -461,7 +682,6 @@ def main():
     sampler = ClockSampler(local_rank)
     sampler.start()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    n_ctx_start = shape.context + 1 + args.warmup
     ev0.record()
     for _ in range(args.steps):
         do_step()
@@ -474,22 +694,10 @@ def main():
                   for k, v in L.lorc_profile_read(wl.ctx).items()}
     launches_per_step = wl.launches_per_step if use_graph else (L.lorc_launch_count(wl.ctx) - launches0) / args.steps
     # the attention calls alone (all layers), on the cache as it stands after the timed steps
-    ea0, ea1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     attn_reps = max(3, min(args.steps, 16))
-    def attn_only():
-        if use_graph:
-            wl.g_attn.replay()
-        else:
-            wl._layers(None, [q[0] for q in wl.q], append=False)
-    attn_only()
-    torch.cuda.synchronize()
-    ea0.record()
-    for _ in range(attn_reps):
-        attn_only()
-    ea1.record()
+    attn_ms_step = time_attention(wl, attn_reps, use_graph)
     barrier()
     clocks = sampler.stop()
-    attn_ms = ea0.elapsed_time(ea1) / attn_reps * args.steps
     # the dominant kernel alone: the same attention calls again, launched one by one with a CUDA event before and
     # after every kernel on the launching stream (the library's own stage bracketing)
     score_prof = None
@@ -510,6 +718,14 @@ def main():
     if rc:
         raise RuntimeError(f"device status {rc}: {L.lorc_last_error(wl.ctx)}")
     launches = int(round(launches_per_step * args.steps))
+    tokens_mid = wl.tokens0 + b * (1 + args.warmup + args.steps)      # cached tokens the attention-only pass sees
+
+    # the oracle on the units the GPU just ran: CPU baseline and observed parity (rank 0 of a 1-GPU run only)
+    cpu = None
+    if do_oracle:
+        per_rank, desc, threads, parity = oracle_leg(wl, shape, oracle_layers)
+        step_s = per_rank * sum(wl.ranks) * b
+        cpu = ({"value": b / step_s, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}, parity)
 
     # end-to-end: host buffers in, host buffers out, every step
     e2e = None
@@ -531,59 +747,85 @@ def main():
         d2h = n_layers * oh[0].numel() * 2
         e2e = (e2e_s, h2d, d2h)
 
-    ms, attn_ms, e2e_s = max_over_ranks([ms, attn_ms, e2e[0] if e2e else 0.0], dist, device)
+    ms, attn_ms_step, e2e_s = max_over_ranks([ms, attn_ms_step, e2e[0] if e2e else 0.0], dist, device)
+    ranks_used = list(wl.ranks)
+    wl.close()
+
+    # the uncompressed mode on the same shape, and the other configurations, a few steps each (1-GPU runs only)
+    full_leg, others = None, None
+    if rank == 0 and world == 1 and not args.full_rank and not args.debug_fp32 and args.layers == 0:
+        if not args.no_full_rank_leg:
+            try:
+                full_leg = attention_leg(L, shape, device, peaks, full_rank=True, steps=4)
+            except Exception as exc:
+                full_leg = {"error": str(exc)[:200]}
+        if not args.no_other_configs:
+            others = {}
+            for name in ("cfg3_8b_long", "cfg4_70b_progressive", "cfg5_ragged_r256", "cfg5_ragged_r128"):
+                if name == shape.name:
+                    continue
+                try:
+                    others[name] = attention_leg(L, synth.CONFIGS[name], device, peaks, steps=4)
+                except Exception as exc:
+                    others[name] = {"error": str(exc)[:200]}
 
     if rank == 0:
         value = whole_job_rate(b, args.steps, world, ms * 1e-3)
-        n_ctx_mid = n_ctx_start + args.steps      # context the attention-only pass sees
-        flops, byts = algorithmic_counts(shape, wl.ranks, b, n_ctx_mid)
         if args.full_rank:
-            # uncompressed mode: scores and PV over whole keys and values, 2 n bf16 numbers read per token
-            n, Hq, dh = shape.n, shape.n_q_heads, shape.d_head
-            flops = len(wl.ranks) * b * n_ctx_mid * 4.0 * Hq * dh
-            byts = len(wl.ranks) * (b * n_ctx_mid * 2.0 * 2.0 * n + 4.0 * b * Hq * dh)
-        attn_ms_step = attn_ms / args.steps
-        t_tc = flops / (peaks["bf16_tflops_sustained"] * 1e12)
+            flops, byts = full_rank_counts(shape, n_layers, b, tokens_mid)
+        else:
+            flops, byts = algorithmic_counts(shape, ranks_used, b, tokens_mid)
+        timed_s = ms * 1e-3
+        which, tc_peak = pick_tensor_peak(peaks, timed_s, clocks)
         t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
+        t_tc = flops / (tc_peak * 1e12)
+        t_burst = flops / (peaks["bf16_tflops"] * 1e12)
+        t_sust = flops / (peaks["bf16_tflops_sustained"] * 1e12)
         achieved = flops / (attn_ms_step * 1e-3) / 1e12
+        attn_s = attn_ms_step * 1e-3
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": shape.name, "layers": n_layers, "batch": b, "context": shape.context,
-                       "ranks_mean": sum(wl.ranks) / len(wl.ranks), "l2": "inputs larger than L2 (latent cache %.1f GB)" %
-                       (sum(2 * 2 * r for r in wl.ranks) * b * n_ctx_mid / 1e9),
+                       "ranks_mean": sum(ranks_used) / len(ranks_used), "l2": "inputs larger than L2 (latent cache %.1f GB)" %
+                       (sum(2 * 2 * r for r in ranks_used) * tokens_mid / 1e9),
                        "kernel_path": {1: "plain fp32 CUDA-core", 2: "tcgen05", 3: "mma.sync streaming kernel (uncompressed mode)"}.get(path, str(path)),
                        "replicas": world, "launch": "cuda graph per step" if use_graph else "call by call",
                        "mode": "full-rank reference (uncompressed KV cache)" if args.full_rank else "latent"},
-            "decode_attn": {"ms_per_step": attn_ms_step, "tokens_per_s": b * world / (attn_ms_step * 1e-3),
-                            "roofline_ms": max(t_tc, t_hbm) * 1e3, "frac_of_roofline": max(t_tc, t_hbm) * 1e3 / attn_ms_step,
-                            "hbm_gbs": byts / (attn_ms_step * 1e-3) / 1e9},
+            "decode_attn": {"ms_per_step": attn_ms_step, "tokens_per_s": b * world / attn_s,
+                            "roofline_ms": max(t_tc, t_hbm) * 1e3, "frac_of_roofline": max(t_tc, t_hbm) / attn_s,
+                            "frac_burst": max(t_burst, t_hbm) / attn_s, "frac_sustained": max(t_sust, t_hbm) / attn_s,
+                            "peak_used": which + " bf16 peak (timed region %.3f s, median SM clock under load %s MHz)" %
+                            (timed_s, (clocks or {}).get("sm_mhz")),
+                            "hbm_gbs": byts / attn_s / 1e9},
             "clocks": clocks, "gpu_launches": launches,
         }
         line["decode_attn"].update({"achieved_tflops": achieved, "flops_per_step": flops, "bytes_per_step": byts})
         if score_prof:
-            # lorc_score_kernel: key reconstruction C_K.B_K on the tensor cores, RoPE and q.k in its epilogue.
-            # Algorithmic FLOPs per launch = batch * context * (2 r_k n + 2 H_q d_h), mean over the layers.
+            # lorc_score_kernel: key reconstruction C_K.B_K on the tensor cores, RoPE, q.k and the softmax numerators in
+            # its epilogue.  Algorithmic FLOPs per launch = cached tokens * (2 r_k n + 2 H_q d_h), mean over the layers.
             n, Hq, dh = shape.n, shape.n_q_heads, shape.d_head
-            k_flops = sum(b * n_ctx_mid * (2.0 * r * n + 2.0 * Hq * dh) for r in wl.ranks) / len(wl.ranks)
+            k_flops = sum(tokens_mid * (2.0 * r * n + 2.0 * Hq * dh) for r in ranks_used) / len(ranks_used)
             k_ms = score_prof[0]
             k_ach = k_flops / (k_ms * 1e-3) / 1e12
-            mean_r = sum(wl.ranks) / len(wl.ranks)
+            mean_r = sum(ranks_used) / len(ranks_used)
             traffic = None
             if SCORE_KERNEL_TRAFFIC is not None:
                 t = SCORE_KERNEL_TRAFFIC
-                scale = b * n_ctx_mid / float(t["batch"] * t["context"])
+                scale = tokens_mid / float(t["batch"] * t["context"])
                 traffic = (t["read_bytes"] * mean_r / t["rank"] + t["write_bytes"]) * scale
-            line["roofline"] = {"bound": "tensor", "achieved": k_ach, "peak": peaks["bf16_tflops_sustained"],
-                                "unit": "TFLOP/s", "frac": k_ach / peaks["bf16_tflops_sustained"], "traffic": traffic,
-                                "peak_source": peaks["source"] + " (sustained bf16: the kernel runs inside a long step)",
+            line["roofline"] = {"bound": "tensor", "achieved": k_ach, "peak": tc_peak,
+                                "unit": "TFLOP/s", "frac": k_ach / tc_peak,
+                                "frac_burst": k_ach / peaks["bf16_tflops"],
+                                "frac_sustained": k_ach / peaks["bf16_tflops_sustained"], "traffic": traffic,
+                                "peak_source": peaks["source"] + " (" + which + " bf16 peak; see decode_attn.peak_used)",
                                 "kernel": "lorc_score_kernel", "launch_ms": k_ms, "launches_per_step": score_prof[1],
                                 "flops_per_launch": k_flops,
                                 "timing": "CUDA events around every launch, call-by-call pass after the timed steps",
                                 "stage_ms_per_step": score_prof[2]}
         else:
-            gbs = byts / (attn_ms_step * 1e-3) / 1e9
+            gbs = byts / attn_s / 1e9
             line["roofline"] = {"bound": "hbm" if args.full_rank else "alu", "achieved": gbs if args.full_rank else achieved,
                                 "peak": peaks["hbm_gbs"] if args.full_rank else None,
                                 "unit": "GB/s" if args.full_rank else "TFLOP/s",
@@ -594,11 +836,12 @@ def main():
         if e2e:
             line["e2e"] = {"value": b * e2e_steps * world / e2e_s, "unit": UNIT, "h2d_bytes_per_step": e2e[1],
                            "d2h_bytes_per_step": e2e[2], "steps": e2e_steps}
-        if not args.no_cpu_baseline and world >= 1:
-            per_rank, desc, threads, units = oracle_sample(shape, n_layers)
-            step_s = per_rank * sum(wl.ranks) * b
-            line["cpu_baseline"] = {"value": b / step_s, "unit": UNIT, "cores": threads, "kind": "oracle",
-                                    "sample": desc}
+        if cpu:
+            line["cpu_baseline"], line["parity"] = cpu
+        if full_leg is not None:
+            line["full_rank"] = full_leg
+        if others is not None:
+            line["other_configs"] = others
         print(json.dumps(line))
     if dist is not None:
         dist.barrier()
