@@ -12,7 +12,8 @@ Notation (row-vector convention, K = X W_k as in the Preliminary section):
   W [D,n]  key or value weight        W ~= A B,  A = U_r Sigma_r [D,r],  B = V_r^T [r,n]
   C = X A  the latent ("compressed") cache row, width r = d_c        (Sec. 3.1)
 
-Every function is pinned by tests/test_oracle_pins.py to something the paper or
+Every function is pinned by tests/test_oracle_pins.py (the schedule functions by
+tests/test_schedule.py) to something the paper or
 the mathematics fixes (full-rank identity, Eckart-Young, Theorem 1, RoPE closed
 forms, brute-force attention, a library attention routine).  The numeric
 tolerance used when comparing the GPU to this oracle is not from the paper
@@ -90,6 +91,58 @@ def compression_ratio(d_c: int, h: int, d: int) -> float:
     """rho = d_c / (h * d): the retained fraction of the cache width (Sec. 3.1, "Compression Ratio")."""
     return d_c / float(h * d)
 
+
+
+# --------------------------------------------------------------------------
+# progressive compression schedule (Sec. 3.2; Algorithm 1, the two loops before the matrix compression)
+# --------------------------------------------------------------------------
+def condition_number(W: np.ndarray) -> float:
+    """kappa(W) = ||W||_2 ||W^+||_2 = sigma_max(W) / sigma_min(W)  (Sec. 3.2, the condition-number equation),
+    sigma_min being the smallest of the min(D, n) singular values of W [D, n]."""
+    s = np.linalg.svd(np.asarray(W, dtype=np.float64), compute_uv=False)
+    return float(s[0] / s[-1])
+
+
+def cumulative_log_condition(kappa_k, kappa_v) -> np.ndarray:
+    """log of the cumulative condition numbers, log kappa~_l = sum_{j >= l} (log kappa(W_k^j) + log kappa(W_v^j))
+    (Sec. 3.2, "Cumulative Condition Number": the product runs from layer l to the last layer).  Returned in log
+    form because the product itself overflows for deep models; the compression-dimension equation only uses logs."""
+    lk = np.log(np.asarray(kappa_k, dtype=np.float64)) + np.log(np.asarray(kappa_v, dtype=np.float64))
+    L = lk.shape[0]
+    out = np.empty(L, dtype=np.float64)
+    acc = 0.0
+    for l in range(L - 1, -1, -1):          # Algorithm 1 walks l = L .. 1
+        acc += lk[l]
+        out[l] = acc
+    return out
+
+
+def compression_dimensions(log_kappa_tilde, d_min: float, d_max: float) -> np.ndarray:
+    """Real-valued d_c^l of the compression-dimension equation (Sec. 3.2, Eq. "dc"):
+        d_c^l = d_max * [1 - (max_i log k~_i - log k~_l) / (max_i log k~_i - min_i log k~_i) * (1 - d_min / d_max)].
+    The layer with the largest cumulative condition number keeps d_max, the one with the smallest d_min.
+    When all layers are equally sensitive the fraction is 0/0; every layer then keeps d_max."""
+    lk = np.asarray(log_kappa_tilde, dtype=np.float64)
+    hi, lo = float(np.max(lk)), float(np.min(lk))
+    if hi == lo:
+        return np.full(lk.shape, float(d_max))
+    return d_max * (1.0 - (hi - lk) / (hi - lo) * (1.0 - d_min / d_max))
+
+
+def progressive_schedule(kappa_k, kappa_v, d_min: float, d_max: float, quantum: int = 1,
+                         log_threshold=None):
+    """Per-layer compression decision of Algorithm 1: (d_c [L] integers, skip [L] booleans).
+
+    d_c is Eq. "dc" rounded to the nearest multiple of `quantum` (ties to even; at least one quantum): the paper's
+    equation is real-valued and does not say how it is rounded (reading).  A layer is skipped
+    ("Skip compression for layer l") when its cumulative condition number exceeds the threshold; the comparison is
+    made on log kappa~_l against `log_threshold` because the product of 2 (L - l + 1) condition numbers is far
+    beyond the thresholds the paper quotes (30, 90), whose scale it does not define (reading: a parameter)."""
+    lk = cumulative_log_condition(kappa_k, kappa_v)
+    d = compression_dimensions(lk, d_min, d_max)
+    d = np.maximum(np.rint(d / quantum) * quantum, quantum).astype(np.int64)
+    skip = np.zeros(lk.shape, dtype=bool) if log_threshold is None else lk > float(log_threshold)
+    return d, skip
 
 # --------------------------------------------------------------------------
 # cache write (Sec. 3.1: the cache keeps X times the Sigma-carrying factor, for keys and for values)

@@ -402,3 +402,37 @@ def test_rel_l2_rows_metric():
     want = np.array([[3.0, 4.0], [0.0, 2.0]])
     got = np.array([[3.0, 4.5], [0.0, 2.0]])
     assert O.rel_l2_rows(got, want) == pytest.approx(0.1)
+
+
+def _golden_eckart_young():
+    import os
+    rows = []
+    with open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "eckart_young.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                n, p, r, t, e = line.split()
+                rows.append((int(n), float(p), int(r), float(t), float(e)))
+    return rows
+
+
+# closed-form values for the benchmark spectra (n = 1024: ranks of the 8B and 70B schedules), as listed with the
+# workload definitions; the golden file is written by tests/golden/make_eckart_young.py
+LISTED = {(128, 0.8, 32): (0.1159262, 0.2297970), (1024, 0.8, 128): (0.0644362, 0.1688638),
+          (1024, 0.8, 256): (0.0337240, 0.1221633), (1024, 0.8, 384): (0.0208377, 0.0960276),
+          (1024, 0.8, 416): (0.0186425, 0.0908288), (1024, 0.8, 512): (0.0134146, 0.0770479),
+          (1024, 0.8, 928): (0.00158316, 0.0264688), (1024, 0.7, 352): (0.0831541, 0.1679115),
+          (1024, 0.7, 864): (0.0109796, 0.0610144)}
+
+
+@pytest.mark.parametrize("n,p,r,tail,eps", _golden_eckart_young())
+def test_eckart_young_benchmark_spectra(n, p, r, tail, eps):
+    """relative_frobenius_error and factors_from_generators on the benchmark's spectra against the closed form."""
+    assert abs(tail - _tail(n, p, r)) <= 1e-12 and abs(eps - math.sqrt(_tail(n, p, r) / _total(n, p))) <= 1e-12
+    lt, le = LISTED[(n, p, r)]
+    assert abs(tail - lt) <= 5e-8 and abs(eps - le) <= 5e-8
+    # square weight (D = n): the error depends on the spectrum alone, so a small D keeps the test fast
+    U, s, V = synth.synth_weight_factors(n, n, p, layer=1, which="k")
+    W = (U * s) @ V.T
+    A, B = O.factors_from_generators(U, s, V, r)
+    assert abs(O.relative_frobenius_error(W, A @ B) - eps) <= 1e-9
+    assert abs(float(np.sum((W - A @ B) ** 2)) - tail) <= 1e-9
