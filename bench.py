@@ -48,6 +48,8 @@ def parse_args():
     ap.add_argument("--no-graph", action="store_true", help="launch call by call instead of replaying a CUDA graph")
     ap.add_argument("--stages", action="store_true",
                     help="call-by-call launches with per-kernel CUDA events; adds a 'stages' object (ms per step)")
+    ap.add_argument("--rope", default="half", choices=["half", "none"],
+                    help="none: layers whose keys take no rotation at attention time (the absorbed score path, HBM-bound)")
     ap.add_argument("--no-full-rank-leg", action="store_true",
                     help="skip the 'full_rank' object (the uncompressed mode timed on the same shape in the same run)")
     ap.add_argument("--no-other-configs", action="store_true",
@@ -193,14 +195,15 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------ workload set-up
-def algorithmic_counts(shape, ranks, batch, tokens):
+def algorithmic_counts(shape, ranks, batch, tokens, rope=True):
     """Per decode step over all layers: tensor-eligible FLOPs and latent+factor bytes of
-    lorc_decode_attn with `tokens` cached tokens in total over the `batch` sequences."""
+    lorc_decode_attn with `tokens` cached tokens in total over the `batch` sequences.  Without rotation the key
+    up-projection is absorbed into the query: 2 H_q r FLOP per token for the scores instead of 2 r n + 2 H_q d_h."""
     n, Hq, dh = shape.n, shape.n_q_heads, shape.d_head
     flops = 0.0
     byts = 0.0
     for r in ranks:
-        per_tok = 2.0 * r * n + 2.0 * Hq * dh + 2.0 * Hq * r
+        per_tok = (2.0 * r * n + 2.0 * Hq * dh if rope else 2.0 * Hq * r) + 2.0 * Hq * r
         flops += tokens * per_tok + batch * 2.0 * Hq * r * dh
         byts += tokens * 2.0 * (r + r) + 2.0 * (r + r) * n + 4.0 * batch * Hq * dh
     return flops, byts
@@ -216,7 +219,7 @@ class Workload:
     """Factors, filled latent caches and per-step inputs of one configuration on one GPU."""
 
     def __init__(self, L, shape, n_layers, total_steps, device, flags, full_rank=False, seeded_cache=False,
-                 keep_layers=(), layer_ids=None):
+                 keep_layers=(), layer_ids=None, rope=True):
         """seeded_cache: fill the caches with seeded synthetic rows instead of running the prompt through
         lorc_append (ragged paged configurations, and the short legs that only time attention).
         keep_layers: layers whose bf16 factors are also kept on the host (for the oracle leg).
@@ -241,8 +244,10 @@ class Workload:
             self.lens0 = [N] * b
         self.tokens0 = sum(self.lens0)
         self.n_max = ((max(self.lens0) + total_steps + 127) // 128) * 128
+        self.rope = rope
         self.ctx = L.lorc_create(n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.d_head,
-                                 shape.rope_theta, max_pos=self.n_max, flags=flags)
+                                 shape.rope_theta, max_pos=self.n_max, flags=flags,
+                                 rope_style=L.LORC_ROPE_HALF_SPLIT if rope else L.LORC_ROPE_NONE)
         self.caches, self.keep, self.host_factors = [], [], {}
         self.seq_lens = torch.zeros(b, dtype=torch.int32, device=device)
         self.page_table = None
@@ -567,13 +572,13 @@ def time_attention(wl, reps, use_graph):
     return e0.elapsed_time(e1) / reps
 
 
-def attention_leg(L, shape, device, peaks, full_rank=False, steps=4, warmup=3, n_layers=None):
+def attention_leg(L, shape, device, peaks, full_rank=False, steps=4, warmup=3, n_layers=None, rope=True):
     """A short, separate run of another configuration (or of the uncompressed mode): builds the workload with
     seeded cache rows, replays `steps` whole decode steps and the attention calls alone, and reports times and
     roofline fractions.  Everything of it is released before it returns."""
     import torch
     n_layers = n_layers or shape.n_layers
-    wl = Workload(L, shape, n_layers, warmup + steps + 3, device, 0, full_rank=full_rank, seeded_cache=True)
+    wl = Workload(L, shape, n_layers, warmup + steps + 3, device, 0, full_rank=full_rank, seeded_cache=True, rope=rope)
     try:
         wl.step()
         torch.cuda.synchronize()
@@ -597,13 +602,14 @@ def attention_leg(L, shape, device, peaks, full_rank=False, steps=4, warmup=3, n
         if full_rank:
             flops, byts = full_rank_counts(shape, n_layers, wl.batch, tokens)
         else:
-            flops, byts = algorithmic_counts(shape, wl.ranks, wl.batch, tokens)
+            flops, byts = algorithmic_counts(shape, wl.ranks, wl.batch, tokens, rope)
         t_hbm = byts / (peaks["hbm_gbs"] * 1e9) * 1e3
         t_burst = flops / (peaks["bf16_tflops"] * 1e12) * 1e3
         t_sust = flops / (peaks["bf16_tflops_sustained"] * 1e12) * 1e3
         return {
             "workload": shape.name, "layers": n_layers, "batch": wl.batch, "cached_tokens": tokens,
-            "mode": "full-rank reference (uncompressed KV cache)" if full_rank else "latent",
+            "mode": "full-rank reference (uncompressed KV cache)" if full_rank else
+                    ("latent" if rope else "latent, no rotation at attention time (absorbed scores)"),
             "kernel_path": {1: "plain fp32 CUDA-core", 2: "tcgen05", 3: "mma.sync streaming kernel"}.get(path, str(path)),
             "step_ms": step_ms, "tokens_per_s": wl.batch / (step_ms * 1e-3),
             "attn_ms_per_step": attn_ms, "attn_tokens_per_s": wl.batch / (attn_ms * 1e-3),
@@ -652,10 +658,11 @@ def main():
         args.no_graph = True
     e2e_steps = 0 if args.no_e2e else max(2, min(args.steps, 8))
     total_steps = args.warmup + args.steps + e2e_steps + 4
-    do_oracle = (not args.no_cpu_baseline) and rank == 0 and world == 1 and not args.full_rank
+    rope = args.rope == "half"
+    do_oracle = (not args.no_cpu_baseline) and rank == 0 and world == 1 and not args.full_rank and rope
     oracle_layers = sorted(set([0, n_layers // 2, n_layers - 1])) if do_oracle else []
     wl = Workload(L, shape, n_layers, total_steps, device, flags, full_rank=args.full_rank,
-                  seeded_cache=bool(shape.paged or shape.ragged[1] > 0), keep_layers=oracle_layers)
+                  seeded_cache=bool(shape.paged or shape.ragged[1] > 0), keep_layers=oracle_layers, rope=rope)
     b = shape.batch
 
     def barrier():
@@ -701,7 +708,7 @@ def main():
     # the dominant kernel alone: the same attention calls again, launched one by one with a CUDA event before and
     # after every kernel on the launching stream (the library's own stage bracketing)
     score_prof = None
-    if not args.debug_fp32 and not args.full_rank:
+    if not args.debug_fp32 and not args.full_rank and rope:
         L.lorc_profile_read(wl.ctx)
         L.lorc_profile_enable(wl.ctx, True)
         prof_reps = max(3, min(args.steps, 8))
@@ -753,7 +760,13 @@ def main():
 
     # the uncompressed mode on the same shape, and the other configurations, a few steps each (1-GPU runs only)
     full_leg, others = None, None
-    if rank == 0 and world == 1 and not args.full_rank and not args.debug_fp32 and args.layers == 0:
+    absorbed_leg = None
+    if rank == 0 and world == 1 and not args.full_rank and not args.debug_fp32 and args.layers == 0 and rope:
+        if not args.no_other_configs:
+            try:
+                absorbed_leg = attention_leg(L, shape, device, peaks, steps=4, rope=False)
+            except Exception as exc:
+                absorbed_leg = {"error": str(exc)[:200]}
         if not args.no_full_rank_leg:
             try:
                 full_leg = attention_leg(L, shape, device, peaks, full_rank=True, steps=4)
@@ -774,7 +787,7 @@ def main():
         if args.full_rank:
             flops, byts = full_rank_counts(shape, n_layers, b, tokens_mid)
         else:
-            flops, byts = algorithmic_counts(shape, ranks_used, b, tokens_mid)
+            flops, byts = algorithmic_counts(shape, ranks_used, b, tokens_mid, rope)
         timed_s = ms * 1e-3
         which, tc_peak = pick_tensor_peak(peaks, timed_s, clocks)
         t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
@@ -792,7 +805,8 @@ def main():
                        (sum(2 * 2 * r for r in ranks_used) * tokens_mid / 1e9),
                        "kernel_path": {1: "plain fp32 CUDA-core", 2: "tcgen05", 3: "mma.sync streaming kernel (uncompressed mode)"}.get(path, str(path)),
                        "replicas": world, "launch": "cuda graph per step" if use_graph else "call by call",
-                       "mode": "full-rank reference (uncompressed KV cache)" if args.full_rank else "latent"},
+                       "mode": "full-rank reference (uncompressed KV cache)" if args.full_rank else
+                       ("latent" if rope else "latent, no rotation at attention time (absorbed scores)")},
             "decode_attn": {"ms_per_step": attn_ms_step, "tokens_per_s": b * world / attn_s,
                             "roofline_ms": max(t_tc, t_hbm) * 1e3, "frac_of_roofline": max(t_tc, t_hbm) / attn_s,
                             "frac_burst": max(t_burst, t_hbm) / attn_s, "frac_sustained": max(t_sust, t_hbm) / attn_s,
@@ -826,11 +840,12 @@ def main():
                                 "stage_ms_per_step": score_prof[2]}
         else:
             gbs = byts / attn_s / 1e9
-            line["roofline"] = {"bound": "hbm" if args.full_rank else "alu", "achieved": gbs if args.full_rank else achieved,
-                                "peak": peaks["hbm_gbs"] if args.full_rank else None,
-                                "unit": "GB/s" if args.full_rank else "TFLOP/s",
-                                "frac": gbs / peaks["hbm_gbs"] if args.full_rank else None, "traffic": None,
-                                "kernel": "whole lorc_decode_attn (" + {1: "plain fp32 CUDA-core kernels", 3: "mma.sync streaming kernel + merge"}.get(path, str(path)) + ")"}
+            hbm_bound = args.full_rank or not rope
+            line["roofline"] = {"bound": "hbm" if hbm_bound else "alu", "achieved": gbs if hbm_bound else achieved,
+                                "peak": peaks["hbm_gbs"] if hbm_bound else None,
+                                "unit": "GB/s" if hbm_bound else "TFLOP/s",
+                                "frac": gbs / peaks["hbm_gbs"] if hbm_bound else None, "traffic": None,
+                                "kernel": "whole lorc_decode_attn (" + {1: "plain fp32 CUDA-core kernels", 2: "absorbed score kernel + PV + up-projection", 3: "mma.sync streaming kernel + merge"}.get(path, str(path)) + ")"}
         if stages:
             line["stages"] = stages
         if e2e:
@@ -842,6 +857,8 @@ def main():
             line["full_rank"] = full_leg
         if others is not None:
             line["other_configs"] = others
+        if absorbed_leg is not None:
+            line["no_rotation"] = absorbed_leg
         print(json.dumps(line))
     if dist is not None:
         dist.barrier()

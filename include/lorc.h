@@ -53,6 +53,9 @@ extern "C" {
 /* RoPE pairing */
 #define LORC_ROPE_HALF_SPLIT 0  /* pair (j, j + d_head/2) */
 #define LORC_ROPE_INTERLEAVED 1 /* pair (2j, 2j + 1)      */
+#define LORC_ROPE_NONE 2        /* no rotation at attention time: a model without rotary embedding, or one whose
+                                   rotation does not touch the compressed keys.  The scores then take the absorbed
+                                   form of Sec. 3.1 (the W_q' equation), s = (B_K q) . c: keys are never reconstructed */
 
 /* context flags */
 #define LORC_FLAG_DEBUG_FP32 1  /* run the plain fp32 CUDA-core kernels everywhere (debug path) */

@@ -26,6 +26,7 @@ LORC_MODE_LATENT = 0
 LORC_MODE_FULL = 1
 LORC_ROPE_HALF_SPLIT = 0
 LORC_ROPE_INTERLEAVED = 1
+LORC_ROPE_NONE = 2
 LORC_FLAG_DEBUG_FP32 = 1
 LORC_FLAG_PROFILE = 2
 LORC_N_STAGES = 4

@@ -50,6 +50,8 @@ struct lorc_ctx {
     int device = 0;
     int n = 0;                 // n_kv_heads * d_head
     int group = 0;             // n_q_heads / n_kv_heads
+    int pair_style = LORC_ROPE_HALF_SPLIT;   // how the kernels pair the elements of a head (LORC_ROPE_NONE: half split,
+                                              // with a rotation table that holds the identity)
     int sm_count = 0;
     std::vector<LorcLayer> layers;
     float2* rope_table = nullptr;   // [max_pos][d_head/2] (cos, sin)

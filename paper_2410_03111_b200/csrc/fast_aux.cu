@@ -174,11 +174,11 @@ cudaError_t lorc_tc_append(lorc_ctx* ctx, int, const LorcLayer& L, const CacheVi
     if (L.mode == LORC_MODE_FULL)
         append_mma_kernel<true><<<grid, 256, 0, st>>>(x, L.A_tiled, cv, ctx->desc.d_model, L.r_k, L.r_v, T,
                                                       ctx->desc.max_pos, ctx->status_dev, ctx->desc.d_head,
-                                                      ctx->desc.rope_style, ctx->rope_table);
+                                                      ctx->pair_style, ctx->rope_table);
     else
         append_mma_kernel<false><<<grid, 256, 0, st>>>(x, L.A_tiled, cv, ctx->desc.d_model, L.r_k, L.r_v, T,
                                                        ctx->desc.max_pos, ctx->status_dev, ctx->desc.d_head,
-                                                       ctx->desc.rope_style, ctx->rope_table);
+                                                       ctx->pair_style, ctx->rope_table);
     *launches += 1;
     return cudaGetLastError();
 }

@@ -295,7 +295,7 @@ cudaError_t lorc_full_decode(const lorc_ctx* ctx, const CacheView& cv, const bf1
         if (e != cudaSuccess) return e;
         if (known) attr[ctx->device] = true;
     }
-    full_decode_mma_kernel<<<grid, 128, sizeof(FdSmem), st>>>(q, cv, ctx->group, n_splits, d.rope_style, ctx->rope_table, d.max_pos,
+    full_decode_mma_kernel<<<grid, 128, sizeof(FdSmem), st>>>(q, cv, ctx->group, n_splits, ctx->pair_style, ctx->rope_table, d.max_pos,
                                                  part_ml, part_o, ctx->status_dev);
     *launches += 1;
     return cudaGetLastError();

@@ -9,7 +9,8 @@
 #include "common.cuh"
 
 // ---------------------------------------------------------------------------
-// RoPE table: (cos, sin)(pos * theta^(-2j/d_head)), angles in fp64.
+// RoPE table: (cos, sin)(pos * theta^(-2j/d_head)), angles in fp64.  theta <= 0 stands for "no rotation": every entry
+// is (1, 0), and the kernels that rotate by the table leave keys and queries as they are.
 // ---------------------------------------------------------------------------
 __global__ void rope_table_kernel(float2* table, int max_pos, int half, double theta) {
     long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -17,6 +18,10 @@ __global__ void rope_table_kernel(float2* table, int max_pos, int half, double t
     if (i >= total) return;
     int pos = (int)(i / half);
     int j = (int)(i - (long long)pos * half);
+    if (!(theta > 0.0)) {
+        table[i] = make_float2(1.f, 0.f);
+        return;
+    }
     double inv_freq = pow(theta, -(double)j / (double)half);   // theta^(-2j/d_head)
     double s, c;
     sincos((double)pos * inv_freq, &s, &c);
@@ -151,11 +156,11 @@ cudaError_t lorc_generic_append(const lorc_ctx* ctx, const LorcLayer& L, const C
     if (L.mode == LORC_MODE_FULL) {
         append_generic_kernel<true><<<grid, 128, 0, st>>>(
             x, L.A_cat, cv, ctx->desc.d_model, L.r_k, L.r_v, T, ctx->desc.d_head,
-            ctx->desc.rope_style, ctx->rope_table, ctx->desc.max_pos, ctx->status_dev);
+            ctx->pair_style, ctx->rope_table, ctx->desc.max_pos, ctx->status_dev);
     } else {
         append_generic_kernel<false><<<grid, 128, 0, st>>>(
             x, L.A_cat, cv, ctx->desc.d_model, L.r_k, L.r_v, T, ctx->desc.d_head,
-            ctx->desc.rope_style, ctx->rope_table, ctx->desc.max_pos, ctx->status_dev);
+            ctx->pair_style, ctx->rope_table, ctx->desc.max_pos, ctx->status_dev);
     }
     *launches += 1;
     return cudaGetLastError();
@@ -462,7 +467,7 @@ cudaError_t lorc_generic_decode(const lorc_ctx* ctx, const LorcLayer& L, const C
     LorcStageTimer timer(ctx, LORC_STAGE_SCORE, st);
 #define LAUNCH_DEC(DHV, LAT)                                                                      \
     decode_generic_kernel<DHV, LAT><<<grid, 128, 0, st>>>(                                        \
-        q, cv, L.B_k, L.r_k, L.r_v, ctx->n, G, n_splits, d.rope_style, ctx->rope_table, d.max_pos, \
+        q, cv, L.B_k, L.r_k, L.r_v, ctx->n, G, n_splits, ctx->pair_style, ctx->rope_table, d.max_pos, \
         part_ml, part_o, ctx->status_dev)
     if (d.d_head == 128) {
         if (latent) LAUNCH_DEC(128, true); else LAUNCH_DEC(128, false);

@@ -121,7 +121,8 @@ int lorc_create(const lorc_model_desc* desc, lorc_ctx** out) {
     if (desc->n_q_heads % desc->n_kv_heads != 0) return LORC_ERR_ARG;
     if (desc->n_q_heads / desc->n_kv_heads > 8) return LORC_ERR_UNSUPPORTED;
     if (desc->d_head != 64 && desc->d_head != 128) return LORC_ERR_UNSUPPORTED;
-    if (desc->rope_style != LORC_ROPE_HALF_SPLIT && desc->rope_style != LORC_ROPE_INTERLEAVED)
+    if (desc->rope_style != LORC_ROPE_HALF_SPLIT && desc->rope_style != LORC_ROPE_INTERLEAVED &&
+        desc->rope_style != LORC_ROPE_NONE)
         return LORC_ERR_ARG;
     if (desc->d_model % 8 != 0) return LORC_ERR_ARG;
     lorc_ctx* ctx = new (std::nothrow) lorc_ctx();
@@ -129,6 +130,7 @@ int lorc_create(const lorc_model_desc* desc, lorc_ctx** out) {
     ctx->desc = *desc;
     ctx->n = desc->n_kv_heads * desc->d_head;
     ctx->group = desc->n_q_heads / desc->n_kv_heads;
+    ctx->pair_style = desc->rope_style == LORC_ROPE_NONE ? LORC_ROPE_HALF_SPLIT : desc->rope_style;
     ctx->layers.resize(desc->n_layers);
     if (desc->flags & LORC_FLAG_PROFILE) {
         ctx->prof = new (std::nothrow) LorcProfile();
@@ -142,7 +144,8 @@ int lorc_create(const lorc_model_desc* desc, lorc_ctx** out) {
     size_t tbytes = (size_t)desc->max_pos * (desc->d_head / 2) * sizeof(float2);
     if (e == cudaSuccess) e = cudaMalloc(&ctx->rope_table, tbytes);
     if (e == cudaSuccess)
-        e = lorc_generic_build_rope_table(ctx->rope_table, desc->max_pos, desc->d_head, desc->rope_theta, 0);
+        e = lorc_generic_build_rope_table(ctx->rope_table, desc->max_pos, desc->d_head,
+                                          desc->rope_style == LORC_ROPE_NONE ? 0.0 : desc->rope_theta, 0);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         cudaFree(ctx->status_dev);
@@ -208,7 +211,7 @@ int lorc_load_factors(lorc_ctx* ctx, int layer, int mode, int r_k, int r_v, cons
         e = cudaMemcpy2DAsync(L.A_cat + r_k, (size_t)R * sizeof(bf16), A_v, (size_t)r_v * sizeof(bf16),
                               (size_t)r_v * sizeof(bf16), D, cudaMemcpyDeviceToDevice, st);
     if (e == cudaSuccess && L.A_tiled) {
-        const bool pairs = mode == LORC_MODE_FULL && ctx->desc.rope_style == LORC_ROPE_HALF_SPLIT;
+        const bool pairs = mode == LORC_MODE_FULL && ctx->pair_style == LORC_ROPE_HALF_SPLIT;
         e = lorc_fast_retile_factor(L.A_cat, L.A_tiled, D, R, pairs ? r_k : 0, ctx->desc.d_head, st);
     }
     if (e == cudaSuccess && mode == LORC_MODE_LATENT) {

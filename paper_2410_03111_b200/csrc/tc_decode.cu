@@ -63,7 +63,7 @@ void lorc_tc_invalidate_layer(lorc_ctx* ctx, int layer) {
 
 static bool tc_shape_ok(const lorc_ctx* ctx) {
     const lorc_model_desc& d = ctx->desc;
-    return d.d_head == 128 && d.rope_style == LORC_ROPE_HALF_SPLIT && (d.n_kv_heads % 2) == 0 &&
+    return d.d_head == 128 && (d.rope_style == LORC_ROPE_HALF_SPLIT || d.rope_style == LORC_ROPE_NONE) && (d.n_kv_heads % 2) == 0 &&
            (ctx->group == 4 || ctx->group == 8) && (d.n_q_heads == 32 || d.n_q_heads == 64);
 }
 
@@ -82,9 +82,15 @@ static size_t tc_image_area_bytes(const lorc_ctx* ctx, int batch, int max_seq_le
     return lorc_align_up((size_t)batch * tiles * lorc_tc_image_bytes(ctx->desc.n_q_heads), 256);
 }
 
+// the absorbed query of layers without rotation sits between the images and the PV scratch
+static size_t tc_absorbed_bytes(const lorc_ctx* ctx, int batch) {
+    return ctx->desc.rope_style == LORC_ROPE_NONE ? lorc_tc_absorbed_scratch_bytes(ctx, batch) : 0;
+}
+
 size_t lorc_tc_workspace_bytes(const lorc_ctx* ctx, int batch, int max_seq_len) {
     if (!tc_shape_ok(ctx)) return 0;
-    return tc_image_area_bytes(ctx, batch, max_seq_len) + lorc_tc_pv_scratch_bytes(ctx, batch, max_seq_len);
+    return tc_image_area_bytes(ctx, batch, max_seq_len) + tc_absorbed_bytes(ctx, batch) +
+           lorc_tc_pv_scratch_bytes(ctx, batch, max_seq_len);
 }
 
 static bool build_cache_maps(LorcTcLayer& T, const LorcLayer& L, const CacheView& cv) {
@@ -128,6 +134,7 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
         // per context, hence per device: the attribute belongs to the device's copy of the kernel
         cudaError_t e = lorc_tc_score_set_attrs();
         if (e == cudaSuccess) e = lorc_tc_pv_set_attrs();
+        if (e == cudaSuccess) e = lorc_tc_absorbed_set_attrs();
         if (e != cudaSuccess) return e;
         T->attrs_set = true;
     }
@@ -144,11 +151,13 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
 
     const int tiles = (cv.max_seq_len + TILE - 1) / TILE;
     const size_t img_area = tc_image_area_bytes(ctx, cv.batch, cv.max_seq_len);
-    if (img_area >= ws_bytes) return cudaErrorMemoryAllocation;
+    const size_t abs_area = tc_absorbed_bytes(ctx, cv.batch);
+    if (img_area + abs_area >= ws_bytes) return cudaErrorMemoryAllocation;
     uint8_t* pimg = (uint8_t*)ws;
-    void* pv_scratch = (char*)ws + img_area;
+    bf16* qabs = (bf16*)((char*)ws + img_area);
+    void* pv_scratch = (char*)ws + img_area + abs_area;
     LorcPvPlan plan;
-    lorc_tc_pv_plan(ctx, L, cv, n_splits, ws_bytes - img_area, &plan);
+    lorc_tc_pv_plan(ctx, L, cv, n_splits, ws_bytes - img_area - abs_area, &plan);
     if (!plan.fits) return cudaErrorMemoryAllocation;
     // Row maxima [batch, H_q]: all zero between calls (the up-projection kernel clears what the score kernel raised).
     // Owned by the library because that invariant must hold from the first call on.  The table only ever grows, and a
@@ -170,9 +179,16 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
     T->rowmax_dirty = true;
     {
         LorcStageTimer timer(ctx, LORC_STAGE_SCORE, st);
-        cudaError_t e = lorc_tc_score_launch(ctx, L, cv, TL.mapCK, TL.mapBKT, q, pimg, T->rowmax,
-                                             reinterpret_cast<const float4*>(T->rope_tile), tiles,
-                                             (int*)((char*)pv_scratch + plan.off_done), cv.batch * plan.n_blk, st, launches);
+        int* zero = (int*)((char*)pv_scratch + plan.off_done);
+        cudaError_t e;
+        if (d.rope_style == LORC_ROPE_NONE)
+            // no rotation between the key up-projection and the dot product: the up-projection moves to the query
+            e = lorc_tc_score_absorbed_launch(ctx, L, cv, TL.mapCK, q, qabs, pimg, T->rowmax, tiles, zero,
+                                              cv.batch * plan.n_blk, st, launches);
+        else
+            e = lorc_tc_score_launch(ctx, L, cv, TL.mapCK, TL.mapBKT, q, pimg, T->rowmax,
+                                     reinterpret_cast<const float4*>(T->rope_tile), tiles, zero, cv.batch * plan.n_blk, st,
+                                     launches);
         if (e != cudaSuccess) return e;
     }
     const cudaError_t e2 = lorc_tc_pv_launch(ctx, L, cv, TL.mapCV, TL.mapBVT, pimg, T->rowmax, tiles, plan, pv_scratch,

@@ -33,6 +33,15 @@ cudaError_t lorc_tc_score_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheV
                                  const float4* rope_tile, int tiles, int* zero, int n_zero, cudaStream_t st,
                                  int* launches);
 
+// Score kernel of layers without rotation (tc_absorbed.cu): the key up-projection is absorbed into the query
+// (q~ = B_K q, written to `qabs`, lorc_tc_absorbed_scratch_bytes of scratch), the scores are a skinny GEMM over the
+// latent keys.  Same outputs as lorc_tc_score_launch.
+size_t lorc_tc_absorbed_scratch_bytes(const lorc_ctx* ctx, int batch);
+cudaError_t lorc_tc_absorbed_set_attrs();
+cudaError_t lorc_tc_score_absorbed_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, const CUtensorMap& mapCK,
+                                          const bf16* q, bf16* qabs, uint8_t* pimg, unsigned* rowmax, int tiles, int* zero,
+                                          int n_zero, cudaStream_t st, int* launches);
+
 // P.C_V and value up-projection (tc_pv.cu).  mapCV: C_V cache in 64-column x 128-row (or page-sized) swizzled boxes;
 // mapBVT: B_V^T [n, r_v] in swizzled boxes of 64 latent columns x 32 rows.  The plan says how a launch splits the
 // work and where its pieces of scratch lie; the `done` words (plan.n_blk * batch ints at off_done) must be zero when

@@ -8,6 +8,9 @@ from oracle import lorc_oracle as O
 from workloads import synth
 
 
+ROPE_NONE = 2          # LORC_ROPE_NONE: no rotation at attention time
+
+
 def lib():
     import paper_2410_03111_b200 as pkg
     return pkg.load()
@@ -126,8 +129,10 @@ def oracle_decode(prob, ck, cv, q):
     """fp64 decode attention per sequence from given latents; q [b, H_q, d_h]."""
     out = np.empty((len(ck), prob.H_q, prob.d_h))
     for s in range(len(ck)):
-        out[s] = O.decode_attn_latent(ck[s], cv[s], prob.B_k, prob.B_v, q[s], prob.H_kv, prob.theta,
-                                      prob.style)
+        if prob.style == ROPE_NONE:
+            out[s] = O.decode_attn_latent(ck[s], cv[s], prob.B_k, prob.B_v, q[s], prob.H_kv, prob.theta, use_rope=False)
+        else:
+            out[s] = O.decode_attn_latent(ck[s], cv[s], prob.B_k, prob.B_v, q[s], prob.H_kv, prob.theta, prob.style)
     return out
 
 

@@ -80,6 +80,9 @@ CASES = [
     (512, 8, 2, 128, 256, 256, [513, 64, 1000], 0),
     (384, 16, 2, 64, 40, 128, [95, 260], 1),
     (512, 8, 1, 128, 128, 8, [333], 0),
+    # style 2: no rotation at attention time (plain kernels with an identity rotation table)
+    (256, 4, 2, 64, 32, 32, [129], 2),
+    (512, 8, 2, 128, 96, 72, [37, 300], 2),
 ]
 
 

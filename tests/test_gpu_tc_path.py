@@ -282,3 +282,37 @@ def test_full_rank_mode_streaming_kernel(H_q, lens, paged):
             assert O.rel_l2_rows(got[s], want[s]) <= TOL, (n_splits, s, O.rel_l2_rows(got[s], want[s]))
         outs.append(got)
     sess.close()
+
+
+# --------------------------------------------------------------- no rotation: the absorbed score path
+@pytest.mark.parametrize("r_k,r_v,lens,paged", [
+    (96, 72, [1, 37, 300, 700], False),
+    (256, 256, [129, 128, 1000], True),
+    (928, 928, [513, 77], False),
+])
+def test_tc_decode_without_rotation_uses_the_absorbed_scores(r_k, r_v, lens, paged):
+    """LORC_ROPE_NONE: s = (B_K q) . c (Sec. 3.1, the W_q' equation) on the tensor cores, against the oracle, which
+    reconstructs the keys explicitly and applies no rotation."""
+    key = (r_k, r_v, "none")
+    if key not in _PROBS:
+        _PROBS[key] = H.Problem(GEOM["D"], GEOM["H_q"], GEOM["H_kv"], GEOM["d_h"], r_k, r_v, theta=500000.0, layer=21,
+                                style=H.ROPE_NONE)
+    prob = _PROBS[key]
+    b, n_max = len(lens), max(lens) + 3
+    sess = H.Session(prob, max_pos=n_max, batch=b)
+    ck, cv = _latents(prob, lens, 21)
+    # (the descriptor only holds addresses: the tensors behind it must stay alive)
+    if paged:
+        held = H.paged_cache(sess, b, lens, 64, order_seed=5, k_rows=ck, v_rows=cv)
+    else:
+        held = H.contiguous_cache(sess, b, n_max, lens, ck, cv)
+    cache = held[0]
+    worst = 0.0
+    for q_scale in (1.0, 64.0):
+        q = synth.queries(b, GEOM["H_q"], GEOM["d_h"], 21, int(q_scale), q_scale).astype(np.float64)
+        got = H.host_f64(_run(sess, cache, q))
+        want = H.oracle_decode(prob, ck, cv, q)
+        H.assert_rows_close(got, want, TOL, (r_k, q_scale))
+        worst = max(worst, O.rel_l2_rows(got, want))
+    print(f"\n[no rotation] r_k {r_k}: max relative L2 row error {worst:.2e}")
+    sess.close()
