@@ -188,6 +188,15 @@ int lorc_append(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* x
 int lorc_decode_attn(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* q, void* out,
                      int n_splits, void* stream);
 
+/* Decode attention that stops before the value up-projection (Sec. 3.1, the W_o' equation: the orthonormal value
+ * factor can be folded into the output projection, W_o' = B_V,g W_o,h stacked over the heads).  Same arguments as
+ * lorc_decode_attn except the result:
+ *   o_lat [batch, n_q_heads, r_v] device bf16,  o_lat[s, h, :] = sum_n p_n C_V[n, :]  (softmax as in lorc_decode_attn),
+ * so that lorc_decode_attn's out[s, h, :] = o_lat[s, h, :] B_V[:, g(h)].  Compressed (LATENT) layers only.
+ * Errors: as lorc_decode_attn, UNSUPPORTED for an uncompressed layer. */
+int lorc_decode_attn_latent_out(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* q, void* o_lat,
+                                int n_splits, void* stream);
+
 /* Decode attention without any caller-provided or freshly allocated scratch.
  * (The paper has no counterpart to this call; it exists for deployment reasons.)
  * Meant for hosts that cannot allocate device memory when they call in: a server

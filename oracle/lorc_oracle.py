@@ -247,6 +247,32 @@ def decode_attn_latent(c_k: np.ndarray, c_v: np.ndarray, B_k: np.ndarray, B_v: n
     return attention_one_query(q, K, V)
 
 
+def decode_attn_latent_out(c_k: np.ndarray, c_v: np.ndarray, B_k: np.ndarray, q: np.ndarray,
+                           n_kv_heads: int, theta: float, style: int = ROPE_HALF_SPLIT,
+                           use_rope: bool = True) -> np.ndarray:
+    """Decode attention stopped before the value up-projection: o_lat[h] = sum_n p[h, n] c^V_n, [H_q, r_v].
+
+    The probabilities are those of decode_attn_latent (keys reconstructed, rotated, softmax); the values are left
+    as cached latents.  Sec. 3.1 (the W_o' equation) folds the remaining factor into the output projection:
+    decode_attn_latent's output is o_lat[h] B_V[:, g(h)]."""
+    c_k = np.asarray(c_k, dtype=np.float64)
+    c_v = np.asarray(c_v, dtype=np.float64)
+    q = np.asarray(q, dtype=np.float64)
+    N = c_k.shape[0]
+    H_q, d = q.shape
+    G = H_q // n_kv_heads
+    K = (c_k @ np.asarray(B_k, dtype=np.float64)).reshape(N, n_kv_heads, d)
+    if use_rope:
+        K = rope(K, np.arange(N)[:, None], theta, style)
+        q = rope(q, np.full((H_q,), N - 1), theta, style)
+    out = np.empty((H_q, c_v.shape[1]), dtype=np.float64)
+    for h in range(H_q):
+        s = K[:, h // G, :] @ q[h] / math.sqrt(d)
+        p = np.exp(s - np.max(s))
+        out[h] = (p / np.sum(p)) @ c_v
+    return out
+
+
 def decode_attn_full(x: np.ndarray, W_k: np.ndarray, W_v: np.ndarray, q: np.ndarray,
                      n_kv_heads: int, theta: float, style: int = ROPE_HALF_SPLIT,
                      positions=None, q_position=None, use_rope: bool = True) -> np.ndarray:

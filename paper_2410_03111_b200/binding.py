@@ -68,6 +68,7 @@ def _signatures():
         "lorc_set_workspace": ([vp, vp, C.c_size_t], i32),
         "lorc_append": ([vp, i32, cp, vp, i32, vp], i32),
         "lorc_decode_attn": ([vp, i32, cp, vp, vp, i32, vp], i32),
+        "lorc_decode_attn_latent_out": ([vp, i32, cp, vp, vp, i32, vp], i32),
         "lorc_decode_attn_static": ([vp, i32, cp, vp, vp, i32, vp], i32),
         "lorc_decode_step_host": ([vp, i32, cp, vp, vp, vp, i32, vp], i32),
         "lorc_sync_status": ([vp, vp], i32),
@@ -169,6 +170,11 @@ def lorc_append(ctx, layer, cache, x, T=1, stream=None):
 def lorc_decode_attn(ctx, layer, cache, q, out, n_splits=0, stream=None):
     _check(ctx, _lib.lorc_decode_attn(ctx, layer, C.byref(cache), _ptr(q), _ptr(out), n_splits,
                                        _stream(stream)))
+
+
+def lorc_decode_attn_latent_out(ctx, layer, cache, q, o_lat, n_splits=0, stream=None):
+    _check(ctx, _lib.lorc_decode_attn_latent_out(ctx, layer, C.byref(cache), _ptr(q), _ptr(o_lat), n_splits,
+                                                  _stream(stream)))
 
 
 def lorc_decode_attn_static(ctx, layer, cache, q, out, n_splits=0, stream=None):

@@ -126,14 +126,15 @@ cudaError_t lorc_generic_append(const lorc_ctx* ctx, const LorcLayer& L, const C
 bool lorc_full_decode_supported(const lorc_ctx* ctx, const LorcLayer& L);
 cudaError_t lorc_full_decode(const lorc_ctx* ctx, const CacheView& cv, const bf16* q, int n_splits, float* part_ml,
                              float* part_o, cudaStream_t st, int* launches);
+// latent_out: stop before the value up-projection and write the normalised latent output [b, H_q, r_v] to `out`.
 cudaError_t lorc_generic_decode(const lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv,
                                 const bf16* q, bf16* out, int n_splits, float* part_ml,
-                                float* part_o, cudaStream_t st, int* launches);
+                                float* part_o, cudaStream_t st, int* launches, bool latent_out = false);
 // Merge of split partials + value up-projection (also used by the tensor-core path):
 // part_ml [b, H_q, S, 2] (running max in natural-log units, sum), part_o [b, H_q, S, W].
 cudaError_t lorc_generic_combine(const lorc_ctx* ctx, const LorcLayer& L, int batch, int n_splits,
                                  const float* part_ml, const float* part_o, bf16* out,
-                                 cudaStream_t st, int* launches);
+                                 cudaStream_t st, int* launches, bool latent_out = false);
 // token granularity of a split in the plain decode kernel
 #define LORC_GENERIC_TILE 32
 #define LORC_MAX_SPLITS 256

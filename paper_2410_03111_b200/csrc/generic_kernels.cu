@@ -428,14 +428,18 @@ combine_generic_kernel(const float* __restrict__ part_ml, const float* __restric
 
 cudaError_t lorc_generic_combine(const lorc_ctx* ctx, const LorcLayer& L, int batch, int n_splits,
                                  const float* part_ml, const float* part_o, bf16* out,
-                                 cudaStream_t st, int* launches) {
+                                 cudaStream_t st, int* launches, bool latent_out) {
     const lorc_model_desc& d = ctx->desc;
     const bool latent = (L.mode == LORC_MODE_LATENT);
     const int W = latent ? L.r_v : d.d_head;
     dim3 cgrid(d.n_q_heads, batch);
     size_t smem = (size_t)W * sizeof(float);
     LorcStageTimer timer(ctx, LORC_STAGE_COMBINE, st);
-    if (latent)
+    if (latent && latent_out)
+        // merge only: the normalised latent output [b, H_q, r_v] is the result (rows of width W instead of d_head)
+        combine_generic_kernel<false><<<cgrid, 128, smem, st>>>(part_ml, part_o, nullptr, out, W, ctx->n, W, ctx->group,
+                                                               n_splits, ctx->status_dev);
+    else if (latent)
         combine_generic_kernel<true><<<cgrid, 128, smem, st>>>(part_ml, part_o, L.B_v, out, W, ctx->n,
                                                               d.d_head, ctx->group, n_splits,
                                                               ctx->status_dev);
@@ -449,7 +453,7 @@ cudaError_t lorc_generic_combine(const lorc_ctx* ctx, const LorcLayer& L, int ba
 
 cudaError_t lorc_generic_decode(const lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv,
                                 const bf16* q, bf16* out, int n_splits, float* part_ml,
-                                float* part_o, cudaStream_t st, int* launches) {
+                                float* part_o, cudaStream_t st, int* launches, bool latent_out) {
     const lorc_model_desc& d = ctx->desc;
     const int G = ctx->group;
     const bool latent = (L.mode == LORC_MODE_LATENT);
@@ -461,7 +465,7 @@ cudaError_t lorc_generic_decode(const lorc_ctx* ctx, const LorcLayer& L, const C
             cudaError_t e = lorc_full_decode(ctx, cv, q, n_splits, part_ml, part_o, st, launches);
             if (e != cudaSuccess) return e;
         }
-        return lorc_generic_combine(ctx, L, cv.batch, n_splits, part_ml, part_o, out, st, launches);
+        return lorc_generic_combine(ctx, L, cv.batch, n_splits, part_ml, part_o, out, st, launches, false);
     }
     {
     LorcStageTimer timer(ctx, LORC_STAGE_SCORE, st);
@@ -479,5 +483,5 @@ cudaError_t lorc_generic_decode(const lorc_ctx* ctx, const LorcLayer& L, const C
     *launches += 1;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    return lorc_generic_combine(ctx, L, cv.batch, n_splits, part_ml, part_o, out, st, launches);
+    return lorc_generic_combine(ctx, L, cv.batch, n_splits, part_ml, part_o, out, st, launches, latent_out);
 }

@@ -277,8 +277,8 @@ int lorc_append(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* x
     return LORC_OK;
 }
 
-int lorc_decode_attn(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* q, void* out,
-                     int n_splits, void* stream) {
+static int decode_attn_impl(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* q, void* out,
+                            int n_splits, void* stream, bool latent_out) {
     LorcLayer* L;
     int rc = get_layer(ctx, layer, &L);
     if (rc) return rc;
@@ -286,6 +286,8 @@ int lorc_decode_attn(lorc_ctx* ctx, int layer, const lorc_cache* cache, const vo
     if (((uintptr_t)q & 15) || ((uintptr_t)out & 15))
         return fail(ctx, LORC_ERR_ARG, "decode_attn: q and out must be 16-byte aligned");
     if (n_splits < 0) return fail(ctx, LORC_ERR_ARG, "decode_attn: negative n_splits");
+    if (latent_out && L->mode != LORC_MODE_LATENT)
+        return fail(ctx, LORC_ERR_UNSUPPORTED, "decode_attn_latent_out: the layer is not compressed");
     CacheView cv;
     rc = check_cache(ctx, cache, *L, &cv);
     if (rc) return rc;
@@ -300,7 +302,7 @@ int lorc_decode_attn(lorc_ctx* ctx, int layer, const lorc_cache* cache, const vo
         size_t tc = lorc_tc_workspace_bytes(ctx, cv.batch, cv.max_seq_len);
         if (tc > ctx->ws_bytes) return fail(ctx, LORC_ERR_WORKSPACE, "decode_attn: workspace too small");
         e = lorc_tc_decode(ctx, layer, *L, cv, (const bf16*)q, (bf16*)out, n_splits, ctx->ws,
-                           ctx->ws_bytes, st, &launches);
+                           ctx->ws_bytes, st, &launches, latent_out);
         ctx->launches += launches;
         ctx->last_path = 2;
         if (e != cudaSuccess) return fail_cuda(ctx, e, "lorc_decode_attn (tensor-core path)");
@@ -317,11 +319,21 @@ int lorc_decode_attn(lorc_ctx* ctx, int layer, const lorc_cache* cache, const vo
     if (w.total > ctx->ws_bytes) return fail(ctx, LORC_ERR_WORKSPACE, "decode_attn: workspace too small");
     float* part_ml = (float*)((char*)ctx->ws + w.off_ml);
     float* part_o = (float*)((char*)ctx->ws + w.off_o);
-    e = lorc_generic_decode(ctx, *L, cv, (const bf16*)q, (bf16*)out, S, part_ml, part_o, st, &launches);
+    e = lorc_generic_decode(ctx, *L, cv, (const bf16*)q, (bf16*)out, S, part_ml, part_o, st, &launches, latent_out);
     ctx->launches += launches;
     ctx->last_path = lorc_full_decode_supported(ctx, *L) ? 3 : 1;
     if (e != cudaSuccess) return fail_cuda(ctx, e, "lorc_decode_attn");
     return LORC_OK;
+}
+
+int lorc_decode_attn(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* q, void* out,
+                     int n_splits, void* stream) {
+    return decode_attn_impl(ctx, layer, cache, q, out, n_splits, stream, false);
+}
+
+int lorc_decode_attn_latent_out(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* q, void* o_lat,
+                                int n_splits, void* stream) {
+    return decode_attn_impl(ctx, layer, cache, q, o_lat, n_splits, stream, true);
 }
 
 int lorc_decode_step_host(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* x_host,

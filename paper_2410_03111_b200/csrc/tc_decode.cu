@@ -121,7 +121,8 @@ static bool build_cache_maps(LorcTcLayer& T, const LorcLayer& L, const CacheView
 }
 
 cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const CacheView& cv, const bf16* q,
-                           bf16* out, int n_splits, void* ws, size_t ws_bytes, cudaStream_t st, int* launches) {
+                           bf16* out, int n_splits, void* ws, size_t ws_bytes, cudaStream_t st, int* launches,
+                           bool latent_out) {
     LorcTcState* T = tc_state(ctx);
     LorcTcLayer& TL = T->layers[layer];
     const lorc_model_desc& d = ctx->desc;
@@ -192,7 +193,7 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
         if (e != cudaSuccess) return e;
     }
     const cudaError_t e2 = lorc_tc_pv_launch(ctx, L, cv, TL.mapCV, TL.mapBVT, pimg, T->rowmax, tiles, plan, pv_scratch,
-                                             out, st, launches);
+                                             out, latent_out, st, launches);
     if (e2 == cudaSuccess) T->rowmax_dirty = false;
     return e2;
 }

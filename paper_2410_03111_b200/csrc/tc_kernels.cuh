@@ -12,9 +12,10 @@ bool lorc_tc_append_supported(const lorc_ctx* ctx, const LorcLayer& L, const Cac
 // Scratch bytes the tensor-core decode path needs for (batch, max_seq_len), any layer.
 size_t lorc_tc_workspace_bytes(const lorc_ctx* ctx, int batch, int max_seq_len);
 
+// latent_out: `out` receives the normalised latent output [b, H_q, r_v] instead of the up-projected one.
 cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const CacheView& cv,
                            const bf16* q, bf16* out, int n_splits, void* ws, size_t ws_bytes,
-                           cudaStream_t st, int* launches);
+                           cudaStream_t st, int* launches, bool latent_out = false);
 cudaError_t lorc_tc_append(lorc_ctx* ctx, int layer, const LorcLayer& L, const CacheView& cv,
                            const bf16* x, int T, cudaStream_t st, int* launches);
 
@@ -57,7 +58,8 @@ void lorc_tc_pv_plan(const lorc_ctx* ctx, const LorcLayer& L, const CacheView& c
                      LorcPvPlan* plan);
 cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, const CUtensorMap& mapCV,
                               const CUtensorMap& mapBVT, const uint8_t* pimg, unsigned* rowmax, int tiles,
-                              const LorcPvPlan& plan, void* scratch, bf16* out, cudaStream_t st, int* launches);
+                              const LorcPvPlan& plan, void* scratch, bf16* out, bool latent_out, cudaStream_t st,
+                              int* launches);
 
 // A_cat [D, R] (row-major) -> fragment order [R/8][D/32][32 lanes][8] used by the fast append kernel.  The first
 // pair_cols columns (uncompressed mode with half-split rotary pairs: the key columns; otherwise 0) are laid out with the

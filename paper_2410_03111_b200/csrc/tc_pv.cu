@@ -534,6 +534,20 @@ lorc_upproj_kernel(const __grid_constant__ CUtensorMap mapON, const __grid_const
     if (warp == 1) tmem_dealloc(tmem, 32);
 }
 
+// Result of lorc_decode_attn_latent_out: the normalised latent output without the padding columns, and the row maxima
+// left empty for the next call (what the up-projection kernel does otherwise).
+__global__ void latent_out_kernel(const bf16* __restrict__ o_norm, bf16* __restrict__ o_lat, unsigned* rowmax, int rows,
+                                  int r_v, int r_pad) {
+    grid_dep_wait();
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < rows) rowmax[i] = 0u;
+    const int vec = r_v / 8;                              // r_v is a multiple of 8: 16-byte pieces
+    if (i < (long long)rows * vec) {
+        const long long row = i / vec, c = i % vec;
+        reinterpret_cast<uint4*>(o_lat + row * r_v)[c] = reinterpret_cast<const uint4*>(o_norm + row * r_pad)[c];
+    }
+}
+
 // Column blocks and context shares of one PV launch: one CTA per SM, and as few context shares as fill the SMs once
 // (a CTA with four stages in flight pulls its share of the HBM bandwidth alone; fewer shares mean longer streams per
 // CTA and, at one share, no share reduction at all).
@@ -621,7 +635,8 @@ void lorc_tc_pv_plan(const lorc_ctx* ctx, const LorcLayer& L, const CacheView& c
 // score kernel clears it).
 cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, const CUtensorMap& mapCV,
                               const CUtensorMap& mapBVT, const uint8_t* pimg, unsigned* rowmax, int tiles,
-                              const LorcPvPlan& plan, void* scratch, bf16* out, cudaStream_t st, int* launches) {
+                              const LorcPvPlan& plan, void* scratch, bf16* out, bool latent_out, cudaStream_t st,
+                              int* launches) {
     const lorc_model_desc& d = ctx->desc;
     const int n_blk = plan.n_blk, n_csplit = plan.n_csplit;
     const int r_pad = n_blk * 128;
@@ -646,6 +661,14 @@ cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView
         if (e != cudaSuccess) return e;
     }
     LorcStageTimer timer(ctx, LORC_STAGE_COMBINE, st);
+    if (latent_out) {
+        const int rows = cv.batch * d.n_q_heads;
+        const long long work = (long long)rows * (L.r_v / 8);
+        e = lorc_launch_dependent(latent_out_kernel, dim3((unsigned)((work + 255) / 256)), dim3(256), 0, st,
+                                  (const bf16*)o_norm, out, rowmax, rows, L.r_v, r_pad);
+        *launches += 1;
+        return e;
+    }
     // o_norm [b, H_q, r_pad] as (rho, head, sequence) with boxes of 64 rho x G heads x 64/G sequences
     CUtensorMap mapON;
     {

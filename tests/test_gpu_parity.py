@@ -351,3 +351,30 @@ def test_errors_are_reported_not_raised_on_the_device():
         L.lorc_load_factors(sess.ctx, 0, 0, 12, 32, *sess.dev)     # rank not a multiple of 8
     assert e.value.code == L.LORC_ERR_ARG
     sess.close()
+
+
+@pytest.mark.parametrize("flags", [1, 0])
+def test_latent_output_entry_plain_kernels(flags):
+    """lorc_decode_attn_latent_out on the plain kernels (merge without up-projection)."""
+    import torch
+    D, H_q, H_kv, d_h, r_k, r_v = 256, 4, 2, 64, 40, 24
+    lens = [150, 33]
+    prob = H.Problem(D, H_q, H_kv, d_h, r_k, r_v, theta=10000.0, layer=11)
+    sess = H.Session(prob, max_pos=160, batch=2, flags=flags)
+    ck, cv = H.oracle_latents(prob, _xs(lens, D, 11))
+    held = H.contiguous_cache(sess, 2, 160, lens, ck, cv)
+    q = synth.queries(2, H_q, d_h, 11, 0, 8.0).astype(np.float64)
+    o_lat = torch.zeros(2, H_q, r_v, dtype=torch.bfloat16, device="cuda")
+    sess.L.lorc_decode_attn_latent_out(sess.ctx, 0, held[0], H.dev_bf16(q), o_lat, n_splits=3)
+    assert sess.L.lorc_sync_status(sess.ctx) == 0
+    for s in range(2):
+        want = O.decode_attn_latent_out(ck[s], cv[s], prob.B_k, q[s], H_kv, prob.theta)
+        assert O.rel_l2_rows(H.host_f64(o_lat[s]), want) <= TOL_BF16
+    # an uncompressed layer has no latent output
+    full = H.Session(prob, max_pos=160, batch=2, flags=flags, mode=1)
+    heldf = H.contiguous_cache(full, 2, 160, lens)
+    with pytest.raises(sess.L.LorcError) as e:
+        sess.L.lorc_decode_attn_latent_out(full.ctx, 0, heldf[0], H.dev_bf16(q), o_lat)
+    assert e.value.code == sess.L.LORC_ERR_UNSUPPORTED
+    full.close()
+    sess.close()

@@ -316,3 +316,34 @@ def test_tc_decode_without_rotation_uses_the_absorbed_scores(r_k, r_v, lens, pag
         worst = max(worst, O.rel_l2_rows(got, want))
     print(f"\n[no rotation] r_k {r_k}: max relative L2 row error {worst:.2e}")
     sess.close()
+
+
+@pytest.mark.parametrize("style", [0, H.ROPE_NONE])
+def test_tc_latent_output_entry(style):
+    """lorc_decode_attn_latent_out on the tensor-core path: the normalised latent output [b, H_q, r_v] against the
+    oracle, and its product with B_V against lorc_decode_attn's result."""
+    import torch
+    r_k, r_v, lens = 256, 200, [700, 130, 1]
+    prob = H.Problem(GEOM["D"], GEOM["H_q"], GEOM["H_kv"], GEOM["d_h"], r_k, r_v, theta=500000.0, layer=22, style=style)
+    b, n_max = len(lens), max(lens) + 3
+    sess = H.Session(prob, max_pos=n_max, batch=b)
+    ck, cv = _latents(prob, lens, 22)
+    held = H.contiguous_cache(sess, b, n_max, lens, ck, cv)
+    q = synth.queries(b, GEOM["H_q"], GEOM["d_h"], 22, 1, 8.0).astype(np.float64)
+    o_lat = torch.zeros(b, GEOM["H_q"], r_v, dtype=torch.bfloat16, device="cuda")
+    sess.L.lorc_decode_attn_latent_out(sess.ctx, 0, held[0], H.dev_bf16(q), o_lat)
+    assert sess.L.lorc_sync_status(sess.ctx) == 0, sess.L.lorc_last_error(sess.ctx)
+    assert sess.L.lorc_last_path(sess.ctx) == 2
+    got = H.host_f64(o_lat)
+    for s in range(b):
+        want = O.decode_attn_latent_out(ck[s], cv[s], prob.B_k, q[s], GEOM["H_kv"], prob.theta,
+                                        use_rope=style != H.ROPE_NONE)
+        assert O.rel_l2_rows(got[s], want) <= TOL
+    # the ordinary entry afterwards (the row maxima were left empty) agrees with o_lat . B_V
+    out = H.host_f64(_run(sess, held[0], q))
+    G = GEOM["H_q"] // GEOM["H_kv"]
+    for h in range(GEOM["H_q"]):
+        g = h // G
+        proj = got[:, h, :] @ prob.B_v[:, g * 128:(g + 1) * 128]
+        assert O.rel_l2_rows(out[:, h, :], proj) <= TOL
+    sess.close()

@@ -436,3 +436,27 @@ def test_eckart_young_benchmark_spectra(n, p, r, tail, eps):
     A, B = O.factors_from_generators(U, s, V, r)
     assert abs(O.relative_frobenius_error(W, A @ B) - eps) <= 1e-9
     assert abs(float(np.sum((W - A @ B) ** 2)) - tail) <= 1e-9
+
+
+def test_latent_output_times_value_factor_is_the_attention_output():
+    """decode_attn_latent_out (Sec. 3.1, the W_o' fold): multiplying by B_V[:, g(h)] gives decode_attn_latent; with a
+    single cached token it is that token's latent; its rows are convex combinations of the cached latents."""
+    D, H_q, H_kv, d_h, r_k, r_v, N = 96, 8, 2, 16, 24, 20, 37
+    n = H_kv * d_h
+    Uk, sk, Vk = synth.synth_weight_factors(D, n, 0.8, 4, "k")
+    Uv, sv, Vv = synth.synth_weight_factors(D, n, 0.8, 4, "v")
+    Ak, Bk = O.factors_from_generators(Uk, sk, Vk, r_k)
+    Av, Bv = O.factors_from_generators(Uv, sv, Vv, r_v)
+    x = synth.hidden_states(N, D, 4).astype(np.float64)
+    q = synth.queries(1, H_q, d_h, 4, 0, 8.0)[0].astype(np.float64)
+    ck, cv = O.append_latent(x, Ak), O.append_latent(x, Av)
+    for use_rope in (True, False):
+        o_lat = O.decode_attn_latent_out(ck, cv, Bk, q, H_kv, 10000.0, use_rope=use_rope)
+        full = O.decode_attn_latent(ck, cv, Bk, Bv, q, H_kv, 10000.0, use_rope=use_rope)
+        G = H_q // H_kv
+        for h in range(H_q):
+            g = h // G
+            assert np.allclose(o_lat[h] @ Bv[:, g * d_h:(g + 1) * d_h], full[h], atol=1e-12)
+        assert np.all(o_lat.min(axis=0) >= cv.min(axis=0) - 1e-12) and np.all(o_lat.max(axis=0) <= cv.max(axis=0) + 1e-12)
+    one = O.decode_attn_latent_out(ck[:1], cv[:1], Bk, q, H_kv, 10000.0)
+    assert np.allclose(one, np.tile(cv[0], (H_q, 1)), atol=1e-14)
