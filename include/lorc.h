@@ -188,6 +188,21 @@ int lorc_append(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* x
 int lorc_decode_attn(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* q, void* out,
                      int n_splits, void* stream);
 
+/* Prompt processing: attention of the T newest tokens of every sequence (a whole prompt, or one chunk of it) over the
+ * latent cache.  Preliminary section's Attention(Q, K, V) with the usual causal mask; keys and values come from the
+ * cached latents as in lorc_decode_attn (Sec. 3.1), rotated at attention time (appendix).
+ *   q   [batch, T, n_q_heads, d_head] device bf16, un-rotated; out the same shape.
+ *   The T tokens must already be in the cache (lorc_append first) and counted in seq_lens: query t of sequence s sits
+ *   at position seq_lens[s] - T + t and attends to positions 0 .. seq_lens[s] - T + t (the cached prefix in full, the
+ *   new chunk causally).  With T = 1 the result equals lorc_decode_attn's.
+ * On the tensor-core path every key and value of the layer is reconstructed once into the workspace (a transient
+ * bf16 buffer: the method's saving is in the cache, not in this scratch), then attended with a flash-attention
+ * kernel; every call reconstructs the whole cached sequence, so chunks should be large.  Needs a workspace of
+ * lorc_prefill_workspace_bytes(ctx, batch, max_seq_len, T).  A sequence with seq_lens[s] < T sets status ARG.
+ * Errors: ARG, LAYER, WORKSPACE; CAPACITY / EMPTY through the status word. */
+size_t lorc_prefill_workspace_bytes(const lorc_ctx* ctx, int batch, int max_seq_len, int T);
+int lorc_prefill_attn(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* q, void* out, int T, void* stream);
+
 /* Decode attention that stops before the value up-projection (Sec. 3.1, the W_o' equation: the orthonormal value
  * factor can be folded into the output projection, W_o' = B_V,g W_o,h stacked over the heads).  Same arguments as
  * lorc_decode_attn except the result:

@@ -273,6 +273,26 @@ def decode_attn_latent_out(c_k: np.ndarray, c_v: np.ndarray, B_k: np.ndarray, q:
     return out
 
 
+def prefill_attn_latent(c_k: np.ndarray, c_v: np.ndarray, B_k: np.ndarray, B_v: np.ndarray, q: np.ndarray,
+                        n_kv_heads: int, theta: float, style: int = ROPE_HALF_SPLIT,
+                        use_rope: bool = True) -> np.ndarray:
+    """Attention of the T newest tokens of one sequence over its latent cache (prompt processing in chunks).
+
+    c_k [N, r_k], c_v [N, r_v] hold ALL N cached tokens, the T new ones last; q [T, H_q, d_h] are their un-rotated
+    queries.  Query t sits at position N - T + t and attends to the tokens at positions 0 .. N - T + t (the cached
+    prefix in full, the new chunk causally): the Preliminary section's Attention(Q, K, V) with the usual causal mask,
+    keys and values reconstructed from the latents as in decode_attn_latent.  Written as that function applied to
+    each query with the cache cut after its own position.  Returns [T, H_q, d_h]."""
+    q = np.asarray(q, dtype=np.float64)
+    T = q.shape[0]
+    N = np.asarray(c_k).shape[0]
+    out = np.empty(q.shape, dtype=np.float64)
+    for t in range(T):
+        n_t = N - T + t + 1
+        out[t] = decode_attn_latent(c_k[:n_t], c_v[:n_t], B_k, B_v, q[t], n_kv_heads, theta, style, use_rope=use_rope)
+    return out
+
+
 def decode_attn_full(x: np.ndarray, W_k: np.ndarray, W_v: np.ndarray, q: np.ndarray,
                      n_kv_heads: int, theta: float, style: int = ROPE_HALF_SPLIT,
                      positions=None, q_position=None, use_rope: bool = True) -> np.ndarray:

@@ -69,6 +69,8 @@ def _signatures():
         "lorc_append": ([vp, i32, cp, vp, i32, vp], i32),
         "lorc_decode_attn": ([vp, i32, cp, vp, vp, i32, vp], i32),
         "lorc_decode_attn_latent_out": ([vp, i32, cp, vp, vp, i32, vp], i32),
+        "lorc_prefill_workspace_bytes": ([vp, i32, i32, i32], C.c_size_t),
+        "lorc_prefill_attn": ([vp, i32, cp, vp, vp, i32, vp], i32),
         "lorc_decode_attn_static": ([vp, i32, cp, vp, vp, i32, vp], i32),
         "lorc_decode_step_host": ([vp, i32, cp, vp, vp, vp, i32, vp], i32),
         "lorc_sync_status": ([vp, vp], i32),
@@ -170,6 +172,14 @@ def lorc_append(ctx, layer, cache, x, T=1, stream=None):
 def lorc_decode_attn(ctx, layer, cache, q, out, n_splits=0, stream=None):
     _check(ctx, _lib.lorc_decode_attn(ctx, layer, C.byref(cache), _ptr(q), _ptr(out), n_splits,
                                        _stream(stream)))
+
+
+def lorc_prefill_workspace_bytes(ctx, batch, max_seq_len, T):
+    return int(_lib.lorc_prefill_workspace_bytes(ctx, batch, max_seq_len, T))
+
+
+def lorc_prefill_attn(ctx, layer, cache, q, out, T, stream=None):
+    _check(ctx, _lib.lorc_prefill_attn(ctx, layer, C.byref(cache), _ptr(q), _ptr(out), T, _stream(stream)))
 
 
 def lorc_decode_attn_latent_out(ctx, layer, cache, q, o_lat, n_splits=0, stream=None):

@@ -127,9 +127,11 @@ bool lorc_full_decode_supported(const lorc_ctx* ctx, const LorcLayer& L);
 cudaError_t lorc_full_decode(const lorc_ctx* ctx, const CacheView& cv, const bf16* q, int n_splits, float* part_ml,
                              float* part_o, cudaStream_t st, int* launches);
 // latent_out: stop before the value up-projection and write the normalised latent output [b, H_q, r_v] to `out`.
+// T > 1: T queries per sequence (q, out [b, T, H_q, d_head]; partial results for b * T units), query t of a sequence
+// at position seq_lens[s] - T + t, attending to the tokens up to its own.
 cudaError_t lorc_generic_decode(const lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv,
                                 const bf16* q, bf16* out, int n_splits, float* part_ml,
-                                float* part_o, cudaStream_t st, int* launches, bool latent_out = false);
+                                float* part_o, cudaStream_t st, int* launches, bool latent_out = false, int T = 1);
 // Merge of split partials + value up-projection (also used by the tensor-core path):
 // part_ml [b, H_q, S, 2] (running max in natural-log units, sum), part_o [b, H_q, S, W].
 cudaError_t lorc_generic_combine(const lorc_ctx* ctx, const LorcLayer& L, int batch, int n_splits,

@@ -178,7 +178,7 @@ __global__ void __launch_bounds__(128)
 decode_generic_kernel(const bf16* __restrict__ q, CacheView cv, const bf16* __restrict__ B_k, int r_k,
                       int r_v, int n, int G, int n_splits, int rope_style,
                       const float2* __restrict__ rope_table, int max_pos, float* __restrict__ part_ml,
-                      float* __restrict__ part_o, int* status) {
+                      float* __restrict__ part_o, int* status, int T) {
     constexpr int HALF = DH / 2;
     constexpr int SUB = 128 / DH;            // token subsets when DH < 128
     constexpr int TPS = GEN_TILE / SUB;      // tokens per thread in the reconstruction
@@ -191,10 +191,14 @@ decode_generic_kernel(const bf16* __restrict__ q, CacheView cv, const bf16* __re
     __shared__ long long row_s[GEN_TILE];
 
     const int tid = threadIdx.x;
-    const int split = blockIdx.x, g = blockIdx.y, s = blockIdx.z;
+    // With T queries per sequence (prompt processing) blockIdx.z runs over (sequence, query): query t of a chunk of T
+    // sits at position seq_lens[s] - T + t and sees the tokens up to its own, i.e. it is the decode query of the
+    // sequence cut after that token.  sq indexes queries, partial results and outputs; s the cache.
+    const int split = blockIdx.x, g = blockIdx.y, sq = blockIdx.z, s = sq / T;
     const int H_q = G * (int)gridDim.y;
     const int W = LATENT ? r_v : DH;         // width of the output accumulator
-    const int len = cv.seq_lens[s];
+    int len = cv.seq_lens[s];
+    if (T > 1) len = len >= T ? len - (T - 1 - sq % T) : 0;
 
     // token range of this split
     int tiles = (len + GEN_TILE - 1) / GEN_TILE;
@@ -217,7 +221,7 @@ decode_generic_kernel(const bf16* __restrict__ q, CacheView cv, const bf16* __re
             int h = i / HALF, jj = i - h * HALF;
             int ia = (rope_style == LORC_ROPE_HALF_SPLIT) ? jj : 2 * jj;
             int ib = (rope_style == LORC_ROPE_HALF_SPLIT) ? jj + HALF : 2 * jj + 1;
-            const bf16* qp = q + ((long long)s * H_q + g * G + h) * DH;
+            const bf16* qp = q + ((long long)sq * H_q + g * G + h) * DH;
             float a = __bfloat162float(qp[ia]), b = __bfloat162float(qp[ib]);
             float2 cs = rope_table[(long long)qpos * HALF + jj];
             qs[h][ia] = (a * cs.x - b * cs.y) * scale;
@@ -360,7 +364,7 @@ decode_generic_kernel(const bf16* __restrict__ q, CacheView cv, const bf16* __re
 #pragma unroll
     for (int h = 0; h < GEN_GMAX; ++h) {
         if (h >= G) break;
-        long long unit = ((long long)s * H_q + g * G + h) * n_splits + split;
+        long long unit = ((long long)sq * H_q + g * G + h) * n_splits + split;
         if (tid == 0) {
             part_ml[unit * 2 + 0] = m_s[h];
             part_ml[unit * 2 + 1] = l_s[h];
@@ -453,12 +457,12 @@ cudaError_t lorc_generic_combine(const lorc_ctx* ctx, const LorcLayer& L, int ba
 
 cudaError_t lorc_generic_decode(const lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv,
                                 const bf16* q, bf16* out, int n_splits, float* part_ml,
-                                float* part_o, cudaStream_t st, int* launches, bool latent_out) {
+                                float* part_o, cudaStream_t st, int* launches, bool latent_out, int T) {
     const lorc_model_desc& d = ctx->desc;
     const int G = ctx->group;
     const bool latent = (L.mode == LORC_MODE_LATENT);
-    dim3 grid(n_splits, d.n_kv_heads, cv.batch);
-    if (lorc_full_decode_supported(ctx, L)) {
+    dim3 grid(n_splits, d.n_kv_heads, cv.batch * T);
+    if (T == 1 && lorc_full_decode_supported(ctx, L)) {
         // uncompressed mode with 128-wide heads: the streaming kernel on the warp-level tensor cores
         {
             LorcStageTimer timer(ctx, LORC_STAGE_SCORE, st);
@@ -472,7 +476,7 @@ cudaError_t lorc_generic_decode(const lorc_ctx* ctx, const LorcLayer& L, const C
 #define LAUNCH_DEC(DHV, LAT)                                                                      \
     decode_generic_kernel<DHV, LAT><<<grid, 128, 0, st>>>(                                        \
         q, cv, L.B_k, L.r_k, L.r_v, ctx->n, G, n_splits, ctx->pair_style, ctx->rope_table, d.max_pos, \
-        part_ml, part_o, ctx->status_dev)
+        part_ml, part_o, ctx->status_dev, T)
     if (d.d_head == 128) {
         if (latent) LAUNCH_DEC(128, true); else LAUNCH_DEC(128, false);
     } else {
@@ -483,5 +487,5 @@ cudaError_t lorc_generic_decode(const lorc_ctx* ctx, const LorcLayer& L, const C
     *launches += 1;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    return lorc_generic_combine(ctx, L, cv.batch, n_splits, part_ml, part_o, out, st, launches, latent_out);
+    return lorc_generic_combine(ctx, L, cv.batch * T, n_splits, part_ml, part_o, out, st, launches, latent_out);
 }

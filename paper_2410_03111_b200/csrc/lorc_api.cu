@@ -336,6 +336,58 @@ int lorc_decode_attn_latent_out(lorc_ctx* ctx, int layer, const lorc_cache* cach
     return decode_attn_impl(ctx, layer, cache, q, o_lat, n_splits, stream, true);
 }
 
+size_t lorc_prefill_workspace_bytes(const lorc_ctx* ctx, int batch, int max_seq_len, int T) {
+    if (!ctx || batch <= 0 || max_seq_len <= 0 || T <= 0) return 0;
+    int S = generic_default_splits(max_seq_len);
+    size_t gen = ws_layout(ctx, batch * T, S, ctx->n).total;
+    size_t tc = lorc_tc_workspace_bytes(ctx, batch, max_seq_len) ? lorc_tc_prefill_scratch_bytes(ctx, batch, max_seq_len, T) : 0;
+    return (gen > tc ? gen : tc) + 256;
+}
+
+int lorc_prefill_attn(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* q, void* out, int T, void* stream) {
+    LorcLayer* L;
+    int rc = get_layer(ctx, layer, &L);
+    if (rc) return rc;
+    if (!q || !out || T <= 0) return fail(ctx, LORC_ERR_ARG, "prefill_attn: null q or out, or non-positive T");
+    if (((uintptr_t)q & 15) || ((uintptr_t)out & 15))
+        return fail(ctx, LORC_ERR_ARG, "prefill_attn: q and out must be 16-byte aligned");
+    CacheView cv;
+    rc = check_cache(ctx, cache, *L, &cv);
+    if (rc) return rc;
+    if (T > cv.max_seq_len) return fail(ctx, LORC_ERR_ARG, "prefill_attn: T exceeds max_seq_len");
+    if (!ctx->ws) return fail(ctx, LORC_ERR_WORKSPACE, "prefill_attn: no workspace set");
+    cudaStream_t st = (cudaStream_t)stream;
+    int launches = 0;
+    cudaError_t e;
+    if (!(ctx->desc.flags & LORC_FLAG_DEBUG_FP32) && lorc_tc_prefill_supported(ctx, *L, cv)) {
+        if (lorc_tc_prefill_scratch_bytes(ctx, cv.batch, cv.max_seq_len, T) > ctx->ws_bytes)
+            return fail(ctx, LORC_ERR_WORKSPACE, "prefill_attn: workspace too small (see lorc_prefill_workspace_bytes)");
+        LorcStageTimer timer(ctx, LORC_STAGE_SCORE, st);
+        e = lorc_tc_prefill(ctx, layer, *L, cv, (const bf16*)q, (bf16*)out, T, ctx->ws, ctx->ws_bytes, st, &launches);
+        ctx->launches += launches;
+        ctx->last_path = 2;
+        if (e != cudaSuccess) return fail_cuda(ctx, e, "lorc_prefill_attn (tensor-core path)");
+        return LORC_OK;
+    }
+    // plain kernels: every (sequence, query) is a decode query over the sequence cut after its own token
+    const bool latent = (L->mode == LORC_MODE_LATENT);
+    const int W = latent ? L->r_v : ctx->desc.d_head;
+    int S = generic_default_splits(cv.max_seq_len);
+    int tiles = (cv.max_seq_len + LORC_GENERIC_TILE - 1) / LORC_GENERIC_TILE;
+    if (S > tiles) S = tiles;
+    while (S > 1 && ws_layout(ctx, cv.batch * T, S, W).total > ctx->ws_bytes) --S;
+    WsLayout w = ws_layout(ctx, cv.batch * T, S, W);
+    if (w.total > ctx->ws_bytes)
+        return fail(ctx, LORC_ERR_WORKSPACE, "prefill_attn: workspace too small (see lorc_prefill_workspace_bytes)");
+    float* part_ml = (float*)((char*)ctx->ws + w.off_ml);
+    float* part_o = (float*)((char*)ctx->ws + w.off_o);
+    e = lorc_generic_decode(ctx, *L, cv, (const bf16*)q, (bf16*)out, S, part_ml, part_o, st, &launches, false, T);
+    ctx->launches += launches;
+    ctx->last_path = 1;
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "lorc_prefill_attn");
+    return LORC_OK;
+}
+
 int lorc_decode_step_host(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* x_host,
                           const void* q_host, void* out_host, int n_splits, void* stream) {
     LorcLayer* L;

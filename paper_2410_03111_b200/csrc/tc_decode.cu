@@ -22,6 +22,7 @@ constexpr int KC = 64;               // latent columns per TMA box
 struct LorcTcLayer {
     bool has_bkt = false;
     CUtensorMap mapBKT, mapBVT;         // B_K^T in 64 x 128 swizzled boxes; B_V^T in 64 x 32 swizzled boxes
+    CUtensorMap mapBVT128;              // B_V^T in 64 x 128 boxes (reconstruction of values for prompt processing)
     // cache maps are rebuilt only when the cache geometry or pointers change
     const void* k_ptr = nullptr;
     const void* v_ptr = nullptr;
@@ -120,11 +121,9 @@ static bool build_cache_maps(LorcTcLayer& T, const LorcLayer& L, const CacheView
     return true;
 }
 
-cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const CacheView& cv, const bf16* q,
-                           bf16* out, int n_splits, void* ws, size_t ws_bytes, cudaStream_t st, int* launches,
-                           bool latent_out) {
-    LorcTcState* T = tc_state(ctx);
-    LorcTcLayer& TL = T->layers[layer];
+// One-time tables and attributes of the context, the layer's factor maps, and the cache maps for this call.
+static cudaError_t tc_prepare(lorc_ctx* ctx, LorcTcState* T, LorcTcLayer& TL, const LorcLayer& L, const CacheView& cv,
+                              cudaStream_t st) {
     const lorc_model_desc& d = ctx->desc;
     if (!T->rope_tile) {
         cudaError_t e = cudaMalloc(&T->rope_tile, sizeof(float2) * 64 * 33);
@@ -136,6 +135,7 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
         cudaError_t e = lorc_tc_score_set_attrs();
         if (e == cudaSuccess) e = lorc_tc_pv_set_attrs();
         if (e == cudaSuccess) e = lorc_tc_absorbed_set_attrs();
+        if (e == cudaSuccess) e = lorc_tc_prefill_set_attrs();
         if (e != cudaSuccess) return e;
         T->attrs_set = true;
     }
@@ -146,10 +146,25 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
         uint64_t d2[2] = {(uint64_t)L.r_v, (uint64_t)ctx->n}, s2[1] = {(uint64_t)L.r_v * 2};
         uint32_t b2[2] = {KC, 32};          // the up-projection takes a quarter of a head's columns per CTA
         if (!lorc_make_tmap_bf16(&TL.mapBVT, L.B_vT, 2, d2, s2, b2)) return cudaErrorInvalidValue;
+        uint32_t b3[2] = {KC, 128};
+        if (!lorc_make_tmap_bf16(&TL.mapBVT128, L.B_vT, 2, d2, s2, b3)) return cudaErrorInvalidValue;
         TL.has_bkt = true;
     }
     if (!build_cache_maps(TL, L, cv)) return cudaErrorInvalidValue;
 
+    return cudaSuccess;
+}
+
+cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const CacheView& cv, const bf16* q,
+                           bf16* out, int n_splits, void* ws, size_t ws_bytes, cudaStream_t st, int* launches,
+                           bool latent_out) {
+    LorcTcState* T = tc_state(ctx);
+    LorcTcLayer& TL = T->layers[layer];
+    const lorc_model_desc& d = ctx->desc;
+    {
+        cudaError_t e0 = tc_prepare(ctx, T, TL, L, cv, st);
+        if (e0 != cudaSuccess) return e0;
+    }
     const int tiles = (cv.max_seq_len + TILE - 1) / TILE;
     const size_t img_area = tc_image_area_bytes(ctx, cv.batch, cv.max_seq_len);
     const size_t abs_area = tc_absorbed_bytes(ctx, cv.batch);
@@ -196,4 +211,18 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
                                              out, latent_out, st, launches);
     if (e2 == cudaSuccess) T->rowmax_dirty = false;
     return e2;
+}
+
+bool lorc_tc_prefill_supported(const lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv) {
+    return lorc_tc_decode_supported(ctx, L, cv);
+}
+
+cudaError_t lorc_tc_prefill(lorc_ctx* ctx, int layer, const LorcLayer& L, const CacheView& cv, const bf16* q, bf16* out,
+                            int T_new, void* ws, size_t ws_bytes, cudaStream_t st, int* launches) {
+    LorcTcState* T = tc_state(ctx);
+    LorcTcLayer& TL = T->layers[layer];
+    cudaError_t e = tc_prepare(ctx, T, TL, L, cv, st);
+    if (e != cudaSuccess) return e;
+    if (lorc_tc_prefill_scratch_bytes(ctx, cv.batch, cv.max_seq_len, T_new) > ws_bytes) return cudaErrorMemoryAllocation;
+    return lorc_tc_prefill_launch(ctx, L, cv, TL.mapCK, TL.mapCV, TL.mapBKT, TL.mapBVT128, q, out, T_new, ws, st, launches);
 }

@@ -61,6 +61,19 @@ cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView
                               const LorcPvPlan& plan, void* scratch, bf16* out, bool latent_out, cudaStream_t st,
                               int* launches);
 
+// Prompt processing (tc_prefill.cu): attention of the T newest tokens of every sequence (q, out [b, T, H_q, 128]) over
+// the latent cache, causal inside the chunk.  Keys and values are reconstructed once into `scratch`
+// (lorc_tc_prefill_scratch_bytes), then a flash-attention kernel runs over them.  mapBKT / mapBVT128: B_K^T, B_V^T
+// [n, r] in swizzled boxes of 64 latent columns x 128 rows.
+bool lorc_tc_prefill_supported(const lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv);
+size_t lorc_tc_prefill_scratch_bytes(const lorc_ctx* ctx, int batch, int max_seq_len, int T);
+cudaError_t lorc_tc_prefill_set_attrs();
+cudaError_t lorc_tc_prefill_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, const CUtensorMap& mapCK,
+                                   const CUtensorMap& mapCV, const CUtensorMap& mapBKT, const CUtensorMap& mapBVT128,
+                                   const bf16* q, bf16* out, int T, void* scratch, cudaStream_t st, int* launches);
+cudaError_t lorc_tc_prefill(lorc_ctx* ctx, int layer, const LorcLayer& L, const CacheView& cv, const bf16* q, bf16* out,
+                            int T, void* ws, size_t ws_bytes, cudaStream_t st, int* launches);
+
 // A_cat [D, R] (row-major) -> fragment order [R/8][D/32][32 lanes][8] used by the fast append kernel.  The first
 // pair_cols columns (uncompressed mode with half-split rotary pairs: the key columns; otherwise 0) are laid out with the
 // two members of each rotary pair side by side.

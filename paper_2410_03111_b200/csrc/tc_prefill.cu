@@ -1,0 +1,527 @@
+// Prompt processing on the tensor cores (sm_100a): attention of the T newest tokens of every sequence over its latent
+// cache, the cached prefix in full and the new chunk causally (Preliminary section's Attention(Q, K, V) with the usual
+// mask; keys and values reconstructed from the latents of Sec. 3.1, rotation at attention time as in the appendix).
+//
+// With many queries per key the reconstruction is worth keeping: every key and value of the layer is rebuilt ONCE into
+// a transient bf16 buffer (the decode path rebuilds them per query and never stores them), then a flash-attention
+// kernel runs over that buffer.
+//
+//   query kernel        Q^[b, T, H_q, 128] = RoPE(q, position) * log2(e) / sqrt(d_h), fp16
+//   reconstruct kernel  K^[tile, head] = RoPE(C_K[tile, :] . B_K[:, head]),  V[tile, head] = C_V[tile, :] . B_V[:, head]
+//                       one CTA per (128-token tile, KV head): TMA-staged 64-wide slices, tcgen05 (M = 128 tokens,
+//                       N = 128), rotation in the epilogue (thread = token row), 16-bit rows to the buffer: keys as
+//                       fp16 (the scores are then exact to 2^-11 of |q| |k|, four times closer than with bf16 keys;
+//                       a rotated key element must stay below 65504 in magnitude), values as bf16
+//   attention kernel    one CTA per (128 query rows = 128 / G positions x G heads of one KV head): for every 128-key
+//                       tile   S = Q^ K^^T (tcgen05, fp32 in TMEM)  ->  online softmax, thread = query row; the
+//                       probabilities go back into tensor memory as bf16 over the scores  ->  O += P V with P read from
+//                       tensor memory.  The running reference of a row is only raised when a tile exceeds it by more
+//                       than 2^8 (the accumulator is rescaled then), so most tiles need no pass over O.
+#include <cuda_fp16.h>
+#include <math.h>
+
+#include "sm100_ptx.cuh"
+#include "tc_kernels.cuh"
+
+using namespace sm100;
+
+namespace {
+
+constexpr int TILE = 128;
+constexpr int KC = 64;
+constexpr float LOG2E = 1.4426950408889634f;
+
+// ------------------------------------------------------------------------------------------------
+// rotated, scaled queries
+// ------------------------------------------------------------------------------------------------
+__global__ void prefill_query_kernel(const bf16* __restrict__ q, __half* __restrict__ qhat, const int32_t* __restrict__ seq_lens,
+                                     const float2* __restrict__ rope_table, int T, int H_q, int max_pos) {
+    const int t = blockIdx.x, s = blockIdx.y;
+    const int len = seq_lens[s];
+    int pos = len - T + t;
+    if (pos < 0 || pos >= max_pos) pos = 0;                 // such a sequence is rejected by the attention kernel
+    const float scale = rsqrtf(128.f) * LOG2E;
+    for (int i = threadIdx.x; i < H_q * 64; i += blockDim.x) {
+        const int h = i >> 6, j = i & 63;
+        const long long base = (((long long)s * T + t) * H_q + h) * 128;
+        const float a = __bfloat162float(q[base + j]), b = __bfloat162float(q[base + 64 + j]);
+        const float2 cs = rope_table[(long long)pos * 64 + j];
+        qhat[base + j] = __float2half_rn((a * cs.x - b * cs.y) * scale);
+        qhat[base + 64 + j] = __float2half_rn((a * cs.y + b * cs.x) * scale);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// reconstruction of keys (rotated) or values into [b, n_rows, n] bf16
+// ------------------------------------------------------------------------------------------------
+constexpr int R_STAGES = 4;
+constexpr int R_THREADS = 192;       // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+
+struct RecSmem {
+    bf16 A[R_STAGES][TILE * KC];          // latent slice [128 tokens][64]
+    bf16 B[R_STAGES][TILE * KC];          // factor slice [128 features of the head][64]
+    uint64_t full[R_STAGES], empty[R_STAGES], d_full;
+    uint32_t tmem_base;
+};
+
+struct RecParams {
+    bf16* out;                     // [b, n_rows, n]
+    const int32_t* seq_lens;
+    const int32_t* page_table;
+    const float2* rope_table;      // [max_pos][64]
+    int* status;
+    int r, n, n_rows, max_pos;
+    int page_size, max_pages_per_seq, n_pages;
+};
+
+template <bool ROPE>
+__global__ void __launch_bounds__(R_THREADS, 1)
+lorc_reconstruct_kernel(const __grid_constant__ CUtensorMap mapC, const __grid_constant__ CUtensorMap mapBT, const RecParams p) {
+    extern __shared__ uint8_t raw[];
+    RecSmem& sm = *reinterpret_cast<RecSmem*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
+    const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
+    const int tile = blockIdx.x, g = blockIdx.y, s = blockIdx.z;
+    int len = p.seq_lens[s];
+    if (len > p.max_pos || len > p.n_rows) len = 0;          // reported by the attention kernel
+    if (tile * TILE >= len) return;                          // nothing cached in this tile (uniform for the block)
+    const int nkc = (p.r + KC - 1) / KC;
+
+    if (tid == 0) {
+        for (int i = 0; i < R_STAGES; ++i) {
+            mbar_init(&sm.full[i], 1);
+            mbar_init(&sm.empty[i], 1);
+        }
+        mbar_init(&sm.d_full, 1);
+        fence_barrier_init();
+        prefetch_tensormap(&mapC);
+        prefetch_tensormap(&mapBT);
+    }
+    if (warp == 1) {
+        tmem_alloc(&sm.tmem_base, 128);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = sm.tmem_base;
+    bool ok = true;
+
+    if (warp == 0) {
+        for (int kc = 0; kc < nkc && ok; ++kc) {
+            const int st = kc % R_STAGES;
+            if (!mbar_wait(&sm.empty[st], ((kc / R_STAGES) & 1) ^ 1)) { ok = false; break; }
+            if (elect_one()) {
+                mbar_arrive_expect_tx(&sm.full[st], 2 * TILE * KC * 2);
+                if (p.page_table == nullptr) {
+                    tma_load_3d(sm.A[st], &mapC, &sm.full[st], kc * KC, tile * TILE, s);
+                } else {
+                    // one box per page; pages past the end of the sequence (or with a bad table entry) come from page 0
+                    const int ppt = TILE / p.page_size;
+                    for (int pg = 0; pg < ppt; ++pg) {
+                        const int lp = tile * ppt + pg;
+                        int page = 0;
+                        if ((long long)lp * p.page_size < len && lp < p.max_pages_per_seq) {
+                            page = p.page_table[(long long)s * p.max_pages_per_seq + lp];
+                            if (page < 0 || page >= p.n_pages) {
+                                lorc_set_status(p.status, LORC_ERR_CAPACITY);
+                                page = 0;
+                            }
+                        }
+                        tma_load_3d(sm.A[st] + pg * p.page_size * KC, &mapC, &sm.full[st], kc * KC, 0, page);
+                    }
+                }
+                tma_load_2d(sm.B[st], &mapBT, &sm.full[st], kc * KC, g * 128);
+            }
+            __syncwarp();
+        }
+        if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
+    } else if (warp == 1) {
+        const uint32_t idesc = make_idesc_bf16(128, 128, 0, 0);
+        const int nk_last = (p.r - (nkc - 1) * KC + 15) >> 4;
+        for (int kc = 0; kc < nkc && ok; ++kc) {
+            const int st = kc % R_STAGES;
+            if (!mbar_wait(&sm.full[st], (kc / R_STAGES) & 1)) { ok = false; break; }
+            tc_fence_after_sync();
+            const uint32_t a0 = smem_u32(sm.A[st]), b0 = smem_u32(sm.B[st]);
+            if (elect_one()) {
+                const int nk = (kc + 1 < nkc) ? 4 : nk_last;
+                for (int k = 0; k < nk; ++k)
+                    tc_mma_bf16(tmem, make_smem_desc_sw128(a0 + k * 32, 0, 1024), make_smem_desc_sw128(b0 + k * 32, 0, 1024),
+                                idesc, (kc | k) != 0);
+                tc_commit(&sm.empty[st]);
+            }
+            __syncwarp();
+        }
+        if (ok) {
+            if (elect_one()) tc_commit(&sm.d_full);
+            __syncwarp();
+        }
+        if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
+    } else {
+        if (!mbar_wait(&sm.d_full, 0)) ok = false;
+        if (ok) {
+            tc_fence_after_sync();
+            const int quarter = warp % 4;
+            const int row = quarter * 32 + lane;                     // token of the tile = TMEM lane
+            const int pos = tile * TILE + row;
+            bf16* dst = p.out + ((long long)s * p.n_rows + pos) * p.n + g * 128;
+            const float2* cs = p.rope_table + (long long)min(pos, p.max_pos - 1) * 64;
+#pragma unroll
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+                uint32_t ra[32], rb[32];
+                tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + c0, ra);          // elements c0 .. c0 + 31 of the head
+                tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + 64 + c0, rb);     // their partners in the second half
+                tmem_wait_ld();
+                if (pos < p.n_rows) {
+                    uint32_t wa[16], wb[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        float a0 = __uint_as_float(ra[2 * i]), a1 = __uint_as_float(ra[2 * i + 1]);
+                        float b0 = __uint_as_float(rb[2 * i]), b1 = __uint_as_float(rb[2 * i + 1]);
+                        if (ROPE) {
+                            const float4 t = __ldg(reinterpret_cast<const float4*>(cs + c0 + 2 * i));   // (cos, sin) x 2
+                            const float x0 = a0 * t.x - b0 * t.y, y0 = a0 * t.y + b0 * t.x;
+                            const float x1 = a1 * t.z - b1 * t.w, y1 = a1 * t.w + b1 * t.z;
+                            a0 = x0; b0 = y0; a1 = x1; b1 = y1;
+                        }
+                        if (ROPE) {          // keys: fp16
+                            const __half2 pa = __floats2half2_rn(a0, a1), pb = __floats2half2_rn(b0, b1);
+                            wa[i] = *reinterpret_cast<const uint32_t*>(&pa);
+                            wb[i] = *reinterpret_cast<const uint32_t*>(&pb);
+                        } else {             // values: bf16
+                            const __nv_bfloat162 pa = __floats2bfloat162_rn(a0, a1), pb = __floats2bfloat162_rn(b0, b1);
+                            wa[i] = *reinterpret_cast<const uint32_t*>(&pa);
+                            wb[i] = *reinterpret_cast<const uint32_t*>(&pb);
+                        }
+                    }
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        reinterpret_cast<uint4*>(dst + c0)[v] = make_uint4(wa[4 * v], wa[4 * v + 1], wa[4 * v + 2], wa[4 * v + 3]);
+                        reinterpret_cast<uint4*>(dst + 64 + c0)[v] = make_uint4(wb[4 * v], wb[4 * v + 1], wb[4 * v + 2], wb[4 * v + 3]);
+                    }
+                }
+            }
+        }
+        if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, 128);
+}
+
+// ------------------------------------------------------------------------------------------------
+// attention over the reconstructed keys and values
+// ------------------------------------------------------------------------------------------------
+constexpr int F_THREADS = 192;       // warp 0 TMA, warp 1 MMA, warps 2..5 softmax (thread = query row)
+constexpr int F_STAGES = 2;
+constexpr float F_RAISE = 8.f;       // a row's reference is raised only when a tile exceeds it by more than this (log2 units)
+
+struct FaSmem {
+    bf16 Q[2][TILE * KC];                 // query rows [128][two 64-element halves]
+    bf16 K[F_STAGES][2][TILE * KC];       // key tile [128 keys][two halves]
+    bf16 V[F_STAGES][2][TILE * KC];       // value tile [128 keys][two halves]
+    uint64_t q_full, k_full[F_STAGES], v_full[F_STAGES], kv_empty[F_STAGES], s_full, p_ready, o_done;
+    uint32_t tmem_base;
+};
+
+struct FaParams {
+    bf16* out;                     // [b, T, H_q, 128]
+    const int32_t* seq_lens;
+    int* status;
+    int T, H_q, G, n_rows, max_pos;
+};
+
+__global__ void __launch_bounds__(F_THREADS, 1)
+lorc_prefill_attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+                         const __grid_constant__ CUtensorMap mapV, const FaParams p) {
+    extern __shared__ uint8_t raw[];
+    FaSmem& sm = *reinterpret_cast<FaSmem*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
+    const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
+    const int g = blockIdx.y, s = blockIdx.z;
+    const int qp = TILE / p.G;                                // query positions per block
+    const int t0 = blockIdx.x * qp;                           // first position (inside the chunk) of this block
+    int len = p.seq_lens[s];
+    if (len > p.max_pos || len > p.n_rows) {
+        if (tid == 0) lorc_set_status(p.status, LORC_ERR_CAPACITY);
+        len = 0;
+    }
+    if (len < p.T) {                                          // the chunk is not in the cache: nothing to attend
+        if (tid == 0 && len > 0) lorc_set_status(p.status, LORC_ERR_ARG);
+        len = 0;
+    }
+    const int t_last = min(p.T, t0 + qp) - 1;                 // last query position of the block
+    const int n_tiles = len > 0 ? (len - p.T + t_last) / TILE + 1 : 0;
+
+    if (tid == 0) {
+        mbar_init(&sm.q_full, 1);
+        for (int i = 0; i < F_STAGES; ++i) {
+            mbar_init(&sm.k_full[i], 1);
+            mbar_init(&sm.v_full[i], 1);
+            mbar_init(&sm.kv_empty[i], 1);
+        }
+        mbar_init(&sm.s_full, 1);
+        mbar_init(&sm.p_ready, 4);
+        mbar_init(&sm.o_done, 1);
+        fence_barrier_init();
+        prefetch_tensormap(&mapQ);
+        prefetch_tensormap(&mapK);
+        prefetch_tensormap(&mapV);
+    }
+    if (warp == 1) {
+        tmem_alloc(&sm.tmem_base, 256);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = sm.tmem_base;                       // scores / probabilities at column 0, output at column 128
+    bool ok = true;
+
+    if (warp == 0) {
+        if (n_tiles > 0) {
+            if (elect_one()) {
+                // rows of the block: (position t0 + tt, head i of the KV head) -> row tt * G + i; positions past the chunk
+                // read as zero
+                mbar_arrive_expect_tx(&sm.q_full, 2 * TILE * KC * 2);
+                tma_load_4d(sm.Q[0], &mapQ, &sm.q_full, 0, g * p.G, t0, s);
+                tma_load_4d(sm.Q[1], &mapQ, &sm.q_full, 64, g * p.G, t0, s);
+            }
+            __syncwarp();
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const int st = j % F_STAGES;
+                if (!mbar_wait(&sm.kv_empty[st], ((j / F_STAGES) & 1) ^ 1)) { ok = false; break; }
+                if (elect_one()) {
+                    mbar_arrive_expect_tx(&sm.k_full[st], 2 * TILE * KC * 2);
+                    tma_load_3d(sm.K[st][0], &mapK, &sm.k_full[st], g * 128, j * TILE, s);
+                    tma_load_3d(sm.K[st][1], &mapK, &sm.k_full[st], g * 128 + 64, j * TILE, s);
+                    mbar_arrive_expect_tx(&sm.v_full[st], 2 * TILE * KC * 2);
+                    tma_load_3d(sm.V[st][0], &mapV, &sm.v_full[st], g * 128, j * TILE, s);
+                    tma_load_3d(sm.V[st][1], &mapV, &sm.v_full[st], g * 128 + 64, j * TILE, s);
+                }
+                __syncwarp();
+            }
+        }
+        if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
+    } else if (warp == 1) {
+        if (n_tiles > 0) {
+            const uint32_t idesc_s = make_idesc_f16(128, 128);            // S = Q K^T: fp16 operands, both K-major
+            const uint32_t idesc_o = make_idesc_bf16(128, 128, 0, 1);     // O += P V: V is MN-major (a key's elements are contiguous)
+            if (!mbar_wait(&sm.q_full, 0)) ok = false;
+            const uint32_t q0 = smem_u32(sm.Q[0]);
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const int st = j % F_STAGES;
+                if (!mbar_wait(&sm.k_full[st], (j / F_STAGES) & 1)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t k0 = smem_u32(sm.K[st][0]), v0 = smem_u32(sm.V[st][0]);
+                if (elect_one()) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const uint32_t off = (k >> 2) * (TILE * KC * 2) + (k & 3) * 32;
+                        tc_mma_bf16(tmem, make_smem_desc_sw128(q0 + off, 0, 1024), make_smem_desc_sw128(k0 + off, 0, 1024),
+                                    idesc_s, k != 0);
+                    }
+                    tc_commit(&sm.s_full);
+                }
+                __syncwarp();
+                // the softmax warps have replaced the scores by probabilities (and rescaled the output if needed)
+                if (!mbar_wait(&sm.p_ready, j & 1)) { ok = false; break; }
+                if (!mbar_wait(&sm.v_full[st], (j / F_STAGES) & 1)) { ok = false; break; }
+                tc_fence_after_sync();
+                if (elect_one()) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)          // 16 keys per step: 8 columns of packed probabilities, 16 rows of V
+                        tc_mma_bf16_ts(tmem + 128, tmem + k * 8, make_smem_desc_sw128(v0 + k * 2048, TILE * KC * 2, 1024),
+                                       idesc_o, (j | k) != 0);
+                    tc_commit(&sm.kv_empty[st]);
+                    if (j + 1 == n_tiles) tc_commit(&sm.o_done);
+                }
+                __syncwarp();
+            }
+        }
+        if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
+    } else {
+        const int quarter = warp % 4;
+        const int row = quarter * 32 + lane;
+        const int tt = row / p.G, hi = row % p.G;
+        const bool live = len > 0 && t0 + tt < p.T;
+        const int pq = len - p.T + t0 + tt;                     // this row's position: it sees keys 0 .. pq
+        const uint32_t trow = tmem + ((uint32_t)(quarter * 32) << 16);
+        float m_ref = -INFINITY, l = 0.f;
+        for (int j = 0; j < n_tiles && ok; ++j) {
+            if (!mbar_wait(&sm.s_full, j & 1)) { ok = false; break; }
+            tc_fence_after_sync();
+            const int n0 = j * TILE;
+            // pass 1: the tile's maximum over the keys this row may see
+            float mt = -INFINITY;
+#pragma unroll
+            for (int c0 = 0; c0 < TILE; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld32(trow + c0, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (live && n0 + c0 + i <= pq) mt = fmaxf(mt, __uint_as_float(r[i]));
+            }
+            // raise the reference?  (the accesses to tensor memory below are warp-wide: the warp rescales if any of its
+            // rows must, the other rows by a factor of one)
+            const bool raise = mt > m_ref + F_RAISE || (m_ref == -INFINITY && mt > -INFINITY);
+            if (__any_sync(0xffffffffu, raise)) {
+                // what has been accumulated so far shrinks by 2^(old - new)
+                const float alpha = !raise ? 1.f : (m_ref == -INFINITY ? 0.f : exp2f(m_ref - mt));
+                l *= alpha;
+                if (j > 0) {
+#pragma unroll
+                    for (int c0 = 0; c0 < TILE; c0 += 32) {
+                        uint32_t o[32];
+                        tmem_ld32(trow + 128 + c0, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st32(trow + 128 + c0, o);
+                    }
+                }
+                if (raise) m_ref = mt;
+            }
+            // pass 2: probabilities (at most 2^8), rounded to bf16, packed two per column over the scores they came from
+#pragma unroll
+            for (int c0 = 0; c0 < TILE; c0 += 32) {
+                uint32_t r[32], w[16];
+                tmem_ld32(trow + c0, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const bool v0 = live && n0 + c0 + 2 * i <= pq, v1 = live && n0 + c0 + 2 * i + 1 <= pq;
+                    const __nv_bfloat162 pr = __floats2bfloat162_rn(v0 ? exp2f(__uint_as_float(r[2 * i]) - m_ref) : 0.f,
+                                                                    v1 ? exp2f(__uint_as_float(r[2 * i + 1]) - m_ref) : 0.f);
+                    l += __low2float(pr) + __high2float(pr);
+                    w[i] = *reinterpret_cast<const uint32_t*>(&pr);
+                }
+                // columns c0 / 2 .. c0 / 2 + 15 lie below column c0 + 32: every score they overwrite has been read
+                tmem_st16(trow + c0 / 2, w);
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.p_ready);
+        }
+        if (n_tiles > 0 && ok) {
+            if (!mbar_wait(&sm.o_done, 0)) ok = false;
+        }
+        if (ok) {
+            tc_fence_after_sync();
+            const bool has_out = t0 + tt < p.T;                // (rows past the chunk still take part in the warp-wide loads)
+            const float inv = l > 0.f ? 1.f / l : 0.f;
+            // a NaN means non-finite numbers in the cache, the factors or the query (or a key beyond the fp16 range)
+            if (has_out && l != l) lorc_set_status(p.status, LORC_ERR_ARG);
+            if (has_out && !(l > 0.f) && l == l && hi == 0 && g == 0 && tt == 0) lorc_set_status(p.status, LORC_ERR_EMPTY);
+            bf16* dst = p.out + (((long long)s * p.T + (has_out ? t0 + tt : 0)) * p.H_q + g * p.G + hi) * 128;
+#pragma unroll
+            for (int c0 = 0; c0 < TILE; c0 += 32) {
+                uint32_t o[32];
+                if (n_tiles > 0) {
+                    tmem_ld32(trow + 128 + c0, o);
+                    tmem_wait_ld();
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) o[i] = 0u;
+                }
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                    uint32_t w[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(o[v * 8 + 2 * e]) * inv,
+                                                                        __uint_as_float(o[v * 8 + 2 * e + 1]) * inv);
+                        w[e] = *reinterpret_cast<const uint32_t*>(&b2);
+                    }
+                    if (has_out) reinterpret_cast<uint4*>(dst + c0)[v] = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+            }
+        }
+        if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, 256);
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+// scratch: [Q^ | K^ | V], rows of the key / value buffers rounded up to whole tiles
+static size_t prefill_rows(int max_seq_len) { return (size_t)((max_seq_len + TILE - 1) / TILE) * TILE; }
+
+size_t lorc_tc_prefill_scratch_bytes(const lorc_ctx* ctx, int batch, int max_seq_len, int T) {
+    const size_t q = lorc_align_up((size_t)batch * T * ctx->desc.n_q_heads * 128 * sizeof(bf16), 256);
+    const size_t kv = lorc_align_up((size_t)batch * prefill_rows(max_seq_len) * ctx->n * sizeof(bf16), 256);
+    return q + 2 * kv;
+}
+
+cudaError_t lorc_tc_prefill_set_attrs() {
+    cudaError_t e = cudaFuncSetAttribute(lorc_reconstruct_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)sizeof(RecSmem) + 1024);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(lorc_reconstruct_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)sizeof(RecSmem) + 1024);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(lorc_prefill_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)sizeof(FaSmem) + 1024);
+    return e;
+}
+
+cudaError_t lorc_tc_prefill_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, const CUtensorMap& mapCK,
+                                   const CUtensorMap& mapCV, const CUtensorMap& mapBKT, const CUtensorMap& mapBVT128,
+                                   const bf16* q, bf16* out, int T, void* scratch, cudaStream_t st, int* launches) {
+    const lorc_model_desc& d = ctx->desc;
+    const size_t rows = prefill_rows(cv.max_seq_len);
+    const size_t q_bytes = lorc_align_up((size_t)cv.batch * T * d.n_q_heads * 128 * sizeof(bf16), 256);
+    const size_t kv_bytes = lorc_align_up((size_t)cv.batch * rows * ctx->n * sizeof(bf16), 256);
+    bf16* qhat = (bf16*)scratch;
+    bf16* khat = (bf16*)((char*)scratch + q_bytes);
+    bf16* vbuf = (bf16*)((char*)scratch + q_bytes + kv_bytes);
+    const int tiles = (int)(rows / TILE);
+
+    prefill_query_kernel<<<dim3(T, cv.batch), 256, 0, st>>>(q, reinterpret_cast<__half*>(qhat), cv.seq_lens, ctx->rope_table, T,
+                                                            d.n_q_heads, d.max_pos);
+    *launches += 1;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+
+    RecParams rp;
+    rp.seq_lens = cv.seq_lens; rp.page_table = cv.page_table; rp.rope_table = ctx->rope_table; rp.status = ctx->status_dev;
+    rp.n = ctx->n; rp.n_rows = (int)rows; rp.max_pos = d.max_pos;
+    rp.page_size = cv.page_size; rp.max_pages_per_seq = cv.max_pages_per_seq; rp.n_pages = cv.n_pages;
+    dim3 rgrid(tiles, d.n_kv_heads, cv.batch);
+    rp.out = khat; rp.r = L.r_k;
+    lorc_reconstruct_kernel<true><<<rgrid, R_THREADS, sizeof(RecSmem) + 1024, st>>>(mapCK, mapBKT, rp);
+    *launches += 1;
+    rp.out = vbuf; rp.r = L.r_v;
+    lorc_reconstruct_kernel<false><<<rgrid, R_THREADS, sizeof(RecSmem) + 1024, st>>>(mapCV, mapBVT128, rp);
+    *launches += 1;
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+
+    CUtensorMap mapQ, mapK, mapV;
+    {
+        // Q^ [b, T, H_q, 128]: box = 64 elements x G heads x 128 / G positions
+        uint64_t dims[4] = {128, (uint64_t)d.n_q_heads, (uint64_t)T, (uint64_t)cv.batch};
+        uint64_t str[3] = {128 * 2, (uint64_t)d.n_q_heads * 128 * 2, (uint64_t)T * d.n_q_heads * 128 * 2};
+        uint32_t box[4] = {KC, (uint32_t)ctx->group, (uint32_t)(TILE / ctx->group), 1};
+        if (!lorc_make_tmap_bf16(&mapQ, qhat, 4, dims, str, box)) return cudaErrorInvalidValue;
+        uint64_t kd[3] = {(uint64_t)ctx->n, (uint64_t)rows, (uint64_t)cv.batch};
+        uint64_t ks[2] = {(uint64_t)ctx->n * 2, (uint64_t)rows * ctx->n * 2};
+        uint32_t kb[3] = {KC, TILE, 1};
+        if (!lorc_make_tmap_bf16(&mapK, khat, 3, kd, ks, kb)) return cudaErrorInvalidValue;
+        if (!lorc_make_tmap_bf16(&mapV, vbuf, 3, kd, ks, kb)) return cudaErrorInvalidValue;
+    }
+    FaParams fp;
+    fp.out = out; fp.seq_lens = cv.seq_lens; fp.status = ctx->status_dev;
+    fp.T = T; fp.H_q = d.n_q_heads; fp.G = ctx->group; fp.n_rows = (int)rows; fp.max_pos = d.max_pos;
+    const int qp = TILE / ctx->group;
+    dim3 fgrid((T + qp - 1) / qp, d.n_kv_heads, cv.batch);
+    lorc_prefill_attn_kernel<<<fgrid, F_THREADS, sizeof(FaSmem) + 1024, st>>>(mapQ, mapK, mapV, fp);
+    *launches += 1;
+    return cudaGetLastError();
+}

@@ -142,16 +142,17 @@ def bf16_ulp(x):
     return np.ldexp(1.0, np.maximum(ex - 1, -126) - 7)
 
 
-def assert_rows_close(got, want, tol, tag=None):
+def assert_rows_close(got, want, tol, tag=None, elem_factor=2.0):
     """Both bounds the parity tests use on an output [.., H_q, d_h]: the relative L2 error of every (sequence, head)
     row, and element by element |got - want| <= 2 tol * rms(row) + one bf16 ulp of the expected value.  (The output is
     rounded to bf16 once, which alone is up to half an ulp; the rest of the error is spread over the 64 or 128
     elements of a row with an rms of at most tol * rms(row), so 2 tol * rms(row) leaves a single element some five
-    standard deviations at the measured error level of 3e-3.)"""
+    standard deviations at the measured error level of 3e-3.  Tests with a million elements and a higher error level
+    pass a larger elem_factor.)"""
     got = np.asarray(got, dtype=np.float64)
     want = np.asarray(want, dtype=np.float64)
     err = O.rel_l2_rows(got, want)
     assert err <= tol, (tag, "relative L2 row error", err)
     rms = np.sqrt(np.mean(want ** 2, axis=-1, keepdims=True))
-    excess = np.abs(got - want) - (2.0 * tol * rms + bf16_ulp(want))
+    excess = np.abs(got - want) - (elem_factor * tol * rms + bf16_ulp(want))
     assert np.all(excess <= 0.0), (tag, "element-wise bound exceeded by", float(excess.max()))

@@ -460,3 +460,37 @@ def test_latent_output_times_value_factor_is_the_attention_output():
         assert np.all(o_lat.min(axis=0) >= cv.min(axis=0) - 1e-12) and np.all(o_lat.max(axis=0) <= cv.max(axis=0) + 1e-12)
     one = O.decode_attn_latent_out(ck[:1], cv[:1], Bk, q, H_kv, 10000.0)
     assert np.allclose(one, np.tile(cv[0], (H_q, 1)), atol=1e-14)
+
+
+def test_prefill_attention_is_masked_dense_attention():
+    """prefill_attn_latent against brute force: reconstruct every key and value, rotate, one dense masked softmax per
+    head (query t sees positions <= N - T + t), and against the full-rank uncompressed attention of each prefix."""
+    D, H_q, H_kv, d_h, N, T = 48, 4, 2, 8, 11, 5
+    n = H_kv * d_h
+    Uk, sk, Vk = synth.synth_weight_factors(D, n, 0.8, 6, "k")
+    Uv, sv, Vv = synth.synth_weight_factors(D, n, 0.8, 6, "v")
+    x = synth.hidden_states(N, D, 6).astype(np.float64)
+    q = synth.queries(T, H_q, d_h, 6, 0, 4.0).astype(np.float64)
+    for r in (n, 6):
+        Ak, Bk = O.factors_from_generators(Uk, sk, Vk, r)
+        Av, Bv = O.factors_from_generators(Uv, sv, Vv, r)
+        ck, cv = O.append_latent(x, Ak), O.append_latent(x, Av)
+        got = O.prefill_attn_latent(ck, cv, Bk, Bv, q, H_kv, 10000.0)
+        K = O.rope((ck @ Bk).reshape(N, H_kv, d_h), np.arange(N)[:, None], 10000.0)
+        V = (cv @ Bv).reshape(N, H_kv, d_h)
+        G = H_q // H_kv
+        for t in range(T):
+            pos = N - T + t
+            qh = O.rope(q[t], np.full((H_q,), pos), 10000.0)
+            for h in range(H_q):
+                s = K[:, h // G, :] @ qh[h] / math.sqrt(d_h)
+                s[pos + 1:] = -np.inf                        # causal mask inside the new chunk
+                p = np.exp(s - s.max())
+                want = (p / p.sum()) @ V[:, h // G, :]
+                assert np.allclose(got[t, h], want, atol=1e-12)
+            if r == n:
+                # full rank: the uncompressed model's attention for the prefix that ends at this token
+                W_k, W_v = (Uk * sk) @ Vk.T, (Uv * sv) @ Vv.T
+                assert np.allclose(got[t], O.decode_attn_full(x[:pos + 1], W_k, W_v, q[t], H_kv, 10000.0), atol=1e-10)
+        # the last query is the decode query
+        assert np.allclose(got[-1], O.decode_attn_latent(ck, cv, Bk, Bv, q[-1], H_kv, 10000.0), atol=1e-14)
