@@ -265,7 +265,11 @@ int lorc_append(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* x
     cudaError_t e;
     int path = 1;
     LorcStageTimer timer(ctx, LORC_STAGE_APPEND, st);
-    if (!(ctx->desc.flags & LORC_FLAG_DEBUG_FP32) && lorc_tc_append_supported(ctx, *L, cv, T)) {
+    if (!(ctx->desc.flags & LORC_FLAG_DEBUG_FP32) && lorc_tc_append_gemm_supported(ctx, *L, cv, T)) {
+        // prompt-sized launch: a dense contraction, on tcgen05
+        e = lorc_tc_append_gemm(ctx, *L, cv, (const bf16*)x, T, st, &launches);
+        path = 2;
+    } else if (!(ctx->desc.flags & LORC_FLAG_DEBUG_FP32) && lorc_tc_append_supported(ctx, *L, cv, T)) {
         e = lorc_tc_append(ctx, layer, *L, cv, (const bf16*)x, T, st, &launches);
         path = 2;
     } else {

@@ -18,6 +18,10 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
                            cudaStream_t st, int* launches, bool latent_out = false);
 cudaError_t lorc_tc_append(lorc_ctx* ctx, int layer, const LorcLayer& L, const CacheView& cv,
                            const bf16* x, int T, cudaStream_t st, int* launches);
+// Cache write of compressed layers as a tcgen05 GEMM (tc_append.cu), for launches of at least 128 tokens.
+bool lorc_tc_append_gemm_supported(const lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, int T);
+cudaError_t lorc_tc_append_gemm(lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, const bf16* x, int T,
+                                cudaStream_t st, int* launches);
 
 // Bytes of one probability tile image (128 tokens of one sequence, all query heads): the bf16 numerators as the PV
 // kernel's swizzled MMA operand, then float m[4][H_q] and float l[4][H_q] (reference and sum per 32-token quarter).

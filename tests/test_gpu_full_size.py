@@ -10,8 +10,9 @@ one.  Two kinds of sample:
           are checked against the exactly rounded latents on the way;
   kernel  the oracle reads the cache rows back from the device (bf16 values, exact in fp64) and redoes the attention
           over them: the same check of the attention kernels at a fraction of the cost.
-Every sampled (layer, sequence) is attended with the benchmark's query (scale 8) and again with queries of scale 1
-(near-uniform softmax) and 64 (peaked softmax, where rotation or position errors show).
+Every sampled (layer, sequence) is attended with the benchmark's query (scale 8) and again, on the cache rows the
+device holds, with queries of scale 1 (near-uniform softmax) and 64 (peaked softmax, where rotation or position errors
+show).
 Each test prints the largest error it saw.
 """
 import os
@@ -131,6 +132,8 @@ def test_sampled_outputs_at_full_size(name, layer_ids, chain, kernel):
                 assert np.all(err <= bound), float((err / bound).max())
                 assert np.mean(err > 0) < 0.02          # a different last bit only where fp32 and fp64 sums straddle a tie
                 worst["cache write, error / bound"] = max(worst.get("cache write, error / bound", 0.0), float((err / bound).max()))
+                worst["cache write, fraction of entries off by an ulp"] = max(
+                    worst.get("cache write, fraction of entries off by an ulp", 0.0), float(np.mean(err > 0)))
             rows[s] = (ck, cv)
         for s in kernel_s:
             rows[s] = (_f64(wl.keep[l][0][s, :N]), _f64(wl.keep[l][1][s, :N]))
@@ -142,7 +145,12 @@ def test_sampled_outputs_at_full_size(name, layer_ids, chain, kernel):
             got = _f64(wl.out[l, s])
             helpers.assert_rows_close(got, want, TOL, (name, l, s, 8.0))
             worst[8.0] = max(worst.get(8.0, 0.0), O.rel_l2_rows(got, want))
-        _attend_scales(L, wl, l, rows, fac, shape, sorted(rows), worst)
+        # The other two query scales test the attention kernels, so they run on the rows the device holds (read back;
+        # bf16 values are exact in fp64): a peaked softmax (scale 64) turns a last-bit difference in one large latent
+        # coordinate into a visible change of the output, which is a property of the cache write's rounding, checked
+        # above, not of the attention.
+        held_rows = {s: (_f64(wl.keep[l][0][s, :N]), _f64(wl.keep[l][1][s, :N])) for s in rows}
+        _attend_scales(L, wl, l, held_rows, fac, shape, sorted(rows), worst)
     print(f"\n[full size] {name}: layers {sorted(set(layer_ids[l] for l in by_layer))}, "
           f"{len(chain)} chain + {len(kernel)} kernel samples; max relative L2 row error by query scale "
           + ", ".join(f"{k}: {v:.2e}" for k, v in sorted(worst.items(), key=lambda kv: str(kv[0]))))
