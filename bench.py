@@ -48,6 +48,9 @@ def parse_args():
     ap.add_argument("--no-graph", action="store_true", help="launch call by call instead of replaying a CUDA graph")
     ap.add_argument("--stages", action="store_true",
                     help="call-by-call launches with per-kernel CUDA events; adds a 'stages' object (ms per step)")
+    ap.add_argument("--mode", default="decode", choices=["decode", "prefill"],
+                    help="prefill: time prompt processing (lorc_append + lorc_prefill_attn per chunk and layer) instead of decode steps")
+    ap.add_argument("--chunk", type=int, default=1024, help="--mode prefill: prompt tokens per call")
     ap.add_argument("--rope", default="half", choices=["half", "none"],
                     help="none: layers whose keys take no rotation at attention time (the absorbed score path, HBM-bound)")
     ap.add_argument("--no-full-rank-leg", action="store_true",
@@ -624,6 +627,92 @@ def attention_leg(L, shape, device, peaks, full_rank=False, steps=4, warmup=3, n
         wl.close()
 
 
+def prefill_leg(L, shape, device, peaks, n_layers=None, chunk=1024, reps=2):
+    """Prompt processing of the configuration: for every layer and every chunk of the prompt, lorc_append of the chunk
+    and lorc_prefill_attn of its queries over everything cached so far.  Times the cache writes and the attention
+    calls separately (CUDA events around each group of calls) and reports prompt tokens per second and the fraction of
+    the bf16 tensor peak each reaches on its algorithmic FLOPs:
+      cache write   2 D (r_k + r_v) per token;
+      attention     reconstruction of every cached key and value, 2 (r_k + r_v) n per cached token and call, plus
+                    4 H_q d_h per (query, visible key) pair for Q K^T and P V."""
+    import torch
+    from paper_2410_03111_b200 import host
+    from workloads import device as wdev
+    n_layers = n_layers or shape.n_layers
+    b, N = shape.batch, shape.context
+    n_max = ((N + 127) // 128) * 128
+    ctx = L.lorc_create(n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.d_head, shape.rope_theta,
+                        max_pos=n_max, flags=0)
+    caches, keep = [], []
+    seq_lens = torch.zeros(b, dtype=torch.int32, device=device)
+    ranks = shape.ranks[:n_layers]
+    for l in range(n_layers):
+        r = ranks[l]
+        Uk, sk, Vk = wdev.weight_generators(shape.d_model, shape.n, shape.sigma_p, l, "k", device)
+        Uv, sv, Vv = wdev.weight_generators(shape.d_model, shape.n, shape.sigma_p, l, "v", device)
+        Ak, Bk = host.factors_from_svd(Uk, sk, Vk, r)
+        Av, Bv = host.factors_from_svd(Uv, sv, Vv, r)
+        L.lorc_load_factors(ctx, l, L.LORC_MODE_LATENT, r, r, Ak, Bk, Av, Bv)
+        k = torch.zeros(b, n_max, r, dtype=torch.bfloat16, device=device)
+        v = torch.zeros(b, n_max, r, dtype=torch.bfloat16, device=device)
+        keep.append((k, v))
+        caches.append(L.make_cache(k, v, seq_lens, b, n_max, seq_stride=n_max))
+        del Uk, Vk, Uv, Vv, Ak, Bk, Av, Bv
+    ws = torch.zeros(L.lorc_prefill_workspace_bytes(ctx, b, n_max, chunk), dtype=torch.uint8, device=device)
+    L.lorc_set_workspace(ctx, ws)
+    x = wdev.hidden_states((b, chunk, shape.d_model), 0, 1, device)
+    q = wdev.queries((b, chunk, shape.n_q_heads, shape.d_head), 0, 0, device, 8.0)
+    out = torch.zeros(b, chunk, shape.n_q_heads, shape.d_head, dtype=torch.bfloat16, device=device)
+    chunks = [(c0, min(chunk, N - c0)) for c0 in range(0, N, chunk)]
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    t_app = t_att = 0.0
+    for rep in range(reps + 1):                 # the first pass warms up
+        app_ms = att_ms = 0.0
+        for (c0, T) in chunks:
+            seq_lens.fill_(c0 + T)
+            e0, e1, e2 = ev(), ev(), ev()
+            e0.record()
+            for l in range(n_layers):
+                L.lorc_append(ctx, l, caches[l], x[:, :T].contiguous() if T != chunk else x, T=T)
+            e1.record()
+            for l in range(n_layers):
+                L.lorc_prefill_attn(ctx, l, caches[l], q[:, :T].contiguous() if T != chunk else q,
+                                    out[:, :T].contiguous() if T != chunk else out, T)
+            e2.record()
+            torch.cuda.synchronize()
+            app_ms += e0.elapsed_time(e1)
+            att_ms += e1.elapsed_time(e2)
+        if rep > 0:
+            t_app += app_ms
+            t_att += att_ms
+    t_app /= reps
+    t_att /= reps
+    path = L.lorc_last_path(ctx)
+    rc = L.lorc_sync_status(ctx)
+    if rc:
+        raise RuntimeError(f"device status {rc}: {L.lorc_last_error(ctx)}")
+    n, Hq, dh = shape.n, shape.n_q_heads, shape.d_head
+    f_app = sum(2.0 * shape.d_model * 2 * r for r in ranks) * b * N
+    f_rec = sum(sum(2.0 * 2 * r * n * (c0 + T) for (c0, T) in chunks) for r in ranks) * b
+    pairs = sum(T * c0 + T * (T + 1) / 2.0 for (c0, T) in chunks)
+    f_att = n_layers * 4.0 * Hq * dh * pairs * b
+    L.lorc_destroy(ctx)
+    del keep, caches, ws
+    torch.cuda.empty_cache()
+    res = {
+        "workload": shape.name, "layers": n_layers, "batch": b, "prompt_tokens": N, "chunk": chunk,
+        "kernel_path": {1: "plain fp32 CUDA-core", 2: "tcgen05"}.get(path, str(path)),
+        "append_ms": t_app, "attn_ms": t_att, "prompt_tokens_per_s": b * N / ((t_app + t_att) * 1e-3),
+        "append": {"flops": f_app, "achieved_tflops": f_app / (t_app * 1e-3) / 1e12,
+                   "frac_of_bf16_burst": f_app / (t_app * 1e-3) / 1e12 / peaks["bf16_tflops"]},
+        "attention": {"flops_reconstruction": f_rec, "flops_qk_pv": f_att,
+                      "achieved_tflops": (f_rec + f_att) / (t_att * 1e-3) / 1e12,
+                      "frac_of_bf16_burst": (f_rec + f_att) / (t_att * 1e-3) / 1e12 / peaks["bf16_tflops"]},
+        "timing": "CUDA events around the append calls and around the attention calls of every chunk, all layers",
+    }
+    return res
+
+
 def main():
     args = parse_args()
     from workloads import synth
@@ -652,6 +741,17 @@ def main():
         dist.init_process_group("nccl", device_id=device)
 
     peaks = load_peaks()
+    if args.mode == "prefill":
+        if rank == 0:
+            res = prefill_leg(L, shape, device, peaks, n_layers=n_layers, chunk=args.chunk)
+            print(json.dumps({"metric": "LoRC prompt processing tokens/s (latent KV); % of bf16 tensor peak",
+                              "value": res["prompt_tokens_per_s"], "unit": "tokens/s", "n_gpus": 1, "dtype": "bf16",
+                              "data": "synthetic", "higher_is_better": True, "config": {"workload": shape.name},
+                              "prefill": res}))
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return 0
     flags = L.LORC_FLAG_DEBUG_FP32 if args.debug_fp32 else 0
     if args.stages:
         flags |= L.LORC_FLAG_PROFILE
@@ -760,13 +860,18 @@ def main():
 
     # the uncompressed mode on the same shape, and the other configurations, a few steps each (1-GPU runs only)
     full_leg, others = None, None
-    absorbed_leg = None
+    absorbed_leg = prefill = None
     if rank == 0 and world == 1 and not args.full_rank and not args.debug_fp32 and args.layers == 0 and rope:
         if not args.no_other_configs:
             try:
                 absorbed_leg = attention_leg(L, shape, device, peaks, steps=4, rope=False)
             except Exception as exc:
                 absorbed_leg = {"error": str(exc)[:200]}
+        if not args.no_other_configs:
+            try:
+                prefill = prefill_leg(L, shape, device, peaks, n_layers=min(4, shape.n_layers), chunk=1024, reps=1)
+            except Exception as exc:
+                prefill = {"error": str(exc)[:200]}
         if not args.no_full_rank_leg:
             try:
                 full_leg = attention_leg(L, shape, device, peaks, full_rank=True, steps=4)
@@ -859,6 +964,8 @@ def main():
             line["other_configs"] = others
         if absorbed_leg is not None:
             line["no_rotation"] = absorbed_leg
+        if prefill is not None:
+            line["prefill"] = prefill
         print(json.dumps(line))
     if dist is not None:
         dist.barrier()

@@ -296,3 +296,48 @@ def test_ragged_paged_batch_uncompressed_mode():
     sess.close()
     del k, v
     torch.cuda.empty_cache()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("name,layer_ids,T,picks", [
+    # the last 1024 tokens of the 4096-token prompts as the chunk; ranks 928 and 416
+    ("cfg2_8b_progressive", [0, 31], 1024, [(0, 0), (3, 517), (9, 1023), (15, 64)]),
+    # the last 2048 tokens of the 32768-token prompts; rank 256
+    ("cfg3_8b_long", [0], 2048, [(1, 0), (2, 1031), (3, 2047)]),
+])
+def test_prefill_chunk_at_full_size(name, layer_ids, T, picks):
+    """lorc_prefill_attn on the benchmark's shapes: the last T tokens of every prompt attend to the whole cached
+    prompt; sampled (sequence, query) rows against the oracle's decode attention over the cache rows the device holds,
+    cut after the query's own token."""
+    import torch
+    sys.path.insert(0, ROOT)
+    import bench
+    from workloads import device as wdev
+    L = helpers.lib()
+    shape = synth.CONFIGS[name]
+    device = torch.device("cuda", 0)
+    wl = bench.Workload(L, shape, len(layer_ids), 1, device, 0, layer_ids=layer_ids, seeded_cache=True)
+    N = shape.context
+    ws = torch.zeros(L.lorc_prefill_workspace_bytes(wl.ctx, shape.batch, wl.n_max, T), dtype=torch.uint8, device=device)
+    L.lorc_set_workspace(wl.ctx, ws)
+    worst = 0.0
+    for l, lid in enumerate(layer_ids):
+        r = shape.ranks[lid]
+        fac = _factors(shape, lid, r, device)
+        q = wdev.queries((shape.batch, T, shape.n_q_heads, shape.d_head), lid, 555, device, 8.0)
+        out = torch.zeros(shape.batch, T, shape.n_q_heads, shape.d_head, dtype=torch.bfloat16, device=device)
+        L.lorc_prefill_attn(wl.ctx, l, wl.caches[l], q, out, T)
+        torch.cuda.synchronize()
+        assert L.lorc_sync_status(wl.ctx) == 0, L.lorc_last_error(wl.ctx)
+        assert L.lorc_last_path(wl.ctx) == 2
+        for (s, t) in picks:
+            n_t = N - T + t + 1
+            ck, cv = _f64(wl.keep[l][0][s, :n_t]), _f64(wl.keep[l][1][s, :n_t])
+            want = O.decode_attn_latent(ck, cv, fac["k"][1], fac["v"][1], _f64(q[s, t]), shape.n_kv_heads, shape.rope_theta)
+            got = _f64(out[s, t])
+            helpers.assert_rows_close(got, want, TOL, (name, lid, s, t), elem_factor=4.0)
+            worst = max(worst, O.rel_l2_rows(got, want))
+    print(f"\n[full size] prefill chunk of {T} on {name}, layers {layer_ids}: max relative L2 row error {worst:.2e}")
+    wl.close()
+    del ws
+    torch.cuda.empty_cache()

@@ -71,3 +71,52 @@ def test_static_scratch_entry_rejects_what_cannot_fit():
     assert e.value.code == L.LORC_ERR_WORKSPACE
     assert "LORC_STATIC_SCRATCH_BYTES" in str(e.value)
     sess.close()
+
+
+@pytest.mark.parametrize("variant", ["full_layer", "paged_bf16_path", "splits_lowered_to_fit"])
+def test_static_scratch_entry_other_shapes(variant):
+    """The same comparison for an uncompressed layer with 128-wide heads (the streaming kernel fills the fixed array),
+    for a paged cache on a context without the debug flag, and for a batch whose partial results only fit after the
+    split count has been lowered."""
+    import torch
+    L = H.lib()
+    if variant == "full_layer":
+        D, H_q, H_kv, d_h, r_k, r_v, lens, flags, mode = 256, 8, 2, 128, 256, 256, [150, 33], 0, 1
+    elif variant == "paged_bf16_path":
+        D, H_q, H_kv, d_h, r_k, r_v, lens, flags, mode = 256, 8, 2, 64, 40, 24, [130, 47, 64], 0, 0
+    else:
+        # 94 splits are asked for (one per 32-token tile): 56 sequences x 8 heads x 94 x (2 + 64) x 4 B = 11.1 MiB do not
+        # fit the 8 MiB array, so the entry point lowers the split count until they do
+        D, H_q, H_kv, d_h, r_k, r_v, lens, flags, mode = 128, 8, 2, 64, 16, 64, [3000] * 56, 1, 0
+    prob = H.Problem(D, H_q, H_kv, d_h, r_k, r_v, theta=10000.0, layer=42)
+    b, n_max = len(lens), max(lens) + 8
+    sess = H.Session(prob, max_pos=n_max, batch=b, flags=flags, mode=mode)
+    if mode == 1:
+        held = H.contiguous_cache(sess, b, n_max, [max(lens)] * b)
+        x = np.stack([synth.hidden_states(max(lens), D, 42, chunk=s) for s in range(b)]).astype(np.float64)
+        L.lorc_append(sess.ctx, 0, held[0], H.dev_bf16(x), T=max(lens))
+        held[3][:] = torch.tensor(lens, dtype=torch.int32)
+    else:
+        if len(set(lens)) == 1:
+            one = H.oracle_latents(prob, [synth.hidden_states(lens[0], D, 42).astype(np.float64)])
+            ck, cv = [one[0][0]] * b, [one[1][0]] * b
+        else:
+            ck, cv = H.oracle_latents(prob, [synth.hidden_states(n, D, 42, chunk=s).astype(np.float64) for s, n in enumerate(lens)])
+        if variant == "paged_bf16_path":
+            held = H.paged_cache(sess, b, lens, 16, order_seed=3, k_rows=ck, v_rows=cv)
+        else:
+            held = H.contiguous_cache(sess, b, n_max, lens, ck, cv)
+    q = H.dev_bf16(synth.queries(b, H_q, d_h, 42, 1, 8.0))
+    n_splits = 94 if variant == "splits_lowered_to_fit" else 0
+    if n_splits:
+        assert b * H_q * n_splits * (2 + r_v) * 4 > L.LORC_STATIC_SCRATCH_BYTES
+    for call in range(2):
+        ref = torch.zeros(b, H_q, d_h, dtype=torch.bfloat16, device="cuda")
+        got = torch.full((b, H_q, d_h), 3.0, dtype=torch.bfloat16, device="cuda")
+        L.lorc_decode_attn(sess.ctx, 0, held[0], q, ref, n_splits=n_splits)
+        path_ref = L.lorc_last_path(sess.ctx)
+        L.lorc_decode_attn_static(sess.ctx, 0, held[0], q, got, n_splits=n_splits)
+        assert L.lorc_sync_status(sess.ctx) == 0, L.lorc_last_error(sess.ctx)
+        assert L.lorc_last_path(sess.ctx) == path_ref == (3 if variant == "full_layer" else 1)
+        assert O.rel_l2_rows(H.host_f64(got), H.host_f64(ref)) <= 1e-2
+    sess.close()
