@@ -212,6 +212,25 @@ int lorc_prefill_attn(lorc_ctx* ctx, int layer, const lorc_cache* cache, const v
 int lorc_decode_attn_latent_out(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* q, void* o_lat,
                                 int n_splits, void* stream);
 
+/* Context-sharded decode: one sequence's cache split over several GPUs by position, every GPU attending to its own
+ * shard, and the per-shard results merged.  (The method shards by sequence without any exchange; splitting ONE long
+ * context is the case that needs one, and a small one: d_head + 2 numbers per sequence and head.)
+ *
+ * lorc_decode_attn_shard: like lorc_decode_attn, but the cache of this call holds the tokens of sequence s at positions
+ * pos0[s] .. pos0[s] + seq_lens[s] - 1 (device int32 [batch]) and the query sits at position q_pos[s] (device int32
+ * [batch]; not before the shard's last token, below max_pos).  Results:
+ *   out [batch, n_q_heads, d_head] bf16   the attention output over this shard alone (zeros for an empty shard);
+ *   ml  [batch, n_q_heads, 2] fp32        M, a reference for the scores in log2 units, and L = sum_n 2^(s_n - M).
+ * An empty shard (seq_lens[s] = 0) is not an error here: it reports L = 0.  Compressed (LATENT) layers only.
+ *
+ * lorc_merge_shards: outs [n_shards, batch, n_q_heads, d_head] bf16 and mls [n_shards, batch, n_q_heads, 2] fp32 (the
+ * shards' results, gathered on this GPU, e.g. with an NCCL all-gather) ->
+ *   out = sum_r w_r out_r / sum_r w_r,  w_r = L_r 2^(M_r - max_r M_r),
+ * the softmax over the union of the shards.  n_shards <= 64.  Status EMPTY when no shard held a token. */
+int lorc_decode_attn_shard(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* q, const int32_t* pos0,
+                           const int32_t* q_pos, void* out, float* ml, int n_splits, void* stream);
+int lorc_merge_shards(lorc_ctx* ctx, int n_shards, const void* outs, const float* mls, void* out, int batch, void* stream);
+
 /* Decode attention without any caller-provided or freshly allocated scratch.
  * (The paper has no counterpart to this call; it exists for deployment reasons.)
  * Meant for hosts that cannot allocate device memory when they call in: a server

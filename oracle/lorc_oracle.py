@@ -13,7 +13,7 @@ Notation (row-vector convention, K = X W_k as in the Preliminary section):
   C = X A  the latent ("compressed") cache row, width r = d_c        (Sec. 3.1)
 
 Every function is pinned by tests/test_oracle_pins.py (the schedule functions by
-tests/test_schedule.py) to something the paper or
+tests/test_schedule.py, the context-shard functions by tests/test_sharded.py) to something the paper or
 the mathematics fixes (full-rank identity, Eckart-Young, Theorem 1, RoPE closed
 forms, brute-force attention, a library attention routine).  The numeric
 tolerance used when comparing the GPU to this oracle is not from the paper
@@ -291,6 +291,46 @@ def prefill_attn_latent(c_k: np.ndarray, c_v: np.ndarray, B_k: np.ndarray, B_v: 
         n_t = N - T + t + 1
         out[t] = decode_attn_latent(c_k[:n_t], c_v[:n_t], B_k, B_v, q[t], n_kv_heads, theta, style, use_rope=use_rope)
     return out
+
+
+def shard_log2_sum_exp(c_k: np.ndarray, B_k: np.ndarray, q: np.ndarray, n_kv_heads: int, theta: float,
+                        positions, q_position: int, style: int = ROPE_HALF_SPLIT, use_rope: bool = True) -> np.ndarray:
+    """log2 of sum_n exp(s_n) per query head, over the cached rows given (a shard of one context).
+
+    s_n = q^ . k^_n / sqrt(d_h) are the scores of the Preliminary section's attention with keys reconstructed and
+    rotated at `positions` and the query rotated at q_position.  A softmax over a union of disjoint shards weights
+    each shard's own softmax result by exp of this quantity; that is all a context-sharded decode has to exchange
+    besides the shard outputs.  Returns [H_q] (-inf for an empty shard)."""
+    c_k = np.asarray(c_k, dtype=np.float64)
+    q = np.asarray(q, dtype=np.float64)
+    N = c_k.shape[0]
+    H_q, d = q.shape
+    G = H_q // n_kv_heads
+    if N == 0:
+        return np.full((H_q,), -np.inf)
+    K = (c_k @ np.asarray(B_k, dtype=np.float64)).reshape(N, n_kv_heads, d)
+    if use_rope:
+        K = rope(K, np.asarray(positions)[:, None], theta, style)
+        q = rope(q, np.full((H_q,), q_position), theta, style)
+    out = np.empty((H_q,), dtype=np.float64)
+    for h in range(H_q):
+        s = K[:, h // G, :] @ q[h] / math.sqrt(d)
+        m = np.max(s)
+        out[h] = (m + math.log(np.sum(np.exp(s - m)))) / math.log(2.0)
+    return out
+
+
+def merge_context_shards(outs: np.ndarray, log2_sums: np.ndarray) -> np.ndarray:
+    """Attention over the union of disjoint shards from the shards' own results.
+
+    outs [R, ..., d_h]: each shard's attention output (its own softmax); log2_sums [R, ...]: shard_log2_sum_exp.
+    softmax over the union = sum_r w_r out_r / sum_r w_r with w_r = 2^(log2_sums_r): the denominators of the
+    shards' softmaxes add up to the denominator of the whole.  Shards with -inf (no token) drop out."""
+    outs = np.asarray(outs, dtype=np.float64)
+    ls = np.asarray(log2_sums, dtype=np.float64)
+    top = np.max(ls, axis=0)
+    w = np.where(np.isfinite(ls), np.exp2(ls - np.where(np.isfinite(top), top, 0.0)), 0.0)
+    return np.sum(w[..., None] * outs, axis=0) / np.sum(w, axis=0)[..., None]
 
 
 def decode_attn_full(x: np.ndarray, W_k: np.ndarray, W_v: np.ndarray, q: np.ndarray,

@@ -71,6 +71,8 @@ def _signatures():
         "lorc_decode_attn_latent_out": ([vp, i32, cp, vp, vp, i32, vp], i32),
         "lorc_prefill_workspace_bytes": ([vp, i32, i32, i32], C.c_size_t),
         "lorc_prefill_attn": ([vp, i32, cp, vp, vp, i32, vp], i32),
+        "lorc_decode_attn_shard": ([vp, i32, cp, vp, vp, vp, vp, vp, i32, vp], i32),
+        "lorc_merge_shards": ([vp, i32, vp, vp, vp, i32, vp], i32),
         "lorc_decode_attn_static": ([vp, i32, cp, vp, vp, i32, vp], i32),
         "lorc_decode_step_host": ([vp, i32, cp, vp, vp, vp, i32, vp], i32),
         "lorc_sync_status": ([vp, vp], i32),
@@ -185,6 +187,15 @@ def lorc_prefill_attn(ctx, layer, cache, q, out, T, stream=None):
 def lorc_decode_attn_latent_out(ctx, layer, cache, q, o_lat, n_splits=0, stream=None):
     _check(ctx, _lib.lorc_decode_attn_latent_out(ctx, layer, C.byref(cache), _ptr(q), _ptr(o_lat), n_splits,
                                                   _stream(stream)))
+
+
+def lorc_decode_attn_shard(ctx, layer, cache, q, pos0, q_pos, out, ml, n_splits=0, stream=None):
+    _check(ctx, _lib.lorc_decode_attn_shard(ctx, layer, C.byref(cache), _ptr(q), _ptr(pos0), _ptr(q_pos), _ptr(out),
+                                             _ptr(ml), n_splits, _stream(stream)))
+
+
+def lorc_merge_shards(ctx, n_shards, outs, mls, out, batch, stream=None):
+    _check(ctx, _lib.lorc_merge_shards(ctx, n_shards, _ptr(outs), _ptr(mls), _ptr(out), batch, _stream(stream)))
 
 
 def lorc_decode_attn_static(ctx, layer, cache, q, out, n_splits=0, stream=None):

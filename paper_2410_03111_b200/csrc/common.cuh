@@ -131,12 +131,16 @@ cudaError_t lorc_full_decode(const lorc_ctx* ctx, const CacheView& cv, const bf1
 // at position seq_lens[s] - T + t, attending to the tokens up to its own.
 cudaError_t lorc_generic_decode(const lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv,
                                 const bf16* q, bf16* out, int n_splits, float* part_ml,
-                                float* part_o, cudaStream_t st, int* launches, bool latent_out = false, int T = 1);
+                                float* part_o, cudaStream_t st, int* launches, bool latent_out = false, int T = 1,
+                                const int32_t* pos0 = nullptr, const int32_t* q_pos = nullptr, float* ml_out = nullptr);
+// Merge of the results of context shards (lorc_merge_shards).
+cudaError_t lorc_generic_merge_shards(const lorc_ctx* ctx, int n_shards, const bf16* outs, const float* mls, bf16* out,
+                                      int batch, cudaStream_t st, int* launches);
 // Merge of split partials + value up-projection (also used by the tensor-core path):
 // part_ml [b, H_q, S, 2] (running max in natural-log units, sum), part_o [b, H_q, S, W].
 cudaError_t lorc_generic_combine(const lorc_ctx* ctx, const LorcLayer& L, int batch, int n_splits,
                                  const float* part_ml, const float* part_o, bf16* out,
-                                 cudaStream_t st, int* launches, bool latent_out = false);
+                                 cudaStream_t st, int* launches, bool latent_out = false, float* ml_out = nullptr);
 // token granularity of a split in the plain decode kernel
 #define LORC_GENERIC_TILE 32
 #define LORC_MAX_SPLITS 256

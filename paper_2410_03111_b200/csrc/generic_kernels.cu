@@ -178,7 +178,8 @@ __global__ void __launch_bounds__(128)
 decode_generic_kernel(const bf16* __restrict__ q, CacheView cv, const bf16* __restrict__ B_k, int r_k,
                       int r_v, int n, int G, int n_splits, int rope_style,
                       const float2* __restrict__ rope_table, int max_pos, float* __restrict__ part_ml,
-                      float* __restrict__ part_o, int* status, int T) {
+                      float* __restrict__ part_o, int* status, int T, const int32_t* __restrict__ pos0,
+                      const int32_t* __restrict__ q_pos) {
     constexpr int HALF = DH / 2;
     constexpr int SUB = 128 / DH;            // token subsets when DH < 128
     constexpr int TPS = GEN_TILE / SUB;      // tokens per thread in the reconstruction
@@ -199,6 +200,13 @@ decode_generic_kernel(const bf16* __restrict__ q, CacheView cv, const bf16* __re
     const int W = LATENT ? r_v : DH;         // width of the output accumulator
     int len = cv.seq_lens[s];
     if (T > 1) len = len >= T ? len - (T - 1 - sq % T) : 0;
+    // context shards: the cached rows sit at positions p0 .. p0 + len - 1, the query at qpos (not before the last row)
+    const int p0 = pos0 ? pos0[s] : 0;
+    int qpos_abs = q_pos ? q_pos[s] : p0 + len - 1;
+    if (len > 0 && (p0 < 0 || qpos_abs < p0 + len - 1 || qpos_abs >= max_pos)) {
+        if (threadIdx.x == 0) lorc_set_status(status, LORC_ERR_CAPACITY);
+        len = 0;
+    }
 
     // token range of this split
     int tiles = (len + GEN_TILE - 1) / GEN_TILE;
@@ -216,7 +224,7 @@ decode_generic_kernel(const bf16* __restrict__ q, CacheView cv, const bf16* __re
     // rotated, scaled query of the G heads of this KV head
     if (len > 0 && len <= max_pos) {
         const float scale = rsqrtf((float)DH);
-        const int qpos = len - 1;
+        const int qpos = qpos_abs;
         for (int i = tid; i < G * HALF; i += 128) {
             int h = i / HALF, jj = i - h * HALF;
             int ia = (rope_style == LORC_ROPE_HALF_SPLIT) ? jj : 2 * jj;
@@ -289,7 +297,7 @@ decode_generic_kernel(const bf16* __restrict__ q, CacheView cv, const bf16* __re
                 if (pos >= t_end) continue;
                 int ia = (rope_style == LORC_ROPE_HALF_SPLIT) ? jj : 2 * jj;
                 int ib = (rope_style == LORC_ROPE_HALF_SPLIT) ? jj + HALF : 2 * jj + 1;
-                float2 cs = rope_table[(long long)pos * HALF + jj];
+                float2 cs = rope_table[(long long)(p0 + pos) * HALF + jj];
                 float a = Kt[t][ia], b = Kt[t][ib];
                 Kt[t][ia] = a * cs.x - b * cs.y;
                 Kt[t][ib] = a * cs.y + b * cs.x;
@@ -382,7 +390,7 @@ template <bool LATENT>
 __global__ void __launch_bounds__(128)
 combine_generic_kernel(const float* __restrict__ part_ml, const float* __restrict__ part_o,
                        const bf16* __restrict__ B_v, bf16* __restrict__ out, int W, int n, int DH, int G,
-                       int n_splits, int* status) {
+                       int n_splits, int* status, float* __restrict__ ml_out) {
     extern __shared__ float o_lat[];     // [W]
     __shared__ float w_s[LORC_MAX_SPLITS];
     __shared__ float L_s;
@@ -402,7 +410,13 @@ combine_generic_kernel(const float* __restrict__ part_ml, const float* __restric
             L += (double)w * (double)l;
         }
         L_s = (float)L;
-        if (!(L > 0.0)) lorc_set_status(status, LORC_ERR_EMPTY);
+        if (ml_out) {
+            // reference in log2 units and the denominator relative to it (a shard of a context may be empty)
+            ml_out[((long long)s * H_q + h) * 2] = L > 0.0 ? M * 1.4426950408889634f : 0.f;
+            ml_out[((long long)s * H_q + h) * 2 + 1] = (float)L;
+        } else if (!(L > 0.0)) {
+            lorc_set_status(status, LORC_ERR_EMPTY);
+        }
     }
     __syncthreads();
     const float L = L_s;
@@ -432,7 +446,7 @@ combine_generic_kernel(const float* __restrict__ part_ml, const float* __restric
 
 cudaError_t lorc_generic_combine(const lorc_ctx* ctx, const LorcLayer& L, int batch, int n_splits,
                                  const float* part_ml, const float* part_o, bf16* out,
-                                 cudaStream_t st, int* launches, bool latent_out) {
+                                 cudaStream_t st, int* launches, bool latent_out, float* ml_out) {
     const lorc_model_desc& d = ctx->desc;
     const bool latent = (L.mode == LORC_MODE_LATENT);
     const int W = latent ? L.r_v : d.d_head;
@@ -442,22 +456,23 @@ cudaError_t lorc_generic_combine(const lorc_ctx* ctx, const LorcLayer& L, int ba
     if (latent && latent_out)
         // merge only: the normalised latent output [b, H_q, r_v] is the result (rows of width W instead of d_head)
         combine_generic_kernel<false><<<cgrid, 128, smem, st>>>(part_ml, part_o, nullptr, out, W, ctx->n, W, ctx->group,
-                                                               n_splits, ctx->status_dev);
+                                                               n_splits, ctx->status_dev, ml_out);
     else if (latent)
         combine_generic_kernel<true><<<cgrid, 128, smem, st>>>(part_ml, part_o, L.B_v, out, W, ctx->n,
                                                               d.d_head, ctx->group, n_splits,
-                                                              ctx->status_dev);
+                                                              ctx->status_dev, ml_out);
     else
         combine_generic_kernel<false><<<cgrid, 128, smem, st>>>(part_ml, part_o, nullptr, out, W, ctx->n,
                                                                d.d_head, ctx->group, n_splits,
-                                                               ctx->status_dev);
+                                                               ctx->status_dev, ml_out);
     *launches += 1;
     return cudaGetLastError();
 }
 
 cudaError_t lorc_generic_decode(const lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv,
                                 const bf16* q, bf16* out, int n_splits, float* part_ml,
-                                float* part_o, cudaStream_t st, int* launches, bool latent_out, int T) {
+                                float* part_o, cudaStream_t st, int* launches, bool latent_out, int T,
+                                const int32_t* pos0, const int32_t* q_pos, float* ml_out) {
     const lorc_model_desc& d = ctx->desc;
     const int G = ctx->group;
     const bool latent = (L.mode == LORC_MODE_LATENT);
@@ -469,14 +484,14 @@ cudaError_t lorc_generic_decode(const lorc_ctx* ctx, const LorcLayer& L, const C
             cudaError_t e = lorc_full_decode(ctx, cv, q, n_splits, part_ml, part_o, st, launches);
             if (e != cudaSuccess) return e;
         }
-        return lorc_generic_combine(ctx, L, cv.batch, n_splits, part_ml, part_o, out, st, launches, false);
+        return lorc_generic_combine(ctx, L, cv.batch, n_splits, part_ml, part_o, out, st, launches, false, nullptr);
     }
     {
     LorcStageTimer timer(ctx, LORC_STAGE_SCORE, st);
 #define LAUNCH_DEC(DHV, LAT)                                                                      \
     decode_generic_kernel<DHV, LAT><<<grid, 128, 0, st>>>(                                        \
         q, cv, L.B_k, L.r_k, L.r_v, ctx->n, G, n_splits, ctx->pair_style, ctx->rope_table, d.max_pos, \
-        part_ml, part_o, ctx->status_dev, T)
+        part_ml, part_o, ctx->status_dev, T, pos0, q_pos)
     if (d.d_head == 128) {
         if (latent) LAUNCH_DEC(128, true); else LAUNCH_DEC(128, false);
     } else {
@@ -487,5 +502,44 @@ cudaError_t lorc_generic_decode(const lorc_ctx* ctx, const LorcLayer& L, const C
     *launches += 1;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    return lorc_generic_combine(ctx, L, cv.batch * T, n_splits, part_ml, part_o, out, st, launches, latent_out);
+    return lorc_generic_combine(ctx, L, cv.batch * T, n_splits, part_ml, part_o, out, st, launches, latent_out, ml_out);
+}
+
+// ---------------------------------------------------------------------------
+// Merge of context shards: out = sum_r w_r out_r / sum_r w_r,  w_r = L_r 2^(M_r - M),  M = max_r M_r.
+// ---------------------------------------------------------------------------
+__global__ void merge_shards_kernel(const bf16* __restrict__ outs, const float* __restrict__ mls, bf16* __restrict__ out,
+                                    int n_shards, long long rows, int DH, int* status) {
+    const long long row = blockIdx.x;                    // (sequence, head)
+    __shared__ float w_s[64];
+    __shared__ float inv_s;
+    if (threadIdx.x == 0) {
+        float M = -INFINITY;
+        for (int r = 0; r < n_shards; ++r)
+            if (mls[((long long)r * rows + row) * 2 + 1] > 0.f) M = fmaxf(M, mls[((long long)r * rows + row) * 2]);
+        float tot = 0.f;
+        for (int r = 0; r < n_shards; ++r) {
+            const float l = mls[((long long)r * rows + row) * 2 + 1];
+            const float w = l > 0.f ? l * exp2f(mls[((long long)r * rows + row) * 2] - M) : 0.f;
+            w_s[r] = w;
+            tot += w;
+        }
+        inv_s = tot > 0.f ? 1.f / tot : 0.f;
+        if (!(tot > 0.f)) lorc_set_status(status, LORC_ERR_EMPTY);
+    }
+    __syncthreads();
+    for (int j = threadIdx.x; j < DH; j += blockDim.x) {
+        float a = 0.f;
+        for (int r = 0; r < n_shards; ++r)
+            if (w_s[r] != 0.f) a = fmaf(w_s[r], __bfloat162float(outs[((long long)r * rows + row) * DH + j]), a);
+        out[row * DH + j] = __float2bfloat16_rn(a * inv_s);
+    }
+}
+
+cudaError_t lorc_generic_merge_shards(const lorc_ctx* ctx, int n_shards, const bf16* outs, const float* mls, bf16* out,
+                                      int batch, cudaStream_t st, int* launches) {
+    const long long rows = (long long)batch * ctx->desc.n_q_heads;
+    merge_shards_kernel<<<(unsigned)rows, 128, 0, st>>>(outs, mls, out, n_shards, rows, ctx->desc.d_head, ctx->status_dev);
+    *launches += 1;
+    return cudaGetLastError();
 }

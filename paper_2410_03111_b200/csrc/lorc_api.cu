@@ -282,7 +282,8 @@ int lorc_append(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* x
 }
 
 static int decode_attn_impl(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* q, void* out,
-                            int n_splits, void* stream, bool latent_out) {
+                            int n_splits, void* stream, bool latent_out, const int32_t* pos0 = nullptr,
+                            const int32_t* q_pos = nullptr, float* ml_out = nullptr) {
     LorcLayer* L;
     int rc = get_layer(ctx, layer, &L);
     if (rc) return rc;
@@ -292,6 +293,8 @@ static int decode_attn_impl(lorc_ctx* ctx, int layer, const lorc_cache* cache, c
     if (n_splits < 0) return fail(ctx, LORC_ERR_ARG, "decode_attn: negative n_splits");
     if (latent_out && L->mode != LORC_MODE_LATENT)
         return fail(ctx, LORC_ERR_UNSUPPORTED, "decode_attn_latent_out: the layer is not compressed");
+    if (q_pos && L->mode != LORC_MODE_LATENT)
+        return fail(ctx, LORC_ERR_UNSUPPORTED, "decode_attn_shard: the layer is not compressed");
     CacheView cv;
     rc = check_cache(ctx, cache, *L, &cv);
     if (rc) return rc;
@@ -306,7 +309,7 @@ static int decode_attn_impl(lorc_ctx* ctx, int layer, const lorc_cache* cache, c
         size_t tc = lorc_tc_workspace_bytes(ctx, cv.batch, cv.max_seq_len);
         if (tc > ctx->ws_bytes) return fail(ctx, LORC_ERR_WORKSPACE, "decode_attn: workspace too small");
         e = lorc_tc_decode(ctx, layer, *L, cv, (const bf16*)q, (bf16*)out, n_splits, ctx->ws,
-                           ctx->ws_bytes, st, &launches, latent_out);
+                           ctx->ws_bytes, st, &launches, latent_out, pos0, q_pos, ml_out);
         ctx->launches += launches;
         ctx->last_path = 2;
         if (e != cudaSuccess) return fail_cuda(ctx, e, "lorc_decode_attn (tensor-core path)");
@@ -323,7 +326,8 @@ static int decode_attn_impl(lorc_ctx* ctx, int layer, const lorc_cache* cache, c
     if (w.total > ctx->ws_bytes) return fail(ctx, LORC_ERR_WORKSPACE, "decode_attn: workspace too small");
     float* part_ml = (float*)((char*)ctx->ws + w.off_ml);
     float* part_o = (float*)((char*)ctx->ws + w.off_o);
-    e = lorc_generic_decode(ctx, *L, cv, (const bf16*)q, (bf16*)out, S, part_ml, part_o, st, &launches, latent_out);
+    e = lorc_generic_decode(ctx, *L, cv, (const bf16*)q, (bf16*)out, S, part_ml, part_o, st, &launches, latent_out, 1,
+                            pos0, q_pos, ml_out);
     ctx->launches += launches;
     ctx->last_path = lorc_full_decode_supported(ctx, *L) ? 3 : 1;
     if (e != cudaSuccess) return fail_cuda(ctx, e, "lorc_decode_attn");
@@ -338,6 +342,25 @@ int lorc_decode_attn(lorc_ctx* ctx, int layer, const lorc_cache* cache, const vo
 int lorc_decode_attn_latent_out(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* q, void* o_lat,
                                 int n_splits, void* stream) {
     return decode_attn_impl(ctx, layer, cache, q, o_lat, n_splits, stream, true);
+}
+
+int lorc_decode_attn_shard(lorc_ctx* ctx, int layer, const lorc_cache* cache, const void* q, const int32_t* pos0,
+                           const int32_t* q_pos, void* out, float* ml, int n_splits, void* stream) {
+    if (!ctx) return LORC_ERR_ARG;
+    if (!pos0 || !q_pos || !ml) return fail(ctx, LORC_ERR_ARG, "decode_attn_shard: null pos0, q_pos or ml");
+    return decode_attn_impl(ctx, layer, cache, q, out, n_splits, stream, false, pos0, q_pos, ml);
+}
+
+int lorc_merge_shards(lorc_ctx* ctx, int n_shards, const void* outs, const float* mls, void* out, int batch, void* stream) {
+    if (!ctx) return LORC_ERR_ARG;
+    if (!outs || !mls || !out || batch <= 0 || n_shards <= 0 || n_shards > 64)
+        return fail(ctx, LORC_ERR_ARG, "merge_shards: null pointer, or batch / n_shards out of range (1..64 shards)");
+    int launches = 0;
+    cudaError_t e = lorc_generic_merge_shards(ctx, n_shards, (const bf16*)outs, mls, (bf16*)out, batch, (cudaStream_t)stream,
+                                              &launches);
+    ctx->launches += launches;
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "lorc_merge_shards");
+    return LORC_OK;
 }
 
 size_t lorc_prefill_workspace_bytes(const lorc_ctx* ctx, int batch, int max_seq_len, int T) {

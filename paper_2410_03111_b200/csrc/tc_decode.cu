@@ -157,7 +157,7 @@ static cudaError_t tc_prepare(lorc_ctx* ctx, LorcTcState* T, LorcTcLayer& TL, co
 
 cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const CacheView& cv, const bf16* q,
                            bf16* out, int n_splits, void* ws, size_t ws_bytes, cudaStream_t st, int* launches,
-                           bool latent_out) {
+                           bool latent_out, const int32_t* pos0, const int32_t* q_pos, float* ml_out) {
     LorcTcState* T = tc_state(ctx);
     LorcTcLayer& TL = T->layers[layer];
     const lorc_model_desc& d = ctx->desc;
@@ -203,12 +203,12 @@ cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const C
                                               cv.batch * plan.n_blk, st, launches);
         else
             e = lorc_tc_score_launch(ctx, L, cv, TL.mapCK, TL.mapBKT, q, pimg, T->rowmax,
-                                     reinterpret_cast<const float4*>(T->rope_tile), tiles, zero, cv.batch * plan.n_blk, st,
-                                     launches);
+                                     reinterpret_cast<const float4*>(T->rope_tile), tiles, zero, cv.batch * plan.n_blk, pos0,
+                                     q_pos, st, launches);
         if (e != cudaSuccess) return e;
     }
     const cudaError_t e2 = lorc_tc_pv_launch(ctx, L, cv, TL.mapCV, TL.mapBVT, pimg, T->rowmax, tiles, plan, pv_scratch,
-                                             out, latent_out, st, launches);
+                                             out, latent_out, ml_out, st, launches);
     if (e2 == cudaSuccess) T->rowmax_dirty = false;
     return e2;
 }

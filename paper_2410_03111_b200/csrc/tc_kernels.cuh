@@ -13,9 +13,12 @@ bool lorc_tc_append_supported(const lorc_ctx* ctx, const LorcLayer& L, const Cac
 size_t lorc_tc_workspace_bytes(const lorc_ctx* ctx, int batch, int max_seq_len);
 
 // latent_out: `out` receives the normalised latent output [b, H_q, r_v] instead of the up-projected one.
+// pos0, q_pos / ml_out: context shards (see lorc_decode_attn_shard): per sequence the position of the first cached row
+// and of the query, and where to leave (reference, denominator) [b, H_q, 2] of the softmax over this shard.
 cudaError_t lorc_tc_decode(lorc_ctx* ctx, int layer, const LorcLayer& L, const CacheView& cv,
                            const bf16* q, bf16* out, int n_splits, void* ws, size_t ws_bytes,
-                           cudaStream_t st, int* launches, bool latent_out = false);
+                           cudaStream_t st, int* launches, bool latent_out = false, const int32_t* pos0 = nullptr,
+                           const int32_t* q_pos = nullptr, float* ml_out = nullptr);
 cudaError_t lorc_tc_append(lorc_ctx* ctx, int layer, const LorcLayer& L, const CacheView& cv,
                            const bf16* x, int T, cudaStream_t st, int* launches);
 // Cache write of compressed layers as a tcgen05 GEMM (tc_append.cu), for launches of at least 128 tokens.
@@ -30,13 +33,13 @@ __host__ __device__ inline int lorc_tc_image_bytes(int n_q_heads) { return 2 * n
 // Score kernel (tc_score.cu): key reconstruction, rotation, q.k and the softmax numerators; writes one tile image per
 // 128 tokens into pimg [b, tiles, image] and raises the row maxima (integers, as order-preserving keys).  rope_tile:
 // the in-tile rotation table (33 x 32 float4, lorc_tc_rope_tile_fill).  Its first block clears zero[0 .. n_zero).
-#define LORC_SCORE_MAX_BATCH 128     // sequences per launch (larger batches take several launches)
+#define LORC_SCORE_MAX_BATCH 64      // sequences per launch (larger batches take several launches)
 cudaError_t lorc_tc_score_set_attrs();
 cudaError_t lorc_tc_rope_tile_fill(float2* table, double theta, cudaStream_t st);
 cudaError_t lorc_tc_score_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, const CUtensorMap& mapCK,
                                  const CUtensorMap& mapBKT, const bf16* q, uint8_t* pimg, unsigned* rowmax,
-                                 const float4* rope_tile, int tiles, int* zero, int n_zero, cudaStream_t st,
-                                 int* launches);
+                                 const float4* rope_tile, int tiles, int* zero, int n_zero, const int32_t* pos0,
+                                 const int32_t* q_pos, cudaStream_t st, int* launches);
 
 // Score kernel of layers without rotation (tc_absorbed.cu): the key up-projection is absorbed into the query
 // (q~ = B_K q, written to `qabs`, lorc_tc_absorbed_scratch_bytes of scratch), the scores are a skinny GEMM over the
@@ -62,8 +65,8 @@ void lorc_tc_pv_plan(const lorc_ctx* ctx, const LorcLayer& L, const CacheView& c
                      LorcPvPlan* plan);
 cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, const CUtensorMap& mapCV,
                               const CUtensorMap& mapBVT, const uint8_t* pimg, unsigned* rowmax, int tiles,
-                              const LorcPvPlan& plan, void* scratch, bf16* out, bool latent_out, cudaStream_t st,
-                              int* launches);
+                              const LorcPvPlan& plan, void* scratch, bf16* out, bool latent_out, float* ml_out,
+                              cudaStream_t st, int* launches);
 
 // Prompt processing (tc_prefill.cu): attention of the T newest tokens of every sequence (q, out [b, T, H_q, 128]) over
 // the latent cache, causal inside the chunk.  Keys and values are reconstructed once into `scratch`

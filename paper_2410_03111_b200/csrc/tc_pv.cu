@@ -58,6 +58,7 @@ struct Pv2Params {
     unsigned* rowmax;              // [b, H_q]   row maxima of the softmax (order-preserving keys of integers)
     bf16* o_norm;                  // [b, H_q, r_pad]      normalised latent output
     int* done;                     // [b, n_blk]           context shares of a column block that have finished (zero on entry)
+    float* ml_out;                 // NULL, or [b, H_q, 2]: reference M (log2 units) and denominator sum_n 2^(s_n - M)
     const int32_t* seq_lens;
     const int32_t* page_table;
     int* status;
@@ -280,7 +281,11 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
         if (p.n_csplit == 1) {
             if (t < HQ) {
                 sm.l_inv[t] = l_share > 0.f ? 1.f / l_share : 0.f;
-                if (!(l_share > 0.f) && blk == 0) lorc_set_status(p.status, LORC_ERR_EMPTY);
+                if (!(l_share > 0.f) && blk == 0 && !p.ml_out) lorc_set_status(p.status, LORC_ERR_EMPTY);
+                if (p.ml_out && blk == 0) {
+                    p.ml_out[((long long)s * p.H_q + t) * 2] = sm.m_row[t];
+                    p.ml_out[((long long)s * p.H_q + t) * 2 + 1] = l_share;
+                }
             }
             __syncwarp();
             asm volatile("bar.sync 2, 128;" ::: "memory");
@@ -373,7 +378,11 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
                 }
                 if (t < HQ) {
                     sm.l_inv[t] = l_share > 0.f ? 1.f / l_share : 0.f;
-                    if (!(l_share > 0.f) && blk == 0) lorc_set_status(p.status, LORC_ERR_EMPTY);
+                    if (!(l_share > 0.f) && blk == 0 && !p.ml_out) lorc_set_status(p.status, LORC_ERR_EMPTY);
+                    if (p.ml_out && blk == 0) {
+                        p.ml_out[((long long)s * p.H_q + t) * 2] = sm.m_row[t];
+                        p.ml_out[((long long)s * p.H_q + t) * 2 + 1] = l_share;
+                    }
                 }
                 __syncwarp();
                 asm volatile("bar.sync 2, 128;" ::: "memory");
@@ -635,8 +644,8 @@ void lorc_tc_pv_plan(const lorc_ctx* ctx, const LorcLayer& L, const CacheView& c
 // score kernel clears it).
 cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, const CUtensorMap& mapCV,
                               const CUtensorMap& mapBVT, const uint8_t* pimg, unsigned* rowmax, int tiles,
-                              const LorcPvPlan& plan, void* scratch, bf16* out, bool latent_out, cudaStream_t st,
-                              int* launches) {
+                              const LorcPvPlan& plan, void* scratch, bf16* out, bool latent_out, float* ml_out,
+                              cudaStream_t st, int* launches) {
     const lorc_model_desc& d = ctx->desc;
     const int n_blk = plan.n_blk, n_csplit = plan.n_csplit;
     const int r_pad = n_blk * 128;
@@ -647,7 +656,7 @@ cudaError_t lorc_tc_pv_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView
     {
         LorcStageTimer timer(ctx, LORC_STAGE_PV, st);
         Pv2Params p;
-        p.pimg = pimg; p.o_part = o_part; p.rowmax = rowmax; p.o_norm = o_norm; p.done = done;
+        p.pimg = pimg; p.o_part = o_part; p.rowmax = rowmax; p.o_norm = o_norm; p.done = done; p.ml_out = ml_out;
         p.seq_lens = cv.seq_lens; p.page_table = cv.page_table; p.status = ctx->status_dev;
         p.batch = cv.batch; p.H_q = d.n_q_heads; p.n_kv = d.n_kv_heads; p.r_v = L.r_v; p.tiles = tiles;
         p.n_blk = n_blk; p.n_csplit = n_csplit; p.max_pos = d.max_pos;

@@ -43,6 +43,7 @@ struct ScoreSmem {
     uint32_t tmem_base;
     int32_t tile_start[LORC_SCORE_MAX_BATCH + 1];   // first flat tile of every sequence
     int32_t lens[LORC_SCORE_MAX_BATCH];             // checked sequence lengths (0: nothing to do)
+    int32_t qrel[LORC_SCORE_MAX_BATCH];             // query position relative to the first cached row
 };
 
 struct ScoreParams {
@@ -50,6 +51,8 @@ struct ScoreParams {
     uint8_t* pimg;                 // [b, tiles, image]      probability tile images, see lorc_tc_image_bytes
     unsigned* rowmax;              // [b, H_q]  running row maximum (an integer, as an order-preserving key; 0: none yet)
     const int32_t* seq_lens;
+    const int32_t* pos0;           // NULL, or per sequence the position of the first cached row and the position of the
+    const int32_t* q_pos;          // query (context shards: the rows of this cache start at some later position than 0)
     const int32_t* page_table;     // NULL: contiguous
     const float2* rope_table;      // [max_pos][64]
     const float4* rope_tile;       // [33][32]   in-tile rotation table in its shared-memory layout
@@ -151,7 +154,14 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
             lorc_set_status(p.status, LORC_ERR_CAPACITY);
             len = 0;
         }
+        int qr = p.q_pos ? p.q_pos[i] - p.pos0[i] : len - 1;
+        if (qr < len - 1 || qr >= p.max_pos || (p.q_pos && (p.pos0[i] < 0 || p.q_pos[i] >= p.max_pos))) {
+            // the query may not precede a cached key, nor leave the tables
+            lorc_set_status(p.status, LORC_ERR_CAPACITY);
+            len = 0;
+        }
         sm.lens[i] = len > 0 ? len : 0;
+        sm.qrel[i] = qr;
     }
     if (warp == 1) {
         tmem_alloc_pair(&sm.tmem_base, 512);
@@ -283,7 +293,7 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
             Unit un;
             decode_unit(sm, w, rank, n_flat, p.batch, un);
             const int buf = uc & 1;
-            const int delta = max(un.len - 1 - un.tile * TILE, 0);
+            const int delta = max(sm.qrel[un.s] - un.tile * TILE, 0);
             const float4 cs = __ldg(reinterpret_cast<const float4*>(p.rope_table + (long long)delta * 64) + lane);
             uint32_t qa[2 * G], qb[2 * G];
 #pragma unroll
@@ -510,8 +520,8 @@ cudaError_t lorc_tc_rope_tile_fill(float2* table, double theta, cudaStream_t st)
 // shared memory).  The first launch clears `zero[0 .. n_zero)` for the kernels that follow it in the stream.
 cudaError_t lorc_tc_score_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheView& cv, const CUtensorMap& mapCK,
                                  const CUtensorMap& mapBKT, const bf16* q, uint8_t* pimg, unsigned* rowmax,
-                                 const float4* rope_tile, int tiles, int* zero, int n_zero, cudaStream_t st,
-                                 int* launches) {
+                                 const float4* rope_tile, int tiles, int* zero, int n_zero, const int32_t* pos0,
+                                 const int32_t* q_pos, cudaStream_t st, int* launches) {
     const lorc_model_desc& d = ctx->desc;
     const size_t img_bytes = (size_t)lorc_tc_image_bytes(d.n_q_heads);
     for (int s0 = 0; s0 < cv.batch; s0 += LORC_SCORE_MAX_BATCH) {
@@ -521,6 +531,8 @@ cudaError_t lorc_tc_score_launch(lorc_ctx* ctx, const LorcLayer& L, const CacheV
         sp.pimg = pimg + (size_t)s0 * tiles * img_bytes;
         sp.rowmax = rowmax + (size_t)s0 * d.n_q_heads;
         sp.seq_lens = cv.seq_lens + s0;
+        sp.pos0 = pos0 ? pos0 + s0 : nullptr;
+        sp.q_pos = q_pos ? q_pos + s0 : nullptr;
         sp.page_table = cv.page_table;
         sp.rope_table = ctx->rope_table;
         sp.rope_tile = rope_tile;
