@@ -12,11 +12,12 @@
 //                       N = 128), rotation in the epilogue (thread = token row), 16-bit rows to the buffer: keys as
 //                       fp16 (the scores are then exact to 2^-11 of |q| |k|, four times closer than with bf16 keys;
 //                       a rotated key element must stay below 65504 in magnitude), values as bf16
-//   attention kernel    one CTA per (128 query rows = 128 / G positions x G heads of one KV head): for every 128-key
-//                       tile   S = Q^ K^^T (tcgen05, fp32 in TMEM)  ->  online softmax, thread = query row; the
-//                       probabilities go back into tensor memory as bf16 over the scores  ->  O += P V with P read from
-//                       tensor memory.  The running reference of a row is only raised when a tile exceeds it by more
-//                       than 2^8 (the accumulator is rescaled then), so most tiles need no pass over O.
+//   attention kernel    one CTA per two blocks of 128 query rows (128 / G positions x G heads of one KV head each): for
+//                       every 128-key tile and block   S = Q^ K^^T (tcgen05, fp32 in TMEM)  ->  online softmax, thread =
+//                       query row; the probabilities go back into tensor memory as bf16 over the scores  ->  O += P V
+//                       with P read from tensor memory.  The two blocks alternate, so the tensor pipe works on one
+//                       while the other's softmax runs.  The running reference of a row is only raised when a tile
+//                       exceeds it by more than 2^8 (the accumulator is rescaled then), so most tiles need no pass over O.
 #include <cuda_fp16.h>
 #include <math.h>
 
@@ -212,15 +213,20 @@ lorc_reconstruct_kernel(const __grid_constant__ CUtensorMap mapC, const __grid_c
 // ------------------------------------------------------------------------------------------------
 // attention over the reconstructed keys and values
 // ------------------------------------------------------------------------------------------------
-constexpr int F_THREADS = 192;       // warp 0 TMA, warp 1 MMA, warps 2..5 softmax (thread = query row)
+// A CTA owns TWO blocks of 128 query rows (block b: 128 / G positions x the G heads of one KV head) and walks the key
+// tiles once for both.  The blocks alternate on the tensor pipe: while the softmax warps of one block turn its scores
+// into probabilities, the pipe multiplies the other block's probabilities into its output and computes its next
+// scores.  Tensor memory: scores / probabilities of block b at column 128 b, its output at column 256 + 128 b.
+constexpr int F_THREADS = 320;       // warp 0 TMA, warp 1 MMA, warps 2..5 softmax of block 0, warps 6..9 of block 1
 constexpr int F_STAGES = 2;
 constexpr float F_RAISE = 8.f;       // a row's reference is raised only when a tile exceeds it by more than this (log2 units)
 
 struct FaSmem {
-    bf16 Q[2][TILE * KC];                 // query rows [128][two 64-element halves]
+    bf16 Q[2][2][TILE * KC];              // [block][64-element half][128 rows]
     bf16 K[F_STAGES][2][TILE * KC];       // key tile [128 keys][two halves]
     bf16 V[F_STAGES][2][TILE * KC];       // value tile [128 keys][two halves]
-    uint64_t q_full, k_full[F_STAGES], v_full[F_STAGES], kv_empty[F_STAGES], s_full, p_ready, o_done;
+    uint64_t q_full, k_full[F_STAGES], v_full[F_STAGES], k_empty[F_STAGES], v_empty[F_STAGES];
+    uint64_t s_full[2], p_ready[2], o_done;
     uint32_t tmem_base;
 };
 
@@ -231,6 +237,12 @@ struct FaParams {
     int T, H_q, G, n_rows, max_pos;
 };
 
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 __global__ void __launch_bounds__(F_THREADS, 1)
 lorc_prefill_attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                          const __grid_constant__ CUtensorMap mapV, const FaParams p) {
@@ -238,8 +250,9 @@ lorc_prefill_attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_
     FaSmem& sm = *reinterpret_cast<FaSmem*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
     const int g = blockIdx.y, s = blockIdx.z;
-    const int qp = TILE / p.G;                                // query positions per block
-    const int t0 = blockIdx.x * qp;                           // first position (inside the chunk) of this block
+    const int qp = TILE / p.G;                                // query positions per block of 128 rows
+    // the CTAs with the latest positions see the most keys: they go first
+    const int t0 = ((int)gridDim.x - 1 - (int)blockIdx.x) * 2 * qp;   // first position (inside the chunk) of this CTA
     int len = p.seq_lens[s];
     if (len > p.max_pos || len > p.n_rows) {
         if (tid == 0) lorc_set_status(p.status, LORC_ERR_CAPACITY);
@@ -249,7 +262,7 @@ lorc_prefill_attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_
         if (tid == 0 && len > 0) lorc_set_status(p.status, LORC_ERR_ARG);
         len = 0;
     }
-    const int t_last = min(p.T, t0 + qp) - 1;                 // last query position of the block
+    const int t_last = min(p.T, t0 + 2 * qp) - 1;             // last query position of the CTA
     const int n_tiles = len > 0 ? (len - p.T + t_last) / TILE + 1 : 0;
 
     if (tid == 0) {
@@ -257,10 +270,13 @@ lorc_prefill_attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_
         for (int i = 0; i < F_STAGES; ++i) {
             mbar_init(&sm.k_full[i], 1);
             mbar_init(&sm.v_full[i], 1);
-            mbar_init(&sm.kv_empty[i], 1);
+            mbar_init(&sm.k_empty[i], 1);
+            mbar_init(&sm.v_empty[i], 1);
         }
-        mbar_init(&sm.s_full, 1);
-        mbar_init(&sm.p_ready, 4);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&sm.s_full[i], 1);
+            mbar_init(&sm.p_ready[i], 4);
+        }
         mbar_init(&sm.o_done, 1);
         fence_barrier_init();
         prefetch_tensormap(&mapQ);
@@ -268,32 +284,39 @@ lorc_prefill_attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_
         prefetch_tensormap(&mapV);
     }
     if (warp == 1) {
-        tmem_alloc(&sm.tmem_base, 256);
+        tmem_alloc(&sm.tmem_base, 512);
         tmem_relinquish();
     }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    const uint32_t tmem = sm.tmem_base;                       // scores / probabilities at column 0, output at column 128
+    const uint32_t tmem = sm.tmem_base;
     bool ok = true;
 
     if (warp == 0) {
         if (n_tiles > 0) {
             if (elect_one()) {
-                // rows of the block: (position t0 + tt, head i of the KV head) -> row tt * G + i; positions past the chunk
-                // read as zero
-                mbar_arrive_expect_tx(&sm.q_full, 2 * TILE * KC * 2);
-                tma_load_4d(sm.Q[0], &mapQ, &sm.q_full, 0, g * p.G, t0, s);
-                tma_load_4d(sm.Q[1], &mapQ, &sm.q_full, 64, g * p.G, t0, s);
+                // rows of a block: (position, head i of the KV head) -> row (position - first) * G + i; positions past the
+                // chunk read as zero
+                mbar_arrive_expect_tx(&sm.q_full, 4 * TILE * KC * 2);
+                for (int b = 0; b < 2; ++b) {
+                    tma_load_4d(sm.Q[b][0], &mapQ, &sm.q_full, 0, g * p.G, t0 + b * qp, s);
+                    tma_load_4d(sm.Q[b][1], &mapQ, &sm.q_full, 64, g * p.G, t0 + b * qp, s);
+                }
             }
             __syncwarp();
             for (int j = 0; j < n_tiles && ok; ++j) {
                 const int st = j % F_STAGES;
-                if (!mbar_wait(&sm.kv_empty[st], ((j / F_STAGES) & 1) ^ 1)) { ok = false; break; }
+                const uint32_t par = ((j / F_STAGES) & 1) ^ 1;
+                if (!mbar_wait(&sm.k_empty[st], par)) { ok = false; break; }
                 if (elect_one()) {
                     mbar_arrive_expect_tx(&sm.k_full[st], 2 * TILE * KC * 2);
                     tma_load_3d(sm.K[st][0], &mapK, &sm.k_full[st], g * 128, j * TILE, s);
                     tma_load_3d(sm.K[st][1], &mapK, &sm.k_full[st], g * 128 + 64, j * TILE, s);
+                }
+                __syncwarp();
+                if (!mbar_wait(&sm.v_empty[st], par)) { ok = false; break; }
+                if (elect_one()) {
                     mbar_arrive_expect_tx(&sm.v_full[st], 2 * TILE * KC * 2);
                     tma_load_3d(sm.V[st][0], &mapV, &sm.v_full[st], g * 128, j * TILE, s);
                     tma_load_3d(sm.V[st][1], &mapV, &sm.v_full[st], g * 128 + 64, j * TILE, s);
@@ -306,103 +329,139 @@ lorc_prefill_attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_
         if (n_tiles > 0) {
             const uint32_t idesc_s = make_idesc_f16(128, 128);            // S = Q K^T: fp16 operands, both K-major
             const uint32_t idesc_o = make_idesc_bf16(128, 128, 0, 1);     // O += P V: V is MN-major (a key's elements are contiguous)
-            if (!mbar_wait(&sm.q_full, 0)) ok = false;
-            const uint32_t q0 = smem_u32(sm.Q[0]);
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                const int st = j % F_STAGES;
-                if (!mbar_wait(&sm.k_full[st], (j / F_STAGES) & 1)) { ok = false; break; }
-                tc_fence_after_sync();
-                const uint32_t k0 = smem_u32(sm.K[st][0]), v0 = smem_u32(sm.V[st][0]);
+            // The MMAs of one thread run in the order they were issued, and a commit covers everything issued before it:
+            // when s_full[b] fires for tile j + 1, block b's P V of tile j has also finished with the probabilities that
+            // these scores overwrite and with the output a softmax warp may rescale.
+            auto scores = [&](int b, int st) {
+                const uint32_t q0 = smem_u32(sm.Q[b][0]), k0 = smem_u32(sm.K[st][0]);
                 if (elect_one()) {
 #pragma unroll
                     for (int k = 0; k < 8; ++k) {
                         const uint32_t off = (k >> 2) * (TILE * KC * 2) + (k & 3) * 32;
-                        tc_mma_bf16(tmem, make_smem_desc_sw128(q0 + off, 0, 1024), make_smem_desc_sw128(k0 + off, 0, 1024),
-                                    idesc_s, k != 0);
+                        tc_mma_bf16(tmem + b * 128, make_smem_desc_sw128(q0 + off, 0, 1024),
+                                    make_smem_desc_sw128(k0 + off, 0, 1024), idesc_s, k != 0);
                     }
-                    tc_commit(&sm.s_full);
+                    tc_commit(&sm.s_full[b]);
+                    if (b == 1) tc_commit(&sm.k_empty[st]);
                 }
                 __syncwarp();
-                // the softmax warps have replaced the scores by probabilities (and rescaled the output if needed)
-                if (!mbar_wait(&sm.p_ready, j & 1)) { ok = false; break; }
-                if (!mbar_wait(&sm.v_full[st], (j / F_STAGES) & 1)) { ok = false; break; }
+            };
+            if (!mbar_wait(&sm.q_full, 0)) ok = false;
+            if (ok && !mbar_wait(&sm.k_full[0], 0)) ok = false;
+            if (ok) {
                 tc_fence_after_sync();
-                if (elect_one()) {
+                scores(0, 0);
+                scores(1, 0);
+            }
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const int st = j % F_STAGES, st1 = (j + 1) % F_STAGES;
+                const uint32_t v0 = smem_u32(sm.V[st][0]);
+#pragma unroll 1
+                for (int b = 0; b < 2 && ok; ++b) {
+                    // the softmax warps of block b have replaced its scores by probabilities (and rescaled its output if needed)
+                    if (!mbar_wait(&sm.p_ready[b], j & 1)) { ok = false; break; }
+                    if (b == 0 && !mbar_wait(&sm.v_full[st], (j / F_STAGES) & 1)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    if (elect_one()) {
 #pragma unroll
-                    for (int k = 0; k < 8; ++k)          // 16 keys per step: 8 columns of packed probabilities, 16 rows of V
-                        tc_mma_bf16_ts(tmem + 128, tmem + k * 8, make_smem_desc_sw128(v0 + k * 2048, TILE * KC * 2, 1024),
-                                       idesc_o, (j | k) != 0);
-                    tc_commit(&sm.kv_empty[st]);
-                    if (j + 1 == n_tiles) tc_commit(&sm.o_done);
+                        for (int k = 0; k < 8; ++k)      // 16 keys per step: 8 columns of packed probabilities, 16 rows of V
+                            tc_mma_bf16_ts(tmem + 256 + b * 128, tmem + b * 128 + k * 8,
+                                           make_smem_desc_sw128(v0 + k * 2048, TILE * KC * 2, 1024), idesc_o, (j | k) != 0);
+                        if (b == 1) tc_commit(&sm.v_empty[st]);
+                        if (b == 1 && j + 1 == n_tiles) tc_commit(&sm.o_done);
+                    }
+                    __syncwarp();
+                    if (j + 1 < n_tiles) {
+                        if (b == 0 && !mbar_wait(&sm.k_full[st1], ((j + 1) / F_STAGES) & 1)) { ok = false; break; }
+                        tc_fence_after_sync();
+                        scores(b, st1);
+                    }
                 }
-                __syncwarp();
             }
         }
         if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
     } else {
-        const int quarter = warp % 4;
+        const int b = (warp - 2) >> 2;                           // block of this softmax warp
+        const int quarter = warp % 4;                            // the 32 lanes of tensor memory this warp may touch
         const int row = quarter * 32 + lane;
-        const int tt = row / p.G, hi = row % p.G;
+        const int tt = b * qp + row / p.G, hi = row % p.G;
         const bool live = len > 0 && t0 + tt < p.T;
-        const int pq = len - p.T + t0 + tt;                     // this row's position: it sees keys 0 .. pq
-        const uint32_t trow = tmem + ((uint32_t)(quarter * 32) << 16);
-        float m_ref = -INFINITY, l = 0.f;
+        const int pq = live ? len - p.T + t0 + tt : -1;          // this row's position: it sees keys 0 .. pq
+        const uint32_t trow = tmem + ((uint32_t)(quarter * 32) << 16) + b * 128;   // scores / probabilities
+        const uint32_t orow = tmem + ((uint32_t)(quarter * 32) << 16) + 256 + b * 128;
+        float m_ref = -INFINITY, l0 = 0.f, l1 = 0.f;
         for (int j = 0; j < n_tiles && ok; ++j) {
-            if (!mbar_wait(&sm.s_full, j & 1)) { ok = false; break; }
+            if (!mbar_wait(&sm.s_full[b], j & 1)) { ok = false; break; }
             tc_fence_after_sync();
             const int n0 = j * TILE;
-            // pass 1: the tile's maximum over the keys this row may see
-            float mt = -INFINITY;
+            // the whole row of scores in registers
+            uint32_t r0[32], r1[32], r2[32], r3[32];
+            tmem_ld32(trow, r0);
+            tmem_ld32(trow + 32, r1);
+            tmem_ld32(trow + 64, r2);
+            tmem_ld32(trow + 96, r3);
+            tmem_wait_ld();
+            // keys past the row's own position (tiles on the diagonal, rows past the chunk) count as -inf
+            if (__any_sync(0xffffffffu, n0 + TILE - 1 > pq)) {
 #pragma unroll
-            for (int c0 = 0; c0 < TILE; c0 += 32) {
-                uint32_t r[32];
-                tmem_ld32(trow + c0, r);
-                tmem_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (live && n0 + c0 + i <= pq) mt = fmaxf(mt, __uint_as_float(r[i]));
+                for (int i = 0; i < 32; ++i) {
+                    if (n0 + i > pq) r0[i] = 0xff800000u;
+                    if (n0 + 32 + i > pq) r1[i] = 0xff800000u;
+                    if (n0 + 64 + i > pq) r2[i] = 0xff800000u;
+                    if (n0 + 96 + i > pq) r3[i] = 0xff800000u;
+                }
             }
+            float mt0 = -INFINITY, mt1 = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                mt0 = fmaxf(mt0, fmaxf(__uint_as_float(r0[i]), __uint_as_float(r1[i])));
+                mt1 = fmaxf(mt1, fmaxf(__uint_as_float(r2[i]), __uint_as_float(r3[i])));
+            }
+            const float mt = fmaxf(mt0, mt1);
             // raise the reference?  (the accesses to tensor memory below are warp-wide: the warp rescales if any of its
             // rows must, the other rows by a factor of one)
             const bool raise = mt > m_ref + F_RAISE || (m_ref == -INFINITY && mt > -INFINITY);
             if (__any_sync(0xffffffffu, raise)) {
                 // what has been accumulated so far shrinks by 2^(old - new)
                 const float alpha = !raise ? 1.f : (m_ref == -INFINITY ? 0.f : exp2f(m_ref - mt));
-                l *= alpha;
+                l0 *= alpha;
+                l1 *= alpha;
                 if (j > 0) {
-#pragma unroll
-                    for (int c0 = 0; c0 < TILE; c0 += 32) {
-                        uint32_t o[32];
-                        tmem_ld32(trow + 128 + c0, o);
+#pragma unroll 1
+                    for (int c0 = 0; c0 < TILE; c0 += 16) {
+                        uint32_t o[16];
+                        tmem_ld16(orow + c0, o);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                        tmem_st32(trow + 128 + c0, o);
+                        for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st16(orow + c0, o);
                     }
                 }
                 if (raise) m_ref = mt;
             }
-            // pass 2: probabilities (at most 2^8), rounded to bf16, packed two per column over the scores they came from
-#pragma unroll
-            for (int c0 = 0; c0 < TILE; c0 += 32) {
-                uint32_t r[32], w[16];
-                tmem_ld32(trow + c0, r);
-                tmem_wait_ld();
+            // probabilities (at most 2^8), rounded to bf16, packed two per column over the scores they came from
+            const float m_use = m_ref == -INFINITY ? 0.f : m_ref;     // a row that has seen nothing yet: 2^(-inf) = 0
+            auto probs = [&](const uint32_t (&r)[32], int c0) {
+                uint32_t w[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    const bool v0 = live && n0 + c0 + 2 * i <= pq, v1 = live && n0 + c0 + 2 * i + 1 <= pq;
-                    const __nv_bfloat162 pr = __floats2bfloat162_rn(v0 ? exp2f(__uint_as_float(r[2 * i]) - m_ref) : 0.f,
-                                                                    v1 ? exp2f(__uint_as_float(r[2 * i + 1]) - m_ref) : 0.f);
-                    l += __low2float(pr) + __high2float(pr);
+                    const float e0 = ex2_approx(__uint_as_float(r[2 * i]) - m_use);
+                    const float e1 = ex2_approx(__uint_as_float(r[2 * i + 1]) - m_use);
+                    l0 += e0;
+                    l1 += e1;
+                    const __nv_bfloat162 pr = __floats2bfloat162_rn(e0, e1);
                     w[i] = *reinterpret_cast<const uint32_t*>(&pr);
                 }
-                // columns c0 / 2 .. c0 / 2 + 15 lie below column c0 + 32: every score they overwrite has been read
                 tmem_st16(trow + c0 / 2, w);
-            }
+            };
+            probs(r0, 0);
+            probs(r1, 32);
+            probs(r2, 64);
+            probs(r3, 96);
             tmem_wait_st();
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.p_ready);
+            if (lane == 0) mbar_arrive(&sm.p_ready[b]);
         }
         if (n_tiles > 0 && ok) {
             if (!mbar_wait(&sm.o_done, 0)) ok = false;
@@ -410,16 +469,17 @@ lorc_prefill_attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_
         if (ok) {
             tc_fence_after_sync();
             const bool has_out = t0 + tt < p.T;                // (rows past the chunk still take part in the warp-wide loads)
+            const float l = l0 + l1;
             const float inv = l > 0.f ? 1.f / l : 0.f;
             // a NaN means non-finite numbers in the cache, the factors or the query (or a key beyond the fp16 range)
             if (has_out && l != l) lorc_set_status(p.status, LORC_ERR_ARG);
-            if (has_out && !(l > 0.f) && l == l && hi == 0 && g == 0 && tt == 0) lorc_set_status(p.status, LORC_ERR_EMPTY);
+            if (has_out && !(l > 0.f) && l == l && hi == 0 && g == 0 && t0 + tt == 0) lorc_set_status(p.status, LORC_ERR_EMPTY);
             bf16* dst = p.out + (((long long)s * p.T + (has_out ? t0 + tt : 0)) * p.H_q + g * p.G + hi) * 128;
 #pragma unroll
             for (int c0 = 0; c0 < TILE; c0 += 32) {
                 uint32_t o[32];
                 if (n_tiles > 0) {
-                    tmem_ld32(trow + 128 + c0, o);
+                    tmem_ld32(orow + c0, o);
                     tmem_wait_ld();
                 } else {
 #pragma unroll
@@ -442,7 +502,7 @@ lorc_prefill_attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem, 256);
+    if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
 }  // namespace
@@ -519,7 +579,7 @@ cudaError_t lorc_tc_prefill_launch(lorc_ctx* ctx, const LorcLayer& L, const Cach
     FaParams fp;
     fp.out = out; fp.seq_lens = cv.seq_lens; fp.status = ctx->status_dev;
     fp.T = T; fp.H_q = d.n_q_heads; fp.G = ctx->group; fp.n_rows = (int)rows; fp.max_pos = d.max_pos;
-    const int qp = TILE / ctx->group;
+    const int qp = 2 * TILE / ctx->group;                      // query positions per CTA (two blocks of 128 rows)
     dim3 fgrid((T + qp - 1) / qp, d.n_kv_heads, cv.batch);
     lorc_prefill_attn_kernel<<<fgrid, F_THREADS, sizeof(FaSmem) + 1024, st>>>(mapQ, mapK, mapV, fp);
     *launches += 1;
