@@ -8,8 +8,9 @@
 //
 //   query kernel        Q^[b, T, H_q, 128] = RoPE(q, position) * log2(e) / sqrt(d_h), fp16
 //   reconstruct kernel  K^[tile, head] = RoPE(C_K[tile, :] . B_K[:, head]),  V[tile, head] = C_V[tile, :] . B_V[:, head]
-//                       one CTA per (128-token tile, KV head): TMA-staged 64-wide slices, tcgen05 (M = 128 tokens,
-//                       N = 128), rotation in the epilogue (thread = token row), 16-bit rows to the buffer: keys as
+//                       persistent CTAs over (128-token tile, pair of KV heads): TMA-staged 64-wide slices, tcgen05
+//                       (M = 128 tokens, N = 256), rotation in the epilogue (thread = token row) under the next unit's
+//                       MMAs, 16-bit rows to the buffer: keys as
 //                       fp16 (the scores are then exact to 2^-11 of |q| |k|, four times closer than with bf16 keys;
 //                       a rotated key element must stay below 65504 in magnitude), values as bf16
 //   attention kernel    one CTA per two blocks of 128 query rows (128 / G positions x G heads of one KV head each): for
@@ -55,13 +56,19 @@ __global__ void prefill_query_kernel(const bf16* __restrict__ q, __half* __restr
 // ------------------------------------------------------------------------------------------------
 // reconstruction of keys (rotated) or values into [b, n_rows, n] bf16
 // ------------------------------------------------------------------------------------------------
+// Persistent: a CTA walks units (sequence, 128-token tile, pair of KV heads) u = blockIdx.x, blockIdx.x + gridDim.x, ...
+// with the head pair running fastest (the CTAs that work on the same latent rows at the same time share them in L2).
+// Per unit  acc[128 tokens, 256 features] = C[tile, :] . B[:, 2 heads]  in 64-wide slices (M = 128, N = 256); the
+// accumulator is double-buffered in tensor memory, so the epilogue of one unit (rotation, rounding, 512-byte row
+// stores) runs under the MMAs of the next.
 constexpr int R_STAGES = 4;
 constexpr int R_THREADS = 192;       // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+constexpr int R_N = 256;             // features per unit: two KV heads
 
 struct RecSmem {
     bf16 A[R_STAGES][TILE * KC];          // latent slice [128 tokens][64]
-    bf16 B[R_STAGES][TILE * KC];          // factor slice [128 features of the head][64]
-    uint64_t full[R_STAGES], empty[R_STAGES], d_full;
+    bf16 B[R_STAGES][R_N * KC];           // factor slice [256 features][64]
+    uint64_t full[R_STAGES], empty[R_STAGES], acc_full[2], acc_empty[2];
     uint32_t tmem_base;
 };
 
@@ -71,7 +78,7 @@ struct RecParams {
     const int32_t* page_table;
     const float2* rope_table;      // [max_pos][64]
     int* status;
-    int r, n, n_rows, max_pos;
+    int r, n, n_rows, max_pos, batch, tiles, n_hp;
     int page_size, max_pages_per_seq, n_pages;
 };
 
@@ -81,24 +88,35 @@ lorc_reconstruct_kernel(const __grid_constant__ CUtensorMap mapC, const __grid_c
     extern __shared__ uint8_t raw[];
     RecSmem& sm = *reinterpret_cast<RecSmem*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
-    const int tile = blockIdx.x, g = blockIdx.y, s = blockIdx.z;
-    int len = p.seq_lens[s];
-    if (len > p.max_pos || len > p.n_rows) len = 0;          // reported by the attention kernel
-    if (tile * TILE >= len) return;                          // nothing cached in this tile (uniform for the block)
     const int nkc = (p.r + KC - 1) / KC;
+    const int total = p.batch * p.tiles * p.n_hp;
+    // unit -> (sequence, tile, head pair); a unit whose tile lies past the sequence's cached tokens is skipped by
+    // every role alike (sequences beyond the buffer are reported by the attention kernel)
+    auto decode = [&](int u, int& s, int& tile, int& hp) -> bool {
+        hp = u % p.n_hp;
+        const int st = u / p.n_hp;
+        tile = st % p.tiles;
+        s = st / p.tiles;
+        int len = p.seq_lens[s];
+        if (len > p.max_pos || len > p.n_rows) len = 0;
+        return tile * TILE < len;
+    };
 
     if (tid == 0) {
         for (int i = 0; i < R_STAGES; ++i) {
             mbar_init(&sm.full[i], 1);
             mbar_init(&sm.empty[i], 1);
         }
-        mbar_init(&sm.d_full, 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&sm.acc_full[i], 1);
+            mbar_init(&sm.acc_empty[i], 4);
+        }
         fence_barrier_init();
         prefetch_tensormap(&mapC);
         prefetch_tensormap(&mapBT);
     }
     if (warp == 1) {
-        tmem_alloc(&sm.tmem_base, 128);
+        tmem_alloc(&sm.tmem_base, 512);
         tmem_relinquish();
     }
     tc_fence_before_sync();
@@ -108,106 +126,134 @@ lorc_reconstruct_kernel(const __grid_constant__ CUtensorMap mapC, const __grid_c
     bool ok = true;
 
     if (warp == 0) {
-        for (int kc = 0; kc < nkc && ok; ++kc) {
-            const int st = kc % R_STAGES;
-            if (!mbar_wait(&sm.empty[st], ((kc / R_STAGES) & 1) ^ 1)) { ok = false; break; }
-            if (elect_one()) {
-                mbar_arrive_expect_tx(&sm.full[st], 2 * TILE * KC * 2);
-                if (p.page_table == nullptr) {
-                    tma_load_3d(sm.A[st], &mapC, &sm.full[st], kc * KC, tile * TILE, s);
-                } else {
-                    // one box per page; pages past the end of the sequence (or with a bad table entry) come from page 0
-                    const int ppt = TILE / p.page_size;
-                    for (int pg = 0; pg < ppt; ++pg) {
-                        const int lp = tile * ppt + pg;
-                        int page = 0;
-                        if ((long long)lp * p.page_size < len && lp < p.max_pages_per_seq) {
-                            page = p.page_table[(long long)s * p.max_pages_per_seq + lp];
-                            if (page < 0 || page >= p.n_pages) {
-                                lorc_set_status(p.status, LORC_ERR_CAPACITY);
-                                page = 0;
+        uint32_t it = 0;                                         // stages issued so far
+        for (int u = blockIdx.x; u < total && ok; u += gridDim.x) {
+            int s, tile, hp;
+            if (!decode(u, s, tile, hp)) continue;
+            const int len = p.seq_lens[s];
+            for (int kc = 0; kc < nkc && ok; ++kc, ++it) {
+                const int st = it % R_STAGES;
+                if (!mbar_wait(&sm.empty[st], ((it / R_STAGES) & 1) ^ 1)) { ok = false; break; }
+                if (elect_one()) {
+                    mbar_arrive_expect_tx(&sm.full[st], (TILE + R_N) * KC * 2);
+                    if (p.page_table == nullptr) {
+                        tma_load_3d(sm.A[st], &mapC, &sm.full[st], kc * KC, tile * TILE, s);
+                    } else {
+                        // one box per page; pages past the end of the sequence (or with a bad table entry) come from page 0
+                        const int ppt = TILE / p.page_size;
+                        for (int pg = 0; pg < ppt; ++pg) {
+                            const int lp = tile * ppt + pg;
+                            int page = 0;
+                            if ((long long)lp * p.page_size < len && lp < p.max_pages_per_seq) {
+                                page = p.page_table[(long long)s * p.max_pages_per_seq + lp];
+                                if (page < 0 || page >= p.n_pages) {
+                                    lorc_set_status(p.status, LORC_ERR_CAPACITY);
+                                    page = 0;
+                                }
                             }
+                            tma_load_3d(sm.A[st] + pg * p.page_size * KC, &mapC, &sm.full[st], kc * KC, 0, page);
                         }
-                        tma_load_3d(sm.A[st] + pg * p.page_size * KC, &mapC, &sm.full[st], kc * KC, 0, page);
                     }
+                    tma_load_2d(sm.B[st], &mapBT, &sm.full[st], kc * KC, hp * R_N);
+                    tma_load_2d(sm.B[st] + TILE * KC, &mapBT, &sm.full[st], kc * KC, hp * R_N + 128);
                 }
-                tma_load_2d(sm.B[st], &mapBT, &sm.full[st], kc * KC, g * 128);
+                __syncwarp();
             }
-            __syncwarp();
         }
         if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
     } else if (warp == 1) {
-        const uint32_t idesc = make_idesc_bf16(128, 128, 0, 0);
+        const uint32_t idesc = make_idesc_bf16(128, R_N, 0, 0);
         const int nk_last = (p.r - (nkc - 1) * KC + 15) >> 4;
-        for (int kc = 0; kc < nkc && ok; ++kc) {
-            const int st = kc % R_STAGES;
-            if (!mbar_wait(&sm.full[st], (kc / R_STAGES) & 1)) { ok = false; break; }
+        uint32_t it = 0, uc = 0;
+        for (int u = blockIdx.x; u < total && ok; u += gridDim.x) {
+            int s, tile, hp;
+            if (!decode(u, s, tile, hp)) continue;
+            const int buf = uc & 1;
+            if (!mbar_wait(&sm.acc_empty[buf], ((uc >> 1) & 1) ^ 1)) { ok = false; break; }
             tc_fence_after_sync();
-            const uint32_t a0 = smem_u32(sm.A[st]), b0 = smem_u32(sm.B[st]);
-            if (elect_one()) {
-                const int nk = (kc + 1 < nkc) ? 4 : nk_last;
-                for (int k = 0; k < nk; ++k)
-                    tc_mma_bf16(tmem, make_smem_desc_sw128(a0 + k * 32, 0, 1024), make_smem_desc_sw128(b0 + k * 32, 0, 1024),
-                                idesc, (kc | k) != 0);
-                tc_commit(&sm.empty[st]);
+            for (int kc = 0; kc < nkc && ok; ++kc, ++it) {
+                const int st = it % R_STAGES;
+                if (!mbar_wait(&sm.full[st], (it / R_STAGES) & 1)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t a0 = smem_u32(sm.A[st]), b0 = smem_u32(sm.B[st]);
+                if (elect_one()) {
+                    const int nk = (kc + 1 < nkc) ? 4 : nk_last;
+                    for (int k = 0; k < nk; ++k)
+                        tc_mma_bf16(tmem + buf * R_N, make_smem_desc_sw128(a0 + k * 32, 0, 1024),
+                                    make_smem_desc_sw128(b0 + k * 32, 0, 1024), idesc, (kc | k) != 0);
+                    tc_commit(&sm.empty[st]);
+                }
+                __syncwarp();
             }
+            if (!ok) break;
+            if (elect_one()) tc_commit(&sm.acc_full[buf]);
             __syncwarp();
-        }
-        if (ok) {
-            if (elect_one()) tc_commit(&sm.d_full);
-            __syncwarp();
+            ++uc;
         }
         if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
     } else {
-        if (!mbar_wait(&sm.d_full, 0)) ok = false;
-        if (ok) {
+        const int quarter = warp % 4;
+        const int row = quarter * 32 + lane;                         // token of the tile = TMEM lane
+        uint32_t uc = 0;
+        for (int u = blockIdx.x; u < total && ok; u += gridDim.x) {
+            int s, tile, hp;
+            if (!decode(u, s, tile, hp)) continue;
+            const int buf = uc & 1;
+            if (!mbar_wait(&sm.acc_full[buf], (uc >> 1) & 1)) { ok = false; break; }
             tc_fence_after_sync();
-            const int quarter = warp % 4;
-            const int row = quarter * 32 + lane;                     // token of the tile = TMEM lane
             const int pos = tile * TILE + row;
-            bf16* dst = p.out + ((long long)s * p.n_rows + pos) * p.n + g * 128;
             const float2* cs = p.rope_table + (long long)min(pos, p.max_pos - 1) * 64;
+#pragma unroll 1
+            for (int hd = 0; hd < 2; ++hd) {
+                bf16* dst = p.out + ((long long)s * p.n_rows + pos) * p.n + (hp * 2 + hd) * 128;
+                const uint32_t tcol = tmem + ((uint32_t)(quarter * 32) << 16) + buf * R_N + hd * 128;
 #pragma unroll
-            for (int c0 = 0; c0 < 64; c0 += 32) {
-                uint32_t ra[32], rb[32];
-                tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + c0, ra);          // elements c0 .. c0 + 31 of the head
-                tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + 64 + c0, rb);     // their partners in the second half
-                tmem_wait_ld();
-                if (pos < p.n_rows) {
-                    uint32_t wa[16], wb[16];
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    uint32_t ra[32], rb[32];
+                    tmem_ld32(tcol + c0, ra);          // elements c0 .. c0 + 31 of the head
+                    tmem_ld32(tcol + 64 + c0, rb);     // their partners in the second half
+                    tmem_wait_ld();
+                    if (pos < p.n_rows) {
+                        uint32_t wa[16], wb[16];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        float a0 = __uint_as_float(ra[2 * i]), a1 = __uint_as_float(ra[2 * i + 1]);
-                        float b0 = __uint_as_float(rb[2 * i]), b1 = __uint_as_float(rb[2 * i + 1]);
-                        if (ROPE) {
-                            const float4 t = __ldg(reinterpret_cast<const float4*>(cs + c0 + 2 * i));   // (cos, sin) x 2
-                            const float x0 = a0 * t.x - b0 * t.y, y0 = a0 * t.y + b0 * t.x;
-                            const float x1 = a1 * t.z - b1 * t.w, y1 = a1 * t.w + b1 * t.z;
-                            a0 = x0; b0 = y0; a1 = x1; b1 = y1;
+                        for (int i = 0; i < 16; ++i) {
+                            float a0 = __uint_as_float(ra[2 * i]), a1 = __uint_as_float(ra[2 * i + 1]);
+                            float b0 = __uint_as_float(rb[2 * i]), b1 = __uint_as_float(rb[2 * i + 1]);
+                            if (ROPE) {
+                                const float4 t = __ldg(reinterpret_cast<const float4*>(cs + c0 + 2 * i));   // (cos, sin) x 2
+                                const float x0 = a0 * t.x - b0 * t.y, y0 = a0 * t.y + b0 * t.x;
+                                const float x1 = a1 * t.z - b1 * t.w, y1 = a1 * t.w + b1 * t.z;
+                                a0 = x0; b0 = y0; a1 = x1; b1 = y1;
+                            }
+                            if (ROPE) {          // keys: fp16
+                                const __half2 pa = __floats2half2_rn(a0, a1), pb = __floats2half2_rn(b0, b1);
+                                wa[i] = *reinterpret_cast<const uint32_t*>(&pa);
+                                wb[i] = *reinterpret_cast<const uint32_t*>(&pb);
+                            } else {             // values: bf16
+                                const __nv_bfloat162 pa = __floats2bfloat162_rn(a0, a1), pb = __floats2bfloat162_rn(b0, b1);
+                                wa[i] = *reinterpret_cast<const uint32_t*>(&pa);
+                                wb[i] = *reinterpret_cast<const uint32_t*>(&pb);
+                            }
                         }
-                        if (ROPE) {          // keys: fp16
-                            const __half2 pa = __floats2half2_rn(a0, a1), pb = __floats2half2_rn(b0, b1);
-                            wa[i] = *reinterpret_cast<const uint32_t*>(&pa);
-                            wb[i] = *reinterpret_cast<const uint32_t*>(&pb);
-                        } else {             // values: bf16
-                            const __nv_bfloat162 pa = __floats2bfloat162_rn(a0, a1), pb = __floats2bfloat162_rn(b0, b1);
-                            wa[i] = *reinterpret_cast<const uint32_t*>(&pa);
-                            wb[i] = *reinterpret_cast<const uint32_t*>(&pb);
-                        }
-                    }
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        reinterpret_cast<uint4*>(dst + c0)[v] = make_uint4(wa[4 * v], wa[4 * v + 1], wa[4 * v + 2], wa[4 * v + 3]);
-                        reinterpret_cast<uint4*>(dst + 64 + c0)[v] = make_uint4(wb[4 * v], wb[4 * v + 1], wb[4 * v + 2], wb[4 * v + 3]);
+                        for (int v = 0; v < 4; ++v) {
+                            reinterpret_cast<uint4*>(dst + c0)[v] = make_uint4(wa[4 * v], wa[4 * v + 1], wa[4 * v + 2], wa[4 * v + 3]);
+                            reinterpret_cast<uint4*>(dst + 64 + c0)[v] = make_uint4(wb[4 * v], wb[4 * v + 1], wb[4 * v + 2], wb[4 * v + 3]);
+                        }
                     }
                 }
             }
+            // this warp has read its part of the accumulator
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.acc_empty[buf]);
+            ++uc;
         }
         if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem, 128);
+    if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -553,7 +599,9 @@ cudaError_t lorc_tc_prefill_launch(lorc_ctx* ctx, const LorcLayer& L, const Cach
     rp.seq_lens = cv.seq_lens; rp.page_table = cv.page_table; rp.rope_table = ctx->rope_table; rp.status = ctx->status_dev;
     rp.n = ctx->n; rp.n_rows = (int)rows; rp.max_pos = d.max_pos;
     rp.page_size = cv.page_size; rp.max_pages_per_seq = cv.max_pages_per_seq; rp.n_pages = cv.n_pages;
-    dim3 rgrid(tiles, d.n_kv_heads, cv.batch);
+    rp.batch = cv.batch; rp.tiles = tiles; rp.n_hp = d.n_kv_heads / 2;
+    const int units = cv.batch * tiles * rp.n_hp;
+    dim3 rgrid(units < ctx->sm_count ? units : ctx->sm_count);
     rp.out = khat; rp.r = L.r_k;
     lorc_reconstruct_kernel<true><<<rgrid, R_THREADS, sizeof(RecSmem) + 1024, st>>>(mapCK, mapBKT, rp);
     *launches += 1;
