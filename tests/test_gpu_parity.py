@@ -378,3 +378,26 @@ def test_latent_output_entry_plain_kernels(flags):
     assert e.value.code == sess.L.LORC_ERR_UNSUPPORTED
     full.close()
     sess.close()
+
+
+def test_fp32_debug_path_one_sequence_of_32768_tokens():
+    """The plain fp32 kernels over one long sequence (the context length of the long-context configuration) at a
+    small rank, element by element: 256 context splits, 2048 tiles, positions up to 32767 in the rotation table."""
+    import torch
+    N, D, H_q, H_kv, d_h, r_k, r_v = 32768, 256, 8, 2, 64, 32, 24
+    prob = H.Problem(D, H_q, H_kv, d_h, r_k, r_v, theta=500000.0, layer=9)
+    sess = H.Session(prob, max_pos=N, batch=1, flags=H.lib().LORC_FLAG_DEBUG_FP32)
+    # latent rows seeded directly (coordinate i of a row ~ N(0, sigma_i^2), what x A gives for x ~ N(0, I)), bf16-exact
+    rng = np.random.default_rng(99)
+    ck = [synth.to_bf16_exact(rng.standard_normal((N, r_k)) * (np.arange(1, r_k + 1) ** -0.8))]
+    cv = [synth.to_bf16_exact(rng.standard_normal((N, r_v)) * (np.arange(1, r_v + 1) ** -0.8))]
+    held = H.contiguous_cache(sess, 1, N, [N], ck, cv)
+    for q_scale in (1.0, 64.0):
+        q = synth.queries(1, H_q, d_h, 9, int(q_scale), q_scale).astype(np.float64)
+        out = torch.zeros(1, H_q, d_h, dtype=torch.bfloat16, device="cuda")
+        sess.L.lorc_decode_attn(sess.ctx, 0, held[0], H.dev_bf16(q), out)
+        assert sess.L.lorc_sync_status(sess.ctx) == 0, sess.L.lorc_last_error(sess.ctx)
+        assert sess.L.lorc_last_path(sess.ctx) == 1
+        want = H.oracle_decode(prob, ck, cv, q)
+        _check_fp32_path(H.host_f64(out), want)
+    sess.close()
