@@ -6,14 +6,15 @@
 // a transient bf16 buffer (the decode path rebuilds them per query and never stores them), then a flash-attention
 // kernel runs over that buffer.
 //
-//   query kernel        Q^[b, T, H_q, 128] = RoPE(q, position) * log2(e) / sqrt(d_h), fp16
 //   reconstruct kernel  K^[tile, head] = RoPE(C_K[tile, :] . B_K[:, head]),  V[tile, head] = C_V[tile, :] . B_V[:, head]
 //                       persistent CTAs over (128-token tile, pair of KV heads): TMA-staged 64-wide slices, tcgen05
 //                       (M = 128 tokens, N = 256), rotation in the epilogue (thread = token row) under the next unit's
 //                       MMAs, 16-bit rows to the buffer: keys as
 //                       fp16 (the scores are then exact to 2^-11 of |q| |k|, four times closer than with bf16 keys;
 //                       a rotated key element must stay below 65504 in magnitude), values as bf16
-//   attention kernel    one CTA per two blocks of 128 query rows (128 / G positions x G heads of one KV head each): for
+//   attention kernel    one CTA per two blocks of 128 query rows (128 / G positions x G heads of one KV head each); the
+//                       rows are rotated at their positions and scaled in shared memory, Q^ = RoPE(q) log2(e) / sqrt(d_h)
+//                       as fp16, before the first MMA; for
 //                       every 128-key tile and block   S = Q^ K^^T (tcgen05, fp32 in TMEM)  ->  online softmax, thread =
 //                       query row; the probabilities go back into tensor memory as bf16 over the scores  ->  O += P V
 //                       with P read from tensor memory.  The two blocks alternate, so the tensor pipe works on one
@@ -32,26 +33,6 @@ namespace {
 constexpr int TILE = 128;
 constexpr int KC = 64;
 constexpr float LOG2E = 1.4426950408889634f;
-
-// ------------------------------------------------------------------------------------------------
-// rotated, scaled queries
-// ------------------------------------------------------------------------------------------------
-__global__ void prefill_query_kernel(const bf16* __restrict__ q, __half* __restrict__ qhat, const int32_t* __restrict__ seq_lens,
-                                     const float2* __restrict__ rope_table, int T, int H_q, int max_pos) {
-    const int t = blockIdx.x, s = blockIdx.y;
-    const int len = seq_lens[s];
-    int pos = len - T + t;
-    if (pos < 0 || pos >= max_pos) pos = 0;                 // such a sequence is rejected by the attention kernel
-    const float scale = rsqrtf(128.f) * LOG2E;
-    for (int i = threadIdx.x; i < H_q * 64; i += blockDim.x) {
-        const int h = i >> 6, j = i & 63;
-        const long long base = (((long long)s * T + t) * H_q + h) * 128;
-        const float a = __bfloat162float(q[base + j]), b = __bfloat162float(q[base + 64 + j]);
-        const float2 cs = rope_table[(long long)pos * 64 + j];
-        qhat[base + j] = __float2half_rn((a * cs.x - b * cs.y) * scale);
-        qhat[base + 64 + j] = __float2half_rn((a * cs.y + b * cs.x) * scale);
-    }
-}
 
 // ------------------------------------------------------------------------------------------------
 // reconstruction of keys (rotated) or values into [b, n_rows, n] bf16
@@ -271,7 +252,7 @@ struct FaSmem {
     bf16 Q[2][2][TILE * KC];              // [block][64-element half][128 rows]
     bf16 K[F_STAGES][2][TILE * KC];       // key tile [128 keys][two halves]
     bf16 V[F_STAGES][2][TILE * KC];       // value tile [128 keys][two halves]
-    uint64_t q_full, k_full[F_STAGES], v_full[F_STAGES], k_empty[F_STAGES], v_empty[F_STAGES];
+    uint64_t q_full, q_ready, k_full[F_STAGES], v_full[F_STAGES], k_empty[F_STAGES], v_empty[F_STAGES];
     uint64_t s_full[2], p_ready[2], o_done;
     uint32_t tmem_base;
 };
@@ -279,6 +260,7 @@ struct FaSmem {
 struct FaParams {
     bf16* out;                     // [b, T, H_q, 128]
     const int32_t* seq_lens;
+    const float2* rope_table;      // [max_pos][64]
     int* status;
     int T, H_q, G, n_rows, max_pos;
 };
@@ -313,6 +295,7 @@ lorc_prefill_attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_
 
     if (tid == 0) {
         mbar_init(&sm.q_full, 1);
+        mbar_init(&sm.q_ready, 8);
         for (int i = 0; i < F_STAGES; ++i) {
             mbar_init(&sm.k_full[i], 1);
             mbar_init(&sm.v_full[i], 1);
@@ -392,7 +375,7 @@ lorc_prefill_attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_
                 }
                 __syncwarp();
             };
-            if (!mbar_wait(&sm.q_full, 0)) ok = false;
+            if (!mbar_wait(&sm.q_ready, 0)) ok = false;          // the query rows, rotated and scaled in place
             if (ok && !mbar_wait(&sm.k_full[0], 0)) ok = false;
             if (ok) {
                 tc_fence_after_sync();
@@ -436,6 +419,42 @@ lorc_prefill_attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_
         const uint32_t trow = tmem + ((uint32_t)(quarter * 32) << 16) + b * 128;   // scores / probabilities
         const uint32_t orow = tmem + ((uint32_t)(quarter * 32) << 16) + 256 + b * 128;
         float m_ref = -INFINITY, l0 = 0.f, l1 = 0.f;
+        if (n_tiles > 0) {
+            // Q^ = RoPE(q, position) * log2(e) / sqrt(d_h), fp16, in place: this thread's row of the block, 16 bytes at a
+            // time.  The two 64-element halves of a row have the same swizzled layout, so a rotary pair (j, j + 64) sits
+            // at the same offset of both; elements 8 lc ... 8 lc + 7 of row r are its physical 16-byte piece lc ^ (r & 7).
+            if (!mbar_wait(&sm.q_full, 0)) ok = false;
+            if (ok) {
+                const float scale = rsqrtf(128.f) * LOG2E;
+                const float2* cs = p.rope_table + (long long)min(max(pq, 0), p.max_pos - 1) * 64;
+                uint4* h0 = reinterpret_cast<uint4*>(sm.Q[b][0]) + row * 8;
+                uint4* h1 = reinterpret_cast<uint4*>(sm.Q[b][1]) + row * 8;
+#pragma unroll
+                for (int lc = 0; lc < 8; ++lc) {
+                    // logical piece lc of every row at once: the rows of a quarter warp then touch all eight physical
+                    // pieces (no shared-memory bank conflict)
+                    const int pc = lc ^ (row & 7), j0 = 8 * lc;
+                    uint4 a = h0[pc], c = h1[pc];
+                    uint32_t* aw = reinterpret_cast<uint32_t*>(&a);
+                    uint32_t* cw = reinterpret_cast<uint32_t*>(&c);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float4 t = __ldg(reinterpret_cast<const float4*>(cs + j0 + 2 * e));   // (cos, sin) x 2
+                        const float a0 = __uint_as_float(aw[e] << 16), a1 = __uint_as_float(aw[e] & 0xffff0000u);
+                        const float b0 = __uint_as_float(cw[e] << 16), b1 = __uint_as_float(cw[e] & 0xffff0000u);
+                        const __half2 x = __floats2half2_rn((a0 * t.x - b0 * t.y) * scale, (a1 * t.z - b1 * t.w) * scale);
+                        const __half2 y = __floats2half2_rn((a0 * t.y + b0 * t.x) * scale, (a1 * t.w + b1 * t.z) * scale);
+                        aw[e] = *reinterpret_cast<const uint32_t*>(&x);
+                        cw[e] = *reinterpret_cast<const uint32_t*>(&y);
+                    }
+                    h0[pc] = a;
+                    h1[pc] = c;
+                }
+                fence_proxy_async_smem();      // the MMA reads the rows through the asynchronous proxy
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.q_ready);
+            }
+        }
         for (int j = 0; j < n_tiles && ok; ++j) {
             if (!mbar_wait(&sm.s_full[b], j & 1)) { ok = false; break; }
             tc_fence_after_sync();
@@ -556,13 +575,13 @@ lorc_prefill_attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
-// scratch: [Q^ | K^ | V], rows of the key / value buffers rounded up to whole tiles
+// scratch: [K^ | V], rows of the key / value buffers rounded up to whole tiles
 static size_t prefill_rows(int max_seq_len) { return (size_t)((max_seq_len + TILE - 1) / TILE) * TILE; }
 
 size_t lorc_tc_prefill_scratch_bytes(const lorc_ctx* ctx, int batch, int max_seq_len, int T) {
-    const size_t q = lorc_align_up((size_t)batch * T * ctx->desc.n_q_heads * 128 * sizeof(bf16), 256);
+    (void)T;
     const size_t kv = lorc_align_up((size_t)batch * prefill_rows(max_seq_len) * ctx->n * sizeof(bf16), 256);
-    return q + 2 * kv;
+    return 2 * kv;
 }
 
 cudaError_t lorc_tc_prefill_set_attrs() {
@@ -582,18 +601,11 @@ cudaError_t lorc_tc_prefill_launch(lorc_ctx* ctx, const LorcLayer& L, const Cach
                                    const bf16* q, bf16* out, int T, void* scratch, cudaStream_t st, int* launches) {
     const lorc_model_desc& d = ctx->desc;
     const size_t rows = prefill_rows(cv.max_seq_len);
-    const size_t q_bytes = lorc_align_up((size_t)cv.batch * T * d.n_q_heads * 128 * sizeof(bf16), 256);
     const size_t kv_bytes = lorc_align_up((size_t)cv.batch * rows * ctx->n * sizeof(bf16), 256);
-    bf16* qhat = (bf16*)scratch;
-    bf16* khat = (bf16*)((char*)scratch + q_bytes);
-    bf16* vbuf = (bf16*)((char*)scratch + q_bytes + kv_bytes);
+    bf16* khat = (bf16*)scratch;
+    bf16* vbuf = (bf16*)((char*)scratch + kv_bytes);
     const int tiles = (int)(rows / TILE);
-
-    prefill_query_kernel<<<dim3(T, cv.batch), 256, 0, st>>>(q, reinterpret_cast<__half*>(qhat), cv.seq_lens, ctx->rope_table, T,
-                                                            d.n_q_heads, d.max_pos);
-    *launches += 1;
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    cudaError_t e;
 
     RecParams rp;
     rp.seq_lens = cv.seq_lens; rp.page_table = cv.page_table; rp.rope_table = ctx->rope_table; rp.status = ctx->status_dev;
@@ -613,11 +625,11 @@ cudaError_t lorc_tc_prefill_launch(lorc_ctx* ctx, const LorcLayer& L, const Cach
 
     CUtensorMap mapQ, mapK, mapV;
     {
-        // Q^ [b, T, H_q, 128]: box = 64 elements x G heads x 128 / G positions
+        // q [b, T, H_q, 128]: box = 64 elements x G heads x 128 / G positions
         uint64_t dims[4] = {128, (uint64_t)d.n_q_heads, (uint64_t)T, (uint64_t)cv.batch};
         uint64_t str[3] = {128 * 2, (uint64_t)d.n_q_heads * 128 * 2, (uint64_t)T * d.n_q_heads * 128 * 2};
         uint32_t box[4] = {KC, (uint32_t)ctx->group, (uint32_t)(TILE / ctx->group), 1};
-        if (!lorc_make_tmap_bf16(&mapQ, qhat, 4, dims, str, box)) return cudaErrorInvalidValue;
+        if (!lorc_make_tmap_bf16(&mapQ, q, 4, dims, str, box)) return cudaErrorInvalidValue;
         uint64_t kd[3] = {(uint64_t)ctx->n, (uint64_t)rows, (uint64_t)cv.batch};
         uint64_t ks[2] = {(uint64_t)ctx->n * 2, (uint64_t)rows * ctx->n * 2};
         uint32_t kb[3] = {KC, TILE, 1};
@@ -625,7 +637,7 @@ cudaError_t lorc_tc_prefill_launch(lorc_ctx* ctx, const LorcLayer& L, const Cach
         if (!lorc_make_tmap_bf16(&mapV, vbuf, 3, kd, ks, kb)) return cudaErrorInvalidValue;
     }
     FaParams fp;
-    fp.out = out; fp.seq_lens = cv.seq_lens; fp.status = ctx->status_dev;
+    fp.out = out; fp.seq_lens = cv.seq_lens; fp.rope_table = ctx->rope_table; fp.status = ctx->status_dev;
     fp.T = T; fp.H_q = d.n_q_heads; fp.G = ctx->group; fp.n_rows = (int)rows; fp.max_pos = d.max_pos;
     const int qp = 2 * TILE / ctx->group;                      // query positions per CTA (two blocks of 128 rows)
     dim3 fgrid((T + qp - 1) / qp, d.n_kv_heads, cv.batch);
