@@ -870,6 +870,10 @@ def main():
         if not args.no_other_configs:
             try:
                 prefill = prefill_leg(L, shape, device, peaks, n_layers=min(4, shape.n_layers), chunk=1024, reps=1)
+                # the same prompts in one call per layer: the cached keys and values are reconstructed once, not per chunk
+                whole = prefill_leg(L, shape, device, peaks, n_layers=min(4, shape.n_layers), chunk=shape.context, reps=1)
+                prefill["one_call_per_prompt"] = {k: whole[k] for k in ("chunk", "append_ms", "attn_ms", "prompt_tokens_per_s",
+                                                                        "append", "attention")}
             except Exception as exc:
                 prefill = {"error": str(exc)[:200]}
         if not args.no_full_rank_leg:

@@ -253,7 +253,7 @@ struct FaSmem {
     bf16 K[F_STAGES][2][TILE * KC];       // key tile [128 keys][two halves]
     bf16 V[F_STAGES][2][TILE * KC];       // value tile [128 keys][two halves]
     uint64_t q_full, q_ready, k_full[F_STAGES], v_full[F_STAGES], k_empty[F_STAGES], v_empty[F_STAGES];
-    uint64_t s_full[2], p_ready[2], o_done;
+    uint64_t s_full[2], p_half[2], p_ready[2], o_done;
     uint32_t tmem_base;
 };
 
@@ -269,6 +269,22 @@ __device__ __forceinline__ float ex2_approx(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+
+// 32 scores of a row -> probabilities 2^(s - m), rounded to bf16 and packed two per column at tensor-memory address
+// taddr (16 columns); their unrounded sums are added to l0 / l1.  (Packed fp32 adds for the subtraction and the sums
+// were measured 2.5 % slower than these scalar ones: the pack / unpack moves cost more than the adds they save.)
+__device__ __forceinline__ void probs_chunk(const uint32_t (&r)[32], float m, uint32_t taddr, float& l0, float& l1) {
+    uint32_t w[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const float e0 = ex2_approx(__uint_as_float(r[2 * i]) - m), e1 = ex2_approx(__uint_as_float(r[2 * i + 1]) - m);
+        l0 += e0;
+        l1 += e1;
+        const __nv_bfloat162 pr = __floats2bfloat162_rn(e0, e1);
+        w[i] = *reinterpret_cast<const uint32_t*>(&pr);
+    }
+    tmem_st16(taddr, w);
 }
 
 __global__ void __launch_bounds__(F_THREADS, 1)
@@ -304,6 +320,7 @@ lorc_prefill_attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&sm.s_full[i], 1);
+            mbar_init(&sm.p_half[i], 4);
             mbar_init(&sm.p_ready[i], 4);
         }
         mbar_init(&sm.o_done, 1);
@@ -387,15 +404,26 @@ lorc_prefill_attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_
                 const uint32_t v0 = smem_u32(sm.V[st][0]);
 #pragma unroll 1
                 for (int b = 0; b < 2 && ok; ++b) {
-                    // the softmax warps of block b have replaced its scores by probabilities (and rescaled its output if needed)
-                    if (!mbar_wait(&sm.p_ready[b], j & 1)) { ok = false; break; }
+                    // the softmax warps of block b replace its scores by probabilities (and rescale its output first if
+                    // needed); they report the first 64 keys' worth and then the rest, so the first half of P V runs
+                    // while the second half of the exponentials is still being computed
+                    if (!mbar_wait(&sm.p_half[b], j & 1)) { ok = false; break; }
                     if (b == 0 && !mbar_wait(&sm.v_full[st], (j / F_STAGES) & 1)) { ok = false; break; }
                     tc_fence_after_sync();
                     if (elect_one()) {
 #pragma unroll
-                        for (int k = 0; k < 8; ++k)      // 16 keys per step: 8 columns of packed probabilities, 16 rows of V
+                        for (int k = 0; k < 4; ++k)      // 16 keys per step: 8 columns of packed probabilities, 16 rows of V
                             tc_mma_bf16_ts(tmem + 256 + b * 128, tmem + b * 128 + k * 8,
                                            make_smem_desc_sw128(v0 + k * 2048, TILE * KC * 2, 1024), idesc_o, (j | k) != 0);
+                    }
+                    __syncwarp();
+                    if (!mbar_wait(&sm.p_ready[b], j & 1)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    if (elect_one()) {
+#pragma unroll
+                        for (int k = 4; k < 8; ++k)
+                            tc_mma_bf16_ts(tmem + 256 + b * 128, tmem + b * 128 + k * 8,
+                                           make_smem_desc_sw128(v0 + k * 2048, TILE * KC * 2, 1024), idesc_o, 1);
                         if (b == 1) tc_commit(&sm.v_empty[st]);
                         if (b == 1 && j + 1 == n_tiles) tc_commit(&sm.o_done);
                     }
@@ -418,7 +446,7 @@ lorc_prefill_attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_
         const int pq = live ? len - p.T + t0 + tt : -1;          // this row's position: it sees keys 0 .. pq
         const uint32_t trow = tmem + ((uint32_t)(quarter * 32) << 16) + b * 128;   // scores / probabilities
         const uint32_t orow = tmem + ((uint32_t)(quarter * 32) << 16) + 256 + b * 128;
-        float m_ref = -INFINITY, l0 = 0.f, l1 = 0.f;
+        float m_ref = -INFINITY, l0 = 0.f, l1 = 0.f;      // l0 + l1: sum of the row's probabilities
         if (n_tiles > 0) {
             // Q^ = RoPE(q, position) * log2(e) / sqrt(d_h), fp16, in place: this thread's row of the block, 16 bytes at a
             // time.  The two 64-element halves of a row have the same swizzled layout, so a rotary pair (j, j + 64) sits
@@ -476,13 +504,16 @@ lorc_prefill_attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_
                     if (n0 + 96 + i > pq) r3[i] = 0xff800000u;
                 }
             }
-            float mt0 = -INFINITY, mt1 = -INFINITY;
+            // the row maximum: four independent chains
+            float mt0 = -INFINITY, mt1 = -INFINITY, mt2 = -INFINITY, mt3 = -INFINITY;
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                mt0 = fmaxf(mt0, fmaxf(__uint_as_float(r0[i]), __uint_as_float(r1[i])));
-                mt1 = fmaxf(mt1, fmaxf(__uint_as_float(r2[i]), __uint_as_float(r3[i])));
+            for (int i = 0; i < 32; i += 2) {
+                mt0 = max3(mt0, __uint_as_float(r0[i]), __uint_as_float(r0[i + 1]));
+                mt1 = max3(mt1, __uint_as_float(r1[i]), __uint_as_float(r1[i + 1]));
+                mt2 = max3(mt2, __uint_as_float(r2[i]), __uint_as_float(r2[i + 1]));
+                mt3 = max3(mt3, __uint_as_float(r3[i]), __uint_as_float(r3[i + 1]));
             }
-            const float mt = fmaxf(mt0, mt1);
+            const float mt = fmaxf(fmaxf(mt0, mt1), fmaxf(mt2, mt3));
             // raise the reference?  (the accesses to tensor memory below are warp-wide: the warp rescales if any of its
             // rows must, the other rows by a factor of one)
             const bool raise = mt > m_ref + F_RAISE || (m_ref == -INFINITY && mt > -INFINITY);
@@ -506,23 +537,14 @@ lorc_prefill_attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_
             }
             // probabilities (at most 2^8), rounded to bf16, packed two per column over the scores they came from
             const float m_use = m_ref == -INFINITY ? 0.f : m_ref;     // a row that has seen nothing yet: 2^(-inf) = 0
-            auto probs = [&](const uint32_t (&r)[32], int c0) {
-                uint32_t w[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const float e0 = ex2_approx(__uint_as_float(r[2 * i]) - m_use);
-                    const float e1 = ex2_approx(__uint_as_float(r[2 * i + 1]) - m_use);
-                    l0 += e0;
-                    l1 += e1;
-                    const __nv_bfloat162 pr = __floats2bfloat162_rn(e0, e1);
-                    w[i] = *reinterpret_cast<const uint32_t*>(&pr);
-                }
-                tmem_st16(trow + c0 / 2, w);
-            };
-            probs(r0, 0);
-            probs(r1, 32);
-            probs(r2, 64);
-            probs(r3, 96);
+            probs_chunk(r0, m_use, trow, l0, l1);
+            probs_chunk(r1, m_use, trow + 16, l0, l1);
+            tmem_wait_st();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.p_half[b]);
+            probs_chunk(r2, m_use, trow + 32, l0, l1);
+            probs_chunk(r3, m_use, trow + 48, l0, l1);
             tmem_wait_st();
             tc_fence_before_sync();
             __syncwarp();
