@@ -105,3 +105,22 @@ def test_prefill_with_one_token_equals_decode():
     assert O.rel_l2_rows(H.host_f64(out[:, 0]), want) <= TOL
     assert O.rel_l2_rows(H.host_f64(out[:, 0]), H.host_f64(dec)) <= TOL
     sess.close()
+
+
+@pytest.mark.parametrize("lens,T", [([300, 150], 45), ([200], 200)])
+def test_prefill_tensor_core_path_eight_heads_per_kv_head(lens, T):
+    """The 70B head geometry (64 query heads, 8 per KV head): a block of 128 query rows is 16 positions, a CTA covers 32;
+    T = 45 leaves the second block of the last CTA partly past the chunk."""
+    D, H_q, H_kv, d_h, r_k, r_v = 1024, 64, 8, 128, 160, 96
+    prob = H.Problem(D, H_q, H_kv, d_h, r_k, r_v, theta=500000.0, layer=25)
+    b, n_max = len(lens), max(lens) + 3
+    sess = H.Session(prob, max_pos=n_max, batch=b)
+    xs = [synth.hidden_states(int(L), D, 25, chunk=400 + s).astype(np.float64) for s, L in enumerate(lens)]
+    ck, cv = H.oracle_latents(prob, xs)
+    held = H.contiguous_cache(sess, b, n_max, lens, ck, cv)
+    for scale in (1.0, 8.0):
+        q = synth.to_bf16_exact(scale * synth.gaussian((b, T, H_q, d_h), 25, int(scale))).astype(np.float64)
+        out, ws = _run_prefill(sess, held[0], q, T, b, H_q, d_h, max(lens))
+        assert sess.L.lorc_last_path(sess.ctx) == 2, "the tensor-core path was not taken"
+        H.assert_rows_close(H.host_f64(out), _oracle_prefill(prob, ck, cv, q, T), TOL, (T, scale), elem_factor=4.0)
+    sess.close()
