@@ -17,7 +17,7 @@ tests/test_schedule.py, the context-shard functions by tests/test_sharded.py) to
 the mathematics fixes (full-rank identity, Eckart-Young, Theorem 1, RoPE closed
 forms, brute-force attention, a library attention routine).  The numeric
 tolerance used when comparing the GPU to this oracle is not from the paper
-(parity tolerance unpinned by the paper; fixed by the build's target).
+(parity tolerance unpinned by the paper; 1e-2 for bf16 operands with fp32 accumulation, 1e-5 for fp32 arithmetic).
 """
 from __future__ import annotations
 
@@ -38,7 +38,7 @@ def bf16_round(x: np.ndarray) -> np.ndarray:
     bfloat16 keeps 8 significant bits over the float32 exponent range, so the
     spacing at |x| in [2^e, 2^(e+1)) is 2^(e-7), with e floored at -126
     (subnormals).  Rounding is done straight from fp64 (no float32 detour).
-    The paper is silent on the cache precision; bf16 is the build's reading.
+    The paper is silent on the cache precision; bf16 is the reading taken here.
     """
     x = np.asarray(x, dtype=np.float64)
     _, ex = np.frexp(x)                      # x = m * 2^ex, 0.5 <= |m| < 1

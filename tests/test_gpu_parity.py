@@ -1,6 +1,6 @@
 """GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle.
 
-Tolerances (stated by the build's target, not by the paper): max over
+Tolerances (chosen for the arithmetic, not stated by the paper): max over
 (sequence, head) rows of ||gpu - oracle||_2 / ||oracle||_2 <= 1e-2 for the bf16 /
 fp32-accumulate path and <= 1e-5 for the fp32 debug path; the cache write within
 one bf16 unit in the last place of the exactly rounded latent.
