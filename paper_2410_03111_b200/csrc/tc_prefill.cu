@@ -7,9 +7,9 @@
 // kernel runs over that buffer.
 //
 //   reconstruct kernel  K^[tile, head] = RoPE(C_K[tile, :] . B_K[:, head]),  V[tile, head] = C_V[tile, :] . B_V[:, head]
-//                       persistent CTAs over (128-token tile, pair of KV heads): TMA-staged 64-wide slices, tcgen05
-//                       (M = 128 tokens, N = 256), rotation in the epilogue (thread = token row) under the next unit's
-//                       MMAs, 16-bit rows to the buffer: keys as
+//                       persistent CTA pairs over (two 128-token tiles, pair of KV heads): TMA-staged 64-wide slices,
+//                       tcgen05 cta_group::2 (M = 256 tokens, N = 256), rotation in the epilogue (thread = token row)
+//                       under the next unit's MMAs, 16-bit rows to the buffer: keys as
 //                       fp16 (the scores are then exact to 2^-11 of |q| |k|, four times closer than with bf16 keys;
 //                       a rotated key element must stay below 65504 in magnitude), values as bf16
 //   attention kernel    one CTA per two blocks of 128 query rows (128 / G positions x G heads of one KV head each); the
@@ -23,6 +23,7 @@
 #include <cuda_fp16.h>
 #include <math.h>
 
+#include "sm100_pair.cuh"
 #include "sm100_ptx.cuh"
 #include "tc_kernels.cuh"
 
@@ -37,18 +38,19 @@ constexpr float LOG2E = 1.4426950408889634f;
 // ------------------------------------------------------------------------------------------------
 // reconstruction of keys (rotated) or values into [b, n_rows, n] bf16
 // ------------------------------------------------------------------------------------------------
-// Persistent: a CTA walks units (sequence, 128-token tile, pair of KV heads) u = blockIdx.x, blockIdx.x + gridDim.x, ...
-// with the head pair running fastest (the CTAs that work on the same latent rows at the same time share them in L2).
-// Per unit  acc[128 tokens, 256 features] = C[tile, :] . B[:, 2 heads]  in 64-wide slices (M = 128, N = 256); the
-// accumulator is double-buffered in tensor memory, so the epilogue of one unit (rotation, rounding, 512-byte row
-// stores) runs under the MMAs of the next.
-constexpr int R_STAGES = 4;
-constexpr int R_THREADS = 192;       // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+// Persistent CTA PAIRS (clusters of two, cta_group::2 MMAs) walk units (sequence, pair of 128-token tiles, pair of KV
+// heads), the head pair running fastest (the pairs that work on the same latent rows at the same time share them in
+// L2).  Per unit  acc[256 tokens, 256 features] = C[tiles, :] . B[:, 2 heads]  in 64-wide slices: each CTA stages its
+// own 128 tokens and HALF of the factor slice (what a CTA can take in through TMA, not the MMA rate, bounds a
+// single CTA with the whole slice); the accumulator is double-buffered in tensor memory, so the epilogue of one unit
+// (rotation, rounding, 512-byte row stores of the CTA's own tokens) runs under the MMAs of the next.
+constexpr int R_STAGES = 6;
+constexpr int R_THREADS = 192;       // warp 0 TMA, warp 1 MMA (leader CTA issues), warps 2..5 epilogue
 constexpr int R_N = 256;             // features per unit: two KV heads
 
 struct RecSmem {
-    bf16 A[R_STAGES][TILE * KC];          // latent slice [128 tokens][64]
-    bf16 B[R_STAGES][R_N * KC];           // factor slice [256 features][64]
+    bf16 A[R_STAGES][TILE * KC];          // latent slice of this CTA's tile [128 tokens][64]
+    bf16 B[R_STAGES][TILE * KC];          // this CTA's half of the factor slice [128 features][64]
     uint64_t full[R_STAGES], empty[R_STAGES], acc_full[2], acc_empty[2];
     uint32_t tmem_base;
 };
@@ -59,28 +61,30 @@ struct RecParams {
     const int32_t* page_table;
     const float2* rope_table;      // [max_pos][64]
     int* status;
-    int r, n, n_rows, max_pos, batch, tiles, n_hp;
+    int r, n, n_rows, max_pos, batch, tile_pairs, n_hp;
     int page_size, max_pages_per_seq, n_pages;
 };
 
 template <bool ROPE>
-__global__ void __launch_bounds__(R_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(R_THREADS, 1)
 lorc_reconstruct_kernel(const __grid_constant__ CUtensorMap mapC, const __grid_constant__ CUtensorMap mapBT, const RecParams p) {
     extern __shared__ uint8_t raw[];
     RecSmem& sm = *reinterpret_cast<RecSmem*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
+    const int rank = (int)cluster_ctarank();           // 0 = leader (issues the MMAs, owns the full / acc_empty barriers)
+    const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     const int nkc = (p.r + KC - 1) / KC;
-    const int total = p.batch * p.tiles * p.n_hp;
-    // unit -> (sequence, tile, head pair); a unit whose tile lies past the sequence's cached tokens is skipped by
-    // every role alike (sequences beyond the buffer are reported by the attention kernel)
-    auto decode = [&](int u, int& s, int& tile, int& hp) -> bool {
+    const int total = p.batch * p.tile_pairs * p.n_hp;
+    // unit -> (sequence, tile pair, head pair); a unit whose first tile lies past the sequence's cached tokens is
+    // skipped by both CTAs and every role alike (sequences beyond the buffer are reported by the attention kernel)
+    auto decode = [&](int u, int& s, int& tp, int& hp, int& len) -> bool {
         hp = u % p.n_hp;
         const int st = u / p.n_hp;
-        tile = st % p.tiles;
-        s = st / p.tiles;
-        int len = p.seq_lens[s];
+        tp = st % p.tile_pairs;
+        s = st / p.tile_pairs;
+        len = p.seq_lens[s];
         if (len > p.max_pos || len > p.n_rows) len = 0;
-        return tile * TILE < len;
+        return 2 * tp * TILE < len;
     };
 
     if (tid == 0) {
@@ -90,35 +94,43 @@ lorc_reconstruct_kernel(const __grid_constant__ CUtensorMap mapC, const __grid_c
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&sm.acc_full[i], 1);
-            mbar_init(&sm.acc_empty[i], 4);
+            mbar_init(&sm.acc_empty[i], 2 * 4);             // one arrival per epilogue warp, both CTAs
         }
         fence_barrier_init();
         prefetch_tensormap(&mapC);
         prefetch_tensormap(&mapBT);
     }
     if (warp == 1) {
-        tmem_alloc(&sm.tmem_base, 512);
-        tmem_relinquish();
+        tmem_alloc_pair(&sm.tmem_base, 512);
+        tmem_relinquish_pair();
     }
     tc_fence_before_sync();
     __syncthreads();
+    cluster_arrive_release();                            // the peer's barriers are initialised before anyone signals them
+    cluster_wait_acquire();
     tc_fence_after_sync();
     const uint32_t tmem = sm.tmem_base;
     bool ok = true;
 
     if (warp == 0) {
-        uint32_t it = 0;                                         // stages issued so far
-        for (int u = blockIdx.x; u < total && ok; u += gridDim.x) {
-            int s, tile, hp;
-            if (!decode(u, s, tile, hp)) continue;
-            const int len = p.seq_lens[s];
-            for (int kc = 0; kc < nkc && ok; ++kc, ++it) {
-                const int st = it % R_STAGES;
-                if (!mbar_wait(&sm.empty[st], ((it / R_STAGES) & 1) ^ 1)) { ok = false; break; }
+        // ------------------------------------------------------------------ TMA producer (both CTAs)
+        const uint32_t a_base = smem_u32(sm.A[0]), b_base = smem_u32(sm.B[0]);
+        const uint32_t empty0 = smem_u32(&sm.empty[0]), full0 = smem_u32(&sm.full[0]);
+        const uint32_t lead_full0 = mapa_shared(full0, 0);   // all bytes of a stage are counted on the leader's barrier
+        uint32_t st = 0, par = 1;
+        for (int u = pair_id; u < total && ok; u += n_pairs) {
+            int s, tp, hp, len;
+            if (!decode(u, s, tp, hp, len)) continue;
+            const int tile = 2 * tp + rank;
+            for (int kc = 0; kc < nkc; ++kc) {
+                if (!mbar_wait_addr(empty0 + st * 8, par)) { ok = false; break; }
+                const uint32_t lead_bar = lead_full0 + st * 8;
+                const uint32_t a_dst = a_base + st * (TILE * KC * 2);
                 if (elect_one()) {
-                    mbar_arrive_expect_tx(&sm.full[st], (TILE + R_N) * KC * 2);
+                    if (rank == 0) mbar_arrive_expect_tx_addr(full0 + st * 8, 2 * 2 * TILE * KC * 2);
                     if (p.page_table == nullptr) {
-                        tma_load_3d(sm.A[st], &mapC, &sm.full[st], kc * KC, tile * TILE, s);
+                        // (a tile past the buffer's rows reads as zero)
+                        tma_load_3d_pair_addr(a_dst, &mapC, lead_bar, kc * KC, tile * TILE, s);
                     } else {
                         // one box per page; pages past the end of the sequence (or with a bad table entry) come from page 0
                         const int ppt = TILE / p.page_size;
@@ -132,57 +144,73 @@ lorc_reconstruct_kernel(const __grid_constant__ CUtensorMap mapC, const __grid_c
                                     page = 0;
                                 }
                             }
-                            tma_load_3d(sm.A[st] + pg * p.page_size * KC, &mapC, &sm.full[st], kc * KC, 0, page);
+                            tma_load_3d_pair_addr(a_dst + pg * p.page_size * KC * 2, &mapC, lead_bar, kc * KC, 0, page);
                         }
                     }
-                    tma_load_2d(sm.B[st], &mapBT, &sm.full[st], kc * KC, hp * R_N);
-                    tma_load_2d(sm.B[st] + TILE * KC, &mapBT, &sm.full[st], kc * KC, hp * R_N + 128);
+                    tma_load_2d_pair_addr(b_base + st * (TILE * KC * 2), &mapBT, lead_bar, kc * KC, hp * R_N + rank * 128);
                 }
                 __syncwarp();
+                if (++st == R_STAGES) { st = 0; par ^= 1; }
             }
         }
         if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
     } else if (warp == 1) {
-        const uint32_t idesc = make_idesc_bf16(128, R_N, 0, 0);
-        const int nk_last = (p.r - (nkc - 1) * KC + 15) >> 4;
-        uint32_t it = 0, uc = 0;
-        for (int u = blockIdx.x; u < total && ok; u += gridDim.x) {
-            int s, tile, hp;
-            if (!decode(u, s, tile, hp)) continue;
-            const int buf = uc & 1;
-            if (!mbar_wait(&sm.acc_empty[buf], ((uc >> 1) & 1) ^ 1)) { ok = false; break; }
-            tc_fence_after_sync();
-            for (int kc = 0; kc < nkc && ok; ++kc, ++it) {
-                const int st = it % R_STAGES;
-                if (!mbar_wait(&sm.full[st], (it / R_STAGES) & 1)) { ok = false; break; }
+        // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (rank == 0) {
+            const uint32_t idesc = make_idesc_bf16(256, R_N, 0, 0);
+            const int nk_last = (p.r - (nkc - 1) * KC + 15) >> 4;     // 16-column steps the last stage really holds
+            const uint64_t da0 = make_smem_desc_sw128(smem_u32(sm.A[0]), 0, 1024);
+            const uint64_t db0 = make_smem_desc_sw128(smem_u32(sm.B[0]), 0, 1024);
+            const uint32_t a_lo0 = (uint32_t)da0, a_hi = (uint32_t)(da0 >> 32);
+            const uint32_t b_lo0 = (uint32_t)db0, b_hi = (uint32_t)(db0 >> 32);
+            const uint32_t empty0 = smem_u32(&sm.empty[0]), full0 = smem_u32(&sm.full[0]);
+            uint32_t st = 0, par = 0, uc = 0;
+            for (int u = pair_id; u < total && ok; u += n_pairs) {
+                int s, tp, hp, len;
+                if (!decode(u, s, tp, hp, len)) continue;
+                const int buf = uc & 1;
+                if (!mbar_wait(&sm.acc_empty[buf], ((uc >> 1) & 1) ^ 1)) { ok = false; break; }
                 tc_fence_after_sync();
-                const uint32_t a0 = smem_u32(sm.A[st]), b0 = smem_u32(sm.B[st]);
-                if (elect_one()) {
-                    const int nk = (kc + 1 < nkc) ? 4 : nk_last;
-                    for (int k = 0; k < nk; ++k)
-                        tc_mma_bf16(tmem + buf * R_N, make_smem_desc_sw128(a0 + k * 32, 0, 1024),
-                                    make_smem_desc_sw128(b0 + k * 32, 0, 1024), idesc, (kc | k) != 0);
-                    tc_commit(&sm.empty[st]);
+                const uint32_t d = tmem + buf * R_N;
+                for (int kc = 0; kc < nkc; ++kc) {
+                    if (!mbar_wait_addr(full0 + st * 8, par)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t a_lo = a_lo0 + st * (TILE * KC * 2 / 16), b_lo = b_lo0 + st * (TILE * KC * 2 / 16);
+                    if (elect_one()) {
+                        if (kc == 0)
+                            tc_mma_bf16_pair_set(d, a_lo, a_hi, b_lo, b_hi, idesc);
+                        else
+                            tc_mma_bf16_pair_acc(d, a_lo, a_hi, b_lo, b_hi, idesc);
+                        const int nk = (kc + 1 < nkc) ? 4 : nk_last;
+                        if (nk > 1) tc_mma_bf16_pair_acc(d, a_lo + 2, a_hi, b_lo + 2, b_hi, idesc);
+                        if (nk > 2) tc_mma_bf16_pair_acc(d, a_lo + 4, a_hi, b_lo + 4, b_hi, idesc);
+                        if (nk > 3) tc_mma_bf16_pair_acc(d, a_lo + 6, a_hi, b_lo + 6, b_hi, idesc);
+                        tc_commit_pair_addr(empty0 + st * 8);        // frees the stage in both CTAs
+                    }
+                    __syncwarp();
+                    if (++st == R_STAGES) { st = 0; par ^= 1; }
                 }
+                if (!ok) break;
+                if (elect_one()) tc_commit_pair(&sm.acc_full[buf]);   // both CTAs' epilogues may read their accumulators
                 __syncwarp();
+                ++uc;
             }
-            if (!ok) break;
-            if (elect_one()) tc_commit(&sm.acc_full[buf]);
-            __syncwarp();
-            ++uc;
+            if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
         }
-        if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
     } else {
+        // ------------------------------------------------------------------ epilogue (both CTAs): this CTA's 128 tokens
         const int quarter = warp % 4;
         const int row = quarter * 32 + lane;                         // token of the tile = TMEM lane
+        const uint32_t lead_acc_empty[2] = {mapa_shared(smem_u32(&sm.acc_empty[0]), 0),
+                                            mapa_shared(smem_u32(&sm.acc_empty[1]), 0)};
         uint32_t uc = 0;
-        for (int u = blockIdx.x; u < total && ok; u += gridDim.x) {
-            int s, tile, hp;
-            if (!decode(u, s, tile, hp)) continue;
+        for (int u = pair_id; u < total && ok; u += n_pairs) {
+            int s, tp, hp, len;
+            if (!decode(u, s, tp, hp, len)) continue;
             const int buf = uc & 1;
             if (!mbar_wait(&sm.acc_full[buf], (uc >> 1) & 1)) { ok = false; break; }
             tc_fence_after_sync();
-            const int pos = tile * TILE + row;
+            const int pos = (2 * tp + rank) * TILE + row;
             const float2* cs = p.rope_table + (long long)min(pos, p.max_pos - 1) * 64;
 #pragma unroll 1
             for (int hd = 0; hd < 2; ++hd) {
@@ -227,14 +255,17 @@ lorc_reconstruct_kernel(const __grid_constant__ CUtensorMap mapC, const __grid_c
             // this warp has read its part of the accumulator
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.acc_empty[buf]);
+            if (lane == 0) mbar_arrive_cluster(lead_acc_empty[buf]);
             ++uc;
         }
         if (!ok && lane == 0) lorc_set_status(p.status, LORC_ERR_TIMEOUT);
     }
+    // both CTAs are done with tensor memory and with each other's barriers before either lets go
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem, 512);
+    cluster_arrive_release();
+    cluster_wait_acquire();
+    if (warp == 1) tmem_dealloc_pair(tmem, 512);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -633,9 +664,10 @@ cudaError_t lorc_tc_prefill_launch(lorc_ctx* ctx, const LorcLayer& L, const Cach
     rp.seq_lens = cv.seq_lens; rp.page_table = cv.page_table; rp.rope_table = ctx->rope_table; rp.status = ctx->status_dev;
     rp.n = ctx->n; rp.n_rows = (int)rows; rp.max_pos = d.max_pos;
     rp.page_size = cv.page_size; rp.max_pages_per_seq = cv.max_pages_per_seq; rp.n_pages = cv.n_pages;
-    rp.batch = cv.batch; rp.tiles = tiles; rp.n_hp = d.n_kv_heads / 2;
-    const int units = cv.batch * tiles * rp.n_hp;
-    dim3 rgrid(units < ctx->sm_count ? units : ctx->sm_count);
+    rp.batch = cv.batch; rp.tile_pairs = (tiles + 1) / 2; rp.n_hp = d.n_kv_heads / 2;
+    const int units = cv.batch * rp.tile_pairs * rp.n_hp;
+    const int pairs = units < ctx->sm_count / 2 ? units : ctx->sm_count / 2;
+    dim3 rgrid(2 * pairs);
     rp.out = khat; rp.r = L.r_k;
     lorc_reconstruct_kernel<true><<<rgrid, R_THREADS, sizeof(RecSmem) + 1024, st>>>(mapCK, mapBKT, rp);
     *launches += 1;
