@@ -287,6 +287,13 @@ int lorc_last_path(const lorc_ctx* ctx);
  * Without the flag it returns zeros. */
 int lorc_profile_read(lorc_ctx* ctx, float* ms, int64_t* launches);
 
+/* Self-test of the device-side bounded waits.  Every wait of every kernel of the library (on a shared-memory barrier
+ * that a copy or a tensor-core operation completes) runs through one routine with a time limit; when the limit runs out
+ * the kernel stops issuing work, sets the status word to LORC_ERR_TIMEOUT and returns.  This call launches a one-thread
+ * kernel that waits with that routine, with the limit given here (1 ns .. 1 s), on a barrier that nothing signals: the
+ * next lorc_sync_status returns LORC_ERR_TIMEOUT and the context stays usable.  Asynchronous on `stream`. */
+int lorc_selftest_wait_expiry(lorc_ctx* ctx, unsigned long long limit_ns, void* stream);
+
 /* Switches the event bracketing of LORC_FLAG_PROFILE on (on != 0) or off for the calls that
  * follow, on any context; while it is off the launches carry no events and may be captured
  * into a CUDA graph.  Events still pending are kept for the next lorc_profile_read.

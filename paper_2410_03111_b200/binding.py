@@ -71,6 +71,7 @@ def _signatures():
         "lorc_decode_attn_latent_out": ([vp, i32, cp, vp, vp, i32, vp], i32),
         "lorc_prefill_workspace_bytes": ([vp, i32, i32, i32], C.c_size_t),
         "lorc_prefill_attn": ([vp, i32, cp, vp, vp, i32, vp], i32),
+        "lorc_selftest_wait_expiry": ([vp, C.c_ulonglong, vp], i32),
         "lorc_decode_attn_shard": ([vp, i32, cp, vp, vp, vp, vp, vp, i32, vp], i32),
         "lorc_merge_shards": ([vp, i32, vp, vp, vp, i32, vp], i32),
         "lorc_decode_attn_static": ([vp, i32, cp, vp, vp, i32, vp], i32),
@@ -207,6 +208,10 @@ def lorc_decode_attn_static(ctx, layer, cache, q, out, n_splits=0, stream=None):
 def lorc_decode_step_host(ctx, layer, cache, x_host, q_host, out_host, n_splits=0, stream=None):
     _check(ctx, _lib.lorc_decode_step_host(ctx, layer, C.byref(cache), _ptr(x_host), _ptr(q_host),
                                             _ptr(out_host), n_splits, _stream(stream)))
+
+
+def lorc_selftest_wait_expiry(ctx, limit_ns, stream=None):
+    _check(ctx, _lib.lorc_selftest_wait_expiry(ctx, int(limit_ns), _stream(stream)))
 
 
 def lorc_sync_status(ctx, stream=None):

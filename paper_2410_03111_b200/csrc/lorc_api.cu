@@ -5,6 +5,7 @@
 #include <new>
 
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 #include "tc_kernels.cuh"
 
 namespace {
@@ -445,6 +446,31 @@ int lorc_decode_step_host(lorc_ctx* ctx, int layer, const lorc_cache* cache, con
     if (rc) return rc;
     e = cudaMemcpyAsync(out_host, out_d, qb, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "decode_step_host: device to host copy");
+    return LORC_OK;
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// Self-test of the bounded wait: one thread waits, with the library's own wait routine, on a barrier that nothing
+// ever signals; when the (short) limit runs out it reports LORC_ERR_TIMEOUT through the status word like any kernel
+// of the library would, and returns.
+// ---------------------------------------------------------------------------------------------------------------
+__global__ void wait_expiry_kernel(unsigned long long limit_ns, int* status) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        sm100::mbar_init(&bar, 1);
+        sm100::fence_barrier_init();
+        if (!sm100::mbar_wait_for(&bar, 0, limit_ns)) lorc_set_status(status, LORC_ERR_TIMEOUT);
+    }
+}
+
+int lorc_selftest_wait_expiry(lorc_ctx* ctx, unsigned long long limit_ns, void* stream) {
+    if (!ctx) return LORC_ERR_ARG;
+    if (limit_ns == 0 || limit_ns > 1000000000ull)
+        return fail(ctx, LORC_ERR_ARG, "selftest_wait_expiry: the limit must be between 1 ns and 1 s");
+    wait_expiry_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(limit_ns, ctx->status_dev);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "lorc_selftest_wait_expiry");
+    ctx->launches += 1;
     return LORC_OK;
 }
 

@@ -81,16 +81,20 @@ __device__ __forceinline__ void mbar_arrive_expect_tx_addr(uint32_t bar_addr, ui
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_addr), "r"(bytes) : "memory");
 }
 
-// Wait for the phase with the given parity to complete, for at most ~2 seconds.
-#define SM100_WAIT_LIMIT_NS 2000000000ull
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+// Wait for the phase with the given parity to complete, for at most limit_ns; false: the time ran out.
+__device__ __forceinline__ bool mbar_wait_for(uint64_t* bar, uint32_t parity, uint64_t limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
     uint32_t spins = 0;
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((++spins & 0x3ff) == 0 && global_timer_ns() - t0 > SM100_WAIT_LIMIT_NS) return false;
+        if ((++spins & 0x3ff) == 0 && global_timer_ns() - t0 > limit_ns) return false;
     }
+}
+// The limit every kernel of the library waits with: ~2 seconds.
+#define SM100_WAIT_LIMIT_NS 2000000000ull
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    return mbar_wait_for(bar, parity, SM100_WAIT_LIMIT_NS);
 }
 
 static __device__ __noinline__ bool mbar_wait_slow_addr(uint32_t bar_addr, uint32_t parity) {
