@@ -925,6 +925,11 @@ def main():
             "clocks": clocks, "gpu_launches": launches,
         }
         line["decode_attn"].update({"achieved_tflops": achieved, "flops_per_step": flops, "bytes_per_step": byts})
+        sm, sm_max = (clocks or {}).get("sm_mhz"), (clocks or {}).get("sm_max_mhz")
+        if sm and sm_max and t_burst >= t_hbm:
+            # context, not the headline: the same fraction if the burst peak scaled with the SM clock that was sampled
+            # under load (it was measured in a short burst, before the power cap pulls the clock down)
+            line["decode_attn"]["frac_burst_at_sampled_clock"] = (t_burst / attn_s) * sm_max / sm
         if score_prof:
             # lorc_score_kernel: key reconstruction C_K.B_K on the tensor cores, RoPE, q.k and the softmax numerators in
             # its epilogue.  Algorithmic FLOPs per launch = cached tokens * (2 r_k n + 2 H_q d_h), mean over the layers.
