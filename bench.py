@@ -760,7 +760,8 @@ def main():
     total_steps = args.warmup + args.steps + e2e_steps + 4
     rope = args.rope == "half"
     do_oracle = (not args.no_cpu_baseline) and rank == 0 and world == 1 and not args.full_rank and rope
-    oracle_layers = sorted(set([0, n_layers // 2, n_layers - 1])) if do_oracle else []
+    # about ten layers spread over the stack (their ranks span the schedule); every sequence of each is redone
+    oracle_layers = sorted(set(round(i * (n_layers - 1) / 9) for i in range(10))) if do_oracle else []
     wl = Workload(L, shape, n_layers, total_steps, device, flags, full_rank=args.full_rank,
                   seeded_cache=bool(shape.paged or shape.ragged[1] > 0), keep_layers=oracle_layers, rope=rope)
     b = shape.batch
