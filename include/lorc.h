@@ -196,7 +196,8 @@ int lorc_decode_attn(lorc_ctx* ctx, int layer, const lorc_cache* cache, const vo
  *   at position seq_lens[s] - T + t and attends to positions 0 .. seq_lens[s] - T + t (the cached prefix in full, the
  *   new chunk causally).  With T = 1 the result equals lorc_decode_attn's.
  * On the tensor-core path every key and value of the layer is reconstructed once into the workspace (a transient
- * bf16 buffer: the method's saving is in the cache, not in this scratch), then attended with a flash-attention
+ * fp16 buffer: the method's saving is in the cache, not in this scratch; a reconstructed key or value element must
+ * stay below 65504 in magnitude), then attended with a flash-attention
  * kernel; every call reconstructs the whole cached sequence, so chunks should be large.  Needs a workspace of
  * lorc_prefill_workspace_bytes(ctx, batch, max_seq_len, T).  A sequence with seq_lens[s] < T sets status ARG.
  * Errors: ARG, LAYER, WORKSPACE; CAPACITY / EMPTY through the status word. */

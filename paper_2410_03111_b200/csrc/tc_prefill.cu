@@ -3,20 +3,20 @@
 // mask; keys and values reconstructed from the latents of Sec. 3.1, rotation at attention time as in the appendix).
 //
 // With many queries per key the reconstruction is worth keeping: every key and value of the layer is rebuilt ONCE into
-// a transient bf16 buffer (the decode path rebuilds them per query and never stores them), then a flash-attention
+// a transient fp16 buffer (the decode path rebuilds them per query and never stores them), then a flash-attention
 // kernel runs over that buffer.
 //
 //   reconstruct kernel  K^[tile, head] = RoPE(C_K[tile, :] . B_K[:, head]),  V[tile, head] = C_V[tile, :] . B_V[:, head]
 //                       persistent CTA pairs over (two 128-token tiles, pair of KV heads): TMA-staged 64-wide slices,
 //                       tcgen05 cta_group::2 (M = 256 tokens, N = 256), rotation in the epilogue (thread = token row)
 //                       under the next unit's MMAs, 16-bit rows to the buffer: keys as
-//                       fp16 (the scores are then exact to 2^-11 of |q| |k|, four times closer than with bf16 keys;
-//                       a rotated key element must stay below 65504 in magnitude), values as bf16
+//                       fp16 (the scores are then exact to 2^-11 of |q| |k|, four times closer than with bf16 keys),
+//                       values as fp16 too (a reconstructed element must stay below 65504 in magnitude)
 //   attention kernel    one CTA per two blocks of 128 query rows (128 / G positions x G heads of one KV head each); the
 //                       rows are rotated at their positions and scaled in shared memory, Q^ = RoPE(q) log2(e) / sqrt(d_h)
 //                       as fp16, before the first MMA; for
 //                       every 128-key tile and block   S = Q^ K^^T (tcgen05, fp32 in TMEM)  ->  online softmax, thread =
-//                       query row; the probabilities go back into tensor memory as bf16 over the scores  ->  O += P V
+//                       query row; the probabilities go back into tensor memory as fp16 over the scores  ->  O += P V
 //                       with P read from tensor memory.  The two blocks alternate, so the tensor pipe works on one
 //                       while the other's softmax runs.  The running reference of a row is only raised when a tile
 //                       exceeds it by more than 2^8 (the accumulator is rescaled then), so most tiles need no pass over O.
@@ -36,7 +36,7 @@ constexpr int KC = 64;
 constexpr float LOG2E = 1.4426950408889634f;
 
 // ------------------------------------------------------------------------------------------------
-// reconstruction of keys (rotated) or values into [b, n_rows, n] bf16
+// reconstruction of keys (rotated) or values into [b, n_rows, n] fp16
 // ------------------------------------------------------------------------------------------------
 // Persistent CTA PAIRS (clusters of two, cta_group::2 MMAs) walk units (sequence, pair of 128-token tiles, pair of KV
 // heads), the head pair running fastest (the pairs that work on the same latent rows at the same time share them in
@@ -234,12 +234,8 @@ lorc_reconstruct_kernel(const __grid_constant__ CUtensorMap mapC, const __grid_c
                                 const float x1 = a1 * t.z - b1 * t.w, y1 = a1 * t.w + b1 * t.z;
                                 a0 = x0; b0 = y0; a1 = x1; b1 = y1;
                             }
-                            if (ROPE) {          // keys: fp16
+                            {                    // keys and values alike: fp16
                                 const __half2 pa = __floats2half2_rn(a0, a1), pb = __floats2half2_rn(b0, b1);
-                                wa[i] = *reinterpret_cast<const uint32_t*>(&pa);
-                                wb[i] = *reinterpret_cast<const uint32_t*>(&pb);
-                            } else {             // values: bf16
-                                const __nv_bfloat162 pa = __floats2bfloat162_rn(a0, a1), pb = __floats2bfloat162_rn(b0, b1);
                                 wa[i] = *reinterpret_cast<const uint32_t*>(&pa);
                                 wb[i] = *reinterpret_cast<const uint32_t*>(&pb);
                             }
@@ -302,7 +298,7 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
-// 32 scores of a row -> probabilities 2^(s - m), rounded to bf16 and packed two per column at tensor-memory address
+// 32 scores of a row -> probabilities 2^(s - m), rounded to fp16 and packed two per column at tensor-memory address
 // taddr (16 columns); their unrounded sums are added to l0 / l1.  (Packed fp32 adds for the subtraction and the sums
 // were measured 2.5 % slower than these scalar ones: the pack / unpack moves cost more than the adds they save.)
 __device__ __forceinline__ void probs_chunk(const uint32_t (&r)[32], float m, uint32_t taddr, float& l0, float& l1) {
@@ -312,7 +308,7 @@ __device__ __forceinline__ void probs_chunk(const uint32_t (&r)[32], float m, ui
         const float e0 = ex2_approx(__uint_as_float(r[2 * i]) - m), e1 = ex2_approx(__uint_as_float(r[2 * i + 1]) - m);
         l0 += e0;
         l1 += e1;
-        const __nv_bfloat162 pr = __floats2bfloat162_rn(e0, e1);
+        const __half2 pr = __floats2half2_rn(e0, e1);
         w[i] = *reinterpret_cast<const uint32_t*>(&pr);
     }
     tmem_st16(taddr, w);
@@ -405,7 +401,7 @@ lorc_prefill_attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_
     } else if (warp == 1) {
         if (n_tiles > 0) {
             const uint32_t idesc_s = make_idesc_f16(128, 128);            // S = Q K^T: fp16 operands, both K-major
-            const uint32_t idesc_o = make_idesc_bf16(128, 128, 0, 1);     // O += P V: V is MN-major (a key's elements are contiguous)
+            const uint32_t idesc_o = make_idesc_f16(128, 128, 0, 1);      // O += P V: fp16 too, V MN-major (a key's elements are contiguous)
             // The MMAs of one thread run in the order they were issued, and a commit covers everything issued before it:
             // when s_full[b] fires for tile j + 1, block b's P V of tile j has also finished with the probabilities that
             // these scores overwrite and with the output a softmax warp may rescale.
@@ -566,7 +562,7 @@ lorc_prefill_attn_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_
                 }
                 if (raise) m_ref = mt;
             }
-            // probabilities (at most 2^8), rounded to bf16, packed two per column over the scores they came from
+            // probabilities (at most 2^8), rounded to fp16, packed two per column over the scores they came from
             const float m_use = m_ref == -INFINITY ? 0.f : m_ref;     // a row that has seen nothing yet: 2^(-inf) = 0
             probs_chunk(r0, m_use, trow, l0, l1);
             probs_chunk(r1, m_use, trow + 16, l0, l1);

@@ -75,15 +75,17 @@ def test_prefill_tensor_core_path(r_k, r_v, lens, T, paged, style):
     else:
         held = H.contiguous_cache(sess, b, n_max, lens, ck, cv)
     worst = 0.0
-    # (query scale 8 is the benchmark's; the keys are materialised in fp16, so much more peaked softmaxes than that
-    # see the keys' rounding: 2^-11 of |q| |k| per score)
-    for scale in (1.0, 8.0):
+    # (the keys are materialised in fp16: a score carries their rounding, 2^-11 of |q| |k|, which the most peaked
+    # softmaxes here see)
+    for scale in (1.0, 8.0, 64.0):
         q = synth.to_bf16_exact(scale * synth.gaussian((b, T, GEOM["H_q"], GEOM["d_h"]), 23, int(scale))).astype(np.float64)
         out, ws = _run_prefill(sess, held[0], q, T, b, GEOM["H_q"], GEOM["d_h"], max(lens))
         assert sess.L.lorc_last_path(sess.ctx) == 2, "the tensor-core path was not taken"
         got = H.host_f64(out)
         want = _oracle_prefill(prob, ck, cv, q, T)
-        H.assert_rows_close(got, want, TOL, (r_k, T, scale), elem_factor=4.0)
+        # (at scale 64 the error level is 6e-3 of a row and the outputs have up to two million elements: the
+        # largest of so many needs the wider element bound)
+        H.assert_rows_close(got, want, TOL, (r_k, T, scale), elem_factor=4.0 if scale > 8 else 2.0)
         worst = max(worst, O.rel_l2_rows(got, want))
     print(f"\n[prefill] r_k {r_k}, T {T}, lens {lens}: max relative L2 row error {worst:.2e}")
     sess.close()
@@ -122,5 +124,5 @@ def test_prefill_tensor_core_path_eight_heads_per_kv_head(lens, T):
         q = synth.to_bf16_exact(scale * synth.gaussian((b, T, H_q, d_h), 25, int(scale))).astype(np.float64)
         out, ws = _run_prefill(sess, held[0], q, T, b, H_q, d_h, max(lens))
         assert sess.L.lorc_last_path(sess.ctx) == 2, "the tensor-core path was not taken"
-        H.assert_rows_close(H.host_f64(out), _oracle_prefill(prob, ck, cv, q, T), TOL, (T, scale), elem_factor=4.0)
+        H.assert_rows_close(H.host_f64(out), _oracle_prefill(prob, ck, cv, q, T), TOL, (T, scale))
     sess.close()
