@@ -66,6 +66,9 @@ struct Pv2Params {
     int page_size, max_pages_per_seq, n_pages;
 };
 
+// Biased exponent of 2^d for an integer-valued d <= 0 (0, i.e. the number zero, below 2^-126 and for d = -inf).
+__device__ __forceinline__ uint32_t pow2_exponent(float d) { return d >= -126.f ? (uint32_t)(127 + (int)d) : 0u; }
+
 template <int HQ>
 __global__ void __launch_bounds__(P_THREADS, 1)
 lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
@@ -230,6 +233,7 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
         const int frow = (t * 2 * HQ) >> 7;               // row of the image: chunk * HQ + head
         const int fchunk = frow / HQ, fh = frow % HQ;
         const int fpiece0 = ((t * 2 * HQ) & 127) >> 4;    // first 16-byte piece (physical) of this thread
+        const int frot = HQ == 32 ? (t >> 1) & 3 : t & 7;  // rotation of the order in which it takes its pieces
         const float m_mine = sm.m_row[fh];
         const int lh = t % HQ, lpart = t / HQ;            // denominator: head, and which quarters of a tile
         const float m_l = sm.m_row[lh];
@@ -242,21 +246,32 @@ lorc_pv2_kernel(const __grid_constant__ CUtensorMap mapCV, const Pv2Params p) {
 #pragma unroll
             for (int qq = 0; qq < 4 / PARTS; ++qq) {
                 const int qrt = lpart * (4 / PARTS) + qq;
-                const float mq = mt[qrt * HQ + lh];
-                lacc += mq > -INFINITY ? lt[qrt * HQ + lh] * exp2f(fmaxf(mq - m_l, -126.f)) : 0.f;
+                lacc += lt[qrt * HQ + lh] * __uint_as_float(pow2_exponent(mt[qrt * HQ + lh] - m_l) << 23);
+            }
+            // 2^(m - M) of the quarter(s) this thread's pieces belong to, as a bf16 pair (built from the exponent: m and M
+            // are integers).  A piece's quarter is bit 2 of its logical index, physical index xor (head & 7).
+            uint32_t scb[2];
+#pragma unroll
+            for (int hq = 0; hq < 2; ++hq) {
+                const uint32_t e = pow2_exponent(mt[(fchunk * 2 + hq) * HQ + fh] - m_mine) << 7;
+                scb[hq] = e | (e << 16);
             }
             uint4* prow = reinterpret_cast<uint4*>(sm.P[st] + frow * 128);
+            constexpr int NP = (2 * HQ) / 16;                 // 16-byte pieces per thread: 4 or 8
+            uint4 v[NP];
+            // (the pieces are taken in an order rotated by the thread index: the threads of a quarter warp, whose
+            // pieces lie 64 or 128 bytes apart, then touch different banks)
 #pragma unroll
-            for (int j = 0; j < (2 * HQ) / 16; ++j) {
-                const int pp = fpiece0 + j;
-                const int qrt = fchunk * 2 + ((pp ^ (fh & 7)) >> 2);
-                const float mq = mt[qrt * HQ + fh];
-                const __nv_bfloat162 sc = __float2bfloat162_rn(mq > -INFINITY ? exp2f(fmaxf(mq - m_mine, -126.f)) : 0.f);
-                uint4 v = prow[pp];
-                __nv_bfloat162* e = reinterpret_cast<__nv_bfloat162*>(&v);
+            for (int j = 0; j < NP; ++j) v[j] = prow[fpiece0 + ((j + frot) & (NP - 1))];
+#pragma unroll
+            for (int j = 0; j < NP; ++j) {
+                const int pp = fpiece0 + ((j + frot) & (NP - 1));
+                const uint32_t sb = scb[((pp ^ (fh & 7)) >> 2) & 1];
+                const __nv_bfloat162 sc = *reinterpret_cast<const __nv_bfloat162*>(&sb);
+                __nv_bfloat162* e = reinterpret_cast<__nv_bfloat162*>(&v[j]);
 #pragma unroll
                 for (int k = 0; k < 4; ++k) e[k] = __hmul2(e[k], sc);
-                prow[pp] = v;
+                prow[pp] = v[j];
             }
             fence_proxy_async_smem();      // the MMA reads the image through the asynchronous proxy
             __syncwarp();
