@@ -106,6 +106,13 @@ __device__ __forceinline__ void decode_unit(const ScoreSmem& sm, Walk& w, int ra
 // Float index of query head g, pair j, component `half` (0: first half of the head, 1: second) in qrot[][].  One
 // 16-byte piece holds two heads x the thread's two adjacent pairs (e = j & 1), i.e. two packed-fp32 operands; the four
 // c of equal (kk, half, g / 2) are neighbouring pieces, one conflict-free shared-memory access.
+// 2^x for x <= 0 on the special-function unit (relative error 2^-22; the result is rounded to bf16 anyway).
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 template <int G>
 __device__ __forceinline__ int qrot_index(int j, int half, int g) {
     const int kk = j >> 3, c = (j >> 1) & 3, e = j & 1;
@@ -456,7 +463,7 @@ lorc_score_kernel(const __grid_constant__ CUtensorMap mapCK, const __grid_consta
                 for (int m = 0; m < 4; ++m) {
                     const bool valid = n_first + 8 * m < un.len;
                     // p = 2^(s - m), rounded to bf16 (the same rounded value enters the denominator)
-                    const bf16 pr = __float2bfloat16_rn(valid ? exp2f(tot[m][i] - mref) : 0.f);
+                    const bf16 pr = __float2bfloat16_rn(valid ? ex2_approx(tot[m][i] - mref) : 0.f);
                     lsum += __bfloat162float(pr);
                     const int tc = tc0 + 8 * m;
                     *reinterpret_cast<bf16*>(chunk_img + h * 128 + ((((tc >> 3) ^ (h & 7)) << 4) | ((tc & 7) << 1))) = pr;
