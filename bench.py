@@ -63,7 +63,7 @@ def parse_args():
 # DRAM traffic of one lorc_score_kernel launch from an ncu capture of the CURRENT kernel (rank, batch and context of the
 # captured launch; the read traffic is the latent keys, which grow with rank, batch and context, the written traffic
 # the probability images, which grow with batch and context only).  None: no capture of the current kernel yet.
-SCORE_KERNEL_TRAFFIC = {"rank": 928, "batch": 16, "context": 4100, "read_bytes": 123.28e6, "write_bytes": 6.54e6}
+SCORE_KERNEL_TRAFFIC = {"rank": 928, "batch": 16, "context": 4100, "read_bytes": 123.31e6, "write_bytes": 6.72e6}
 
 
 def load_peaks():
