@@ -172,3 +172,53 @@ def test_random_context_cuts_merge_to_the_whole(seed):
     want = H.oracle_decode(prob, ck, cv, q)
     assert O.rel_l2_rows(H.host_f64(merged), want) <= 1.5 * TOL, (seed, cuts)
     sess.close()
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_random_cache_write_equals_oracle_rows(seed):
+    """lorc_append at random token counts (one token: the decode kernel; 128 and more per launch: the tcgen05 GEMM), ranks,
+    prefixes and cache layouts: every written row within one bf16 ulp of the exactly rounded latent, rows before and
+    after the written range untouched."""
+    import torch
+    rng = np.random.default_rng(4000 + seed)
+    H_q, H_kv = [(32, 8), (64, 8)][seed % 2]
+    r_k, r_v = int(rng.integers(1, 129)) * 8, int(rng.integers(1, 129)) * 8
+    b = int(rng.integers(1, 5))
+    T = [1, 1, 3, 16, 40, 128, 130, 200, 257, 64][seed]
+    prefix = [int(x) for x in rng.integers(0, 300, size=b)]
+    lens = [p + T for p in prefix]
+    paged = seed % 3 == 1
+    page_size = [16, 32, 64, 128][seed % 4]
+    prob = _problem(H_q, H_kv, r_k, r_v, 40 + seed % 4)
+    n_max = max(lens) + 3
+    L = H.lib()
+    sess = H.Session(prob, max_pos=n_max, batch=b)
+    x = np.stack([synth.hidden_states(T, prob.D, 44, chunk=10 * seed + s) for s in range(b)]).astype(np.float64)
+    if paged:
+        held = H.paged_cache(sess, b, lens, page_size, order_seed=seed)
+    else:
+        held = H.contiguous_cache(sess, b, n_max, lens)
+    held[1].fill_(3.0)                   # whatever is not written must keep this
+    held[2].fill_(3.0)
+    L.lorc_append(sess.ctx, 0, held[0], H.dev_bf16(x), T=T)
+    assert L.lorc_sync_status(sess.ctx) == 0, L.lorc_last_error(sess.ctx)
+    kk, vv = H.host_f64(held[1]), H.host_f64(held[2])
+    for s in range(b):
+        want_k = O.append_latent_bf16(x[s], prob.A_k)
+        want_v = O.append_latent_bf16(x[s], prob.A_v)
+        exact_k, exact_v = O.append_latent(x[s], prob.A_k), O.append_latent(x[s], prob.A_v)
+        for t in range(T):
+            pos = prefix[s] + t
+            if paged:
+                page = int(held[5][s, pos // page_size])
+                row_k, row_v = kk[page, pos % page_size], vv[page, pos % page_size]
+            else:
+                row_k, row_v = kk[s, pos], vv[s, pos]
+            # one ulp of the rounded value, plus the fp32 accumulation bound where the terms cancel
+            for got, want, exact, A in ((row_k, want_k[t], exact_k[t], prob.A_k), (row_v, want_v[t], exact_v[t], prob.A_v)):
+                slack = 2.0 ** -16 * (np.abs(x[s][t])[:, None] * np.abs(A)).sum(0)
+                assert np.all(np.abs(got - want) <= H.bf16_ulp(want) + slack), (seed, s, t)
+        if not paged:
+            assert np.all(kk[s, :prefix[s]] == 3.0) and np.all(kk[s, lens[s]:] == 3.0)
+            assert np.all(vv[s, :prefix[s]] == 3.0) and np.all(vv[s, lens[s]:] == 3.0)
+    sess.close()
